@@ -1,0 +1,306 @@
+"""Pins for the oracle: every check here compares it with something other than itself.
+
+ * the paper's token-graph picture of visibility on an interleaved token-granular pool
+   (Section 3 "Efficiency", Fig. 2b/2c) evaluated as a dense masked softmax;
+ * the naive batched layout of Appendix B (duplicated prefix, chunks copied in at sync);
+ * the worked example of Section 3 (pool indices and can / cannot attend facts);
+ * plain causal decode when no thread is ever spawned (a library attention routine);
+ * closed forms and invariants of softmax attention.
+"""
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import KVStore, OracleReplay, PoolModel, attend, decode_attention
+from pasta_workloads import Geometry, Script, cfg1_tiny, cfg2_single_request, random_script
+from formulations import NaiveRows, TokenGraph
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def manual_script(ops, geo=None, n_pages=64, seed=7, free_order=None):
+    geo = geo or Geometry(1, 4, 2, 8, 4)
+    order = np.arange(n_pages, dtype=np.int32) if free_order is None else np.asarray(free_order, dtype=np.int32)
+    return Script("manual", geo, n_pages, order, 8, 16, 64, seed, list(ops))
+
+
+def oracle_outputs(script):
+    return {i: r[0] for i, r in OracleReplay(script).run_all().items()}
+
+
+# ------------------------------------------------------------------ other formulations
+@pytest.mark.parametrize("seed", range(12))
+@pytest.mark.parametrize("paper_flow", [True, False])
+def test_token_graph_formulation_agrees(seed, paper_flow):
+    script = random_script(seed, paper_flow=paper_flow)
+    ours = oracle_outputs(script)
+    theirs = TokenGraph(script).run_all()
+    assert ours.keys() == theirs.keys() and ours
+    for i in ours:
+        np.testing.assert_allclose(ours[i][0], theirs[i][0], rtol=0, atol=1e-12)
+        np.testing.assert_allclose(ours[i][1], theirs[i][1], rtol=0, atol=1e-12)
+
+
+@pytest.mark.parametrize("seed", range(12, 24))
+def test_naive_batched_layout_agrees(seed):
+    script = random_script(seed, n_ops=80)
+    ours = oracle_outputs(script)
+    theirs = NaiveRows(script).run_all()
+    assert ours.keys() == theirs.keys()
+    for i in ours:
+        np.testing.assert_allclose(ours[i][0], theirs[i][0], rtol=0, atol=1e-12)
+        np.testing.assert_allclose(ours[i][1], theirs[i][1], rtol=0, atol=1e-12)
+
+
+@pytest.mark.parametrize("variant", ["base", "cutoffs", "chunk16", "chunk33", "append"])
+def test_tiny_config_all_formulations(variant):
+    script = cfg1_tiny(variant)
+    ours = oracle_outputs(script)
+    for other in (TokenGraph(script).run_all(), NaiveRows(script).run_all()):
+        for i in ours:
+            np.testing.assert_allclose(ours[i][0], other[i][0], rtol=0, atol=1e-12)
+
+
+# ------------------------------------------------------------------ the paper's worked example
+def _read_fig2():
+    tokens, withheld, facts = [], [], []
+    with open(os.path.join(GOLDEN, "fig2_worked_example.txt")) as f:
+        for line in f:
+            line = line.split("#")[0].split()
+            if not line:
+                continue
+            if line[0] == "token":
+                tokens.append((line[1], line[2], int(line[3]), int(line[4]), line[5]))
+            elif line[0] == "withheld":
+                withheld.append(line[1])
+            else:
+                facts.append((line[0], line[1], line[2]))
+    return tokens, withheld, facts
+
+
+def test_fig2_worked_example():
+    tokens, withheld, facts = _read_fig2()
+    thread_id = {"main": 0, "fork1": 1, "fork2": 2}
+    # the operations the text describes, timestamp by timestamp
+    ops = [("begin", 0), ("run", 0, 0, 19),                     # the part of the user query before T=0
+           ("run", 0, 0, 2),                                    # T=0: main appends two tokens
+           ("step", ((0, 0, 1),)), ("spawn", 0, 1),             # T=1: <promise/> #1, Fork#1 is created ...
+           ("run", 0, 1, 1),                                    # ... and receives its <async> token
+           ("step", ((0, 1, 1), (0, 0, 1))), ("spawn", 0, 2),   # T=2: Fork#1 "To", main <promise/> #2
+           ("run", 0, 2, 1),                                    #      Fork#2 receives its <async> token
+           ("step", ((0, 1, 1), (0, 2, 1)))]                    # T=3: both forks decode; <sync/> is withheld
+    script = manual_script(ops)
+    # (thread, per-thread token index) of every labelled token
+    nth = {}
+    count = {0: 19, 1: 0, 2: 0}
+    for label, thread, _T, _i, _how in tokens:
+        t = thread_id[thread]
+        nth[label] = (t, count[t]); count[t] += 1
+
+    # --- token-graph pool: the slot indices are those of the text
+    graph = TokenGraph(script)
+    graph.run_all()
+    slot_of = {}
+    seen = {0: 0, 1: 0, 2: 0}
+    for slot, (_req, t) in enumerate(graph.owner):
+        slot_of[(t, seen[t])] = slot; seen[t] += 1
+    by_T = {}
+    for label, thread, T, i, _how in tokens:
+        by_T.setdefault(T, (set(), set()))
+        by_T[T][0].add(i); by_T[T][1].add(slot_of[nth[label]])
+    for T, (want, got) in by_T.items():
+        assert want == got, (T, want, got)      # order inside one timestamp is not fixed by the text
+    assert len(graph.k) == 28                   # next free index is 28; the withheld <sync/> took none
+
+    # --- visibility facts, in both formulations
+    replay = OracleReplay(script)
+    replay.run_all()
+    model = replay.model
+
+    def oracle_sees(label):
+        t, _ = nth[label]
+        pages = {s: model.requests[0].stream_pages[s] for s in (0, 1, 2)}
+        P = model.page_size
+        vis = set(model.visible_slots(0, t))
+        return lambda other: (pages[nth[other][0]][nth[other][1] // P], nth[other][1] % P) in vis
+
+    def graph_sees(label):
+        t, _ = nth[label]
+        vis = set(graph.visible((0, t)))
+        return lambda other: slot_of[nth[other]] in vis
+
+    for verdict, who, what in facts:
+        if what in withheld:
+            assert verdict == "cannot"          # it is in no pool at all
+            continue
+        for sees in (oracle_sees(who), graph_sees(who)):
+            assert sees(what) == (verdict == "can"), (verdict, who, what)
+
+
+# ------------------------------------------------------------------ reduces to a library routine
+def test_no_forks_is_plain_causal_decode():
+    geo = Geometry(1, 8, 2, 16, 4)
+    ops = [("begin", 0), ("run", 0, 0, 37)] + [("step", ((0, 0, 1),)) for _ in range(3)]
+    script = manual_script(ops, geo=geo, free_order=np.random.default_rng(0).permutation(64))
+    replay = OracleReplay(script)
+    ks, vs = [], []
+    from pasta_workloads import run_tensors, step_tensors
+    for i, op in enumerate(script.ops):
+        if op[0] == "run":
+            k, v = run_tensors(script, i, 0); ks.append(k); vs.append(v)
+            replay.apply(i)
+        elif op[0] == "step":
+            k, v, q = step_tensors(script, i, 0); ks.append(k); vs.append(v)
+            out, lse = replay.apply(i)[0]
+            K = torch.cat(ks).double().permute(1, 0, 2)      # [Hkv, n, d]
+            V = torch.cat(vs).double().permute(1, 0, 2)
+            K = K.repeat_interleave(geo.group, dim=0); V = V.repeat_interleave(geo.group, dim=0)
+            ref = torch.nn.functional.scaled_dot_product_attention(
+                q.double().permute(1, 0, 2), K, V)           # [Hq, 1, d]
+            np.testing.assert_allclose(out[0], ref[:, 0].numpy(), rtol=0, atol=1e-12)
+        else:
+            replay.apply(i)
+
+
+# ------------------------------------------------------------------ closed forms
+def _store_with(k, v, page_size=4):
+    n, hkv, d = k.shape
+    n_pages = -(-n // page_size) + 3
+    model = PoolModel(n_pages, page_size, np.random.default_rng(1).permutation(n_pages))
+    store = KVStore(n_pages, page_size, hkv, d)
+    req = model.request_begin()
+    store.write(model.append_run(req, 0, n), k, v)
+    return model, store, req
+
+
+def test_closed_forms():
+    rng = np.random.default_rng(5)
+    n, hkv, hq, d = 23, 2, 6, 8
+    q = rng.standard_normal((1, hq, d))
+    v = rng.standard_normal((n, hkv, d)).astype(np.float32)
+    # equal keys -> uniform weights -> mean of V
+    k = np.broadcast_to(rng.standard_normal((1, hkv, d)), (n, hkv, d)).astype(np.float32)
+    model, store, req = _store_with(k, v)
+    out, lse = decode_attention(model, store, [(req, 0)], q)
+    for h in range(hq):
+        np.testing.assert_allclose(out[0, h], v[:, h // 3].astype(np.float64).mean(0), atol=1e-13)
+        s = float(k[0, h // 3].astype(np.float64) @ q[0, h].astype(np.float32).astype(np.float64)) / np.sqrt(d)
+        assert abs(lse[0, h] - (s + np.log(n))) < 1e-12
+    # constant V -> that constant
+    k2 = rng.standard_normal((n, hkv, d)).astype(np.float32)
+    model, store, req = _store_with(k2, np.full((n, hkv, d), 0.75, dtype=np.float32))
+    out, _ = decode_attention(model, store, [(req, 0)], q)
+    np.testing.assert_allclose(out, 0.75, atol=1e-13)
+    # one key far above the rest -> its V row (kv head 1 only, so the head mapping is pinned too)
+    k3 = np.zeros((n, hkv, d), dtype=np.float32)
+    qq = np.zeros((1, hq, d)); qq[0, :, 0] = 1.0
+    k3[11, 1, 0] = 200.0                       # score 200/sqrt(8) ~ 70 above the others, for heads 3..5
+    model, store, req = _store_with(k3, v)
+    out, _ = decode_attention(model, store, [(req, 0)], qq)
+    for h in range(hq):
+        want = v[11, 1] if h >= 3 else v[:, 0].astype(np.float64).mean(0)
+        np.testing.assert_allclose(out[0, h], want, atol=1e-12)
+    # a single visible token -> exactly its V
+    model, store, req = _store_with(k2[:1], v[:1])
+    out, lse = decode_attention(model, store, [(req, 0)], q)
+    for h in range(hq):
+        assert np.array_equal(out[0, h], v[0, h // 3].astype(np.float64))
+
+
+def test_scale_is_one_over_sqrt_d():
+    # two keys, scores differ by exactly ln(3)*sqrt(d) before scaling -> weights 3/4 and 1/4
+    d = 16
+    k = np.zeros((2, 1, d), dtype=np.float32); k[0, 0, 0] = 1.0
+    v = np.zeros((2, 1, d), dtype=np.float32); v[0, 0, 0] = 1.0; v[1, 0, 1] = 1.0
+    q = np.zeros((1, d)); q[0, 0] = np.log(3.0) * np.sqrt(d)
+    o, lse, w = attend(q, k.astype(np.float64), v.astype(np.float64))
+    np.testing.assert_allclose(w[0], [0.75, 0.25], atol=1e-15)
+    np.testing.assert_allclose(o[0, :2], [0.75, 0.25], atol=1e-15)
+    assert abs(lse[0] - np.log(4.0)) < 1e-14
+
+
+# ------------------------------------------------------------------ invariants
+def test_weights_sum_to_one():
+    script = cfg1_tiny("cutoffs")
+    replay = OracleReplay(script)
+    for i, op in enumerate(script.ops[:-1]):
+        replay.apply(i)
+    from pasta_workloads import step_tensors
+    i = len(script.ops) - 1
+    replay.model.reserve(script.ops[i][1])
+    _, _, q = step_tensors(script, i, 0)
+    _, _, weights = decode_attention(replay.model, replay.stores[0], [(e[0], e[1]) for e in script.ops[i][1]], q,
+                                     return_weights=True)
+    lens = [96, 112 + 17, 128 + 32, 128]
+    for w, n in zip(weights, lens):
+        assert w.shape[1] == n
+        assert np.all(np.abs(w.sum(axis=1) - 1.0) < 1e-14) and np.all(w >= 0)
+
+
+@pytest.mark.parametrize("maker", [lambda: cfg1_tiny("cutoffs"), lambda: random_script(101), lambda: random_script(102)])
+def test_invariant_to_page_placement(maker):
+    a = maker()
+    b = maker()
+    b.free_order = np.random.default_rng(99).permutation(b.n_pages).astype(np.int32)
+    assert not np.array_equal(a.free_order, b.free_order)
+    oa, ob = oracle_outputs(a), oracle_outputs(b)
+    for i in oa:
+        assert np.array_equal(oa[i][0], ob[i][0]) and np.array_equal(oa[i][1], ob[i][1])
+
+
+def test_forks_do_not_see_each_other_and_main_ignores_them_until_sync():
+    geo = Geometry(1, 4, 2, 8, 4)
+    base = [("begin", 0), ("run", 0, 0, 9), ("spawn", 0, 1), ("spawn", 0, 2), ("run", 0, 1, 5)]
+    quiet = base + [("step", ((0, 1, 0), (0, 0, 0)))]
+    noisy = base + [("run", 0, 2, 7), ("step", ((0, 1, 0), (0, 0, 0)))]
+    a = oracle_outputs(manual_script(quiet, geo))
+    b = oracle_outputs(manual_script(noisy, geo))
+    (ia, oa), (ib, ob) = list(a.items())[0], list(b.items())[0]
+    # the step's q is drawn from (seed, op index): make both steps use the same q by comparing through weights instead
+    # -> rebuild with identical op indices: pad the quiet script with a run of zero tokens
+    quiet = base + [("run", 0, 2, 0), ("step", ((0, 1, 0), (0, 0, 0)))]
+    a = oracle_outputs(manual_script(quiet, geo))
+    (ia, oa) = list(a.items())[0]
+    assert ia == ib and np.array_equal(oa[0], ob[0])
+
+
+def test_after_sync_main_sees_union_of_prefix_and_chunks():
+    geo = Geometry(1, 4, 2, 8, 4)
+    ops = [("begin", 0), ("run", 0, 0, 6), ("spawn", 0, 1), ("run", 0, 0, 3), ("spawn", 0, 2),
+           ("run", 0, 1, 5), ("run", 0, 2, 2), ("run", 0, 0, 4),
+           ("finish", 0, 1), ("finish", 0, 2), ("merge", 0, None), ("step", ((0, 0, 1),))]
+    script = manual_script(ops, geo)
+    from pasta_workloads import run_tensors, step_tensors
+    ks, vs = [], []
+    for i, op in enumerate(ops):
+        if op[0] == "run":
+            k, v = run_tensors(script, i, 0); ks.append(k); vs.append(v)
+    k, v, q = step_tensors(script, len(ops) - 1, 0)
+    K = torch.cat(ks + [k]).double().numpy(); V = torch.cat(vs + [v]).double().numpy()
+    o, lse, _ = attend(q[0].double().numpy(), K, V)
+    out = oracle_outputs(script)[len(ops) - 1]
+    np.testing.assert_allclose(out[0][0], o, atol=1e-13)
+    replay = OracleReplay(script); replay.run_all()
+    assert replay.model.view(0, 0) == [(0, 0, 6), (1, 0, 5), (0, 6, 3), (2, 0, 2), (0, 9, 5)]
+
+
+def test_fork_spawned_after_a_sync_sees_merged_chunks_but_earlier_forks_never_do():
+    ops = [("begin", 0), ("run", 0, 0, 5), ("spawn", 0, 1), ("spawn", 0, 2), ("run", 0, 1, 3),
+           ("finish", 0, 1), ("merge", 0, (1,)), ("spawn", 0, 3), ("run", 0, 3, 2), ("run", 0, 2, 1)]
+    replay = OracleReplay(manual_script(ops)); replay.run_all()
+    m = replay.model
+    assert m.view(0, 3) == [(0, 0, 5), (1, 0, 3), (3, 0, 2)]
+    assert m.view(0, 2) == [(0, 0, 5), (2, 0, 1)]
+    assert m.view(0, 0) == [(0, 0, 5), (1, 0, 3)]
+
+
+def test_config2_shapes():
+    for variant in "ab":
+        script = cfg2_single_request(variant)
+        replay = OracleReplay(script, with_kv=False); replay.run_all(attend_steps=[])
+        view = replay.model.view(0, 0)
+        total = sum(n for _, _, n in view)
+        assert total == 769 + sum(script.notes["chunks"])
+        assert [s for s, _, _ in view if s != 0] == [1, 2, 3, 4]
