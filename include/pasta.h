@@ -1,0 +1,216 @@
+/*
+ * pasta.h — C ABI of the decode-attention path for interpreter-driven asynchronous decoding
+ * ("Learning to Keep a Promise", PASTA; Section 3 "Efficiency", Fig. 2b/2c, Appendix B).
+ *
+ * Several threads of one response decode one token each in the same model step.  All of them
+ * keep their KV in ONE pool; a thread attends to the main-thread tokens that existed when it was
+ * spawned plus its own chunk; after <sync/> the main thread attends to everything, each chunk
+ * placed logically right after its <promise/>, and nothing is copied.  This library owns the
+ * bookkeeping of that pool (pages, per-thread segment lists) and runs the per-step attention on
+ * one NVIDIA B200 (sm_100a).  There is no CPU fallback: every compute entry point needs the GPU.
+ *
+ * General conventions
+ *  - Every function returns a pasta_status_t and never throws, aborts or exits.
+ *  - Out-parameters are written only on success.  A failed call leaves the pool unchanged.
+ *  - "host" pointers are read or written during the call only.  "device" pointers must stay
+ *    valid until the stream has executed the work enqueued by the call.
+ *  - One pool belongs to one GPU and is not thread-safe: calls on one pool must not overlap.
+ *  - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  All device
+ *    work of a pool must be issued on streams that are ordered with respect to each other by the
+ *    caller; the simplest use is one stream per pool.
+ *  - Tensors are dense, row-major, bf16 unless stated; the last index is contiguous.
+ */
+#ifndef PASTA_H_
+#define PASTA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct pasta_pool pasta_pool_t;   /* opaque; created by pasta_pool_create, freed by pasta_pool_destroy */
+typedef int32_t pasta_status_t;
+
+enum {
+  PASTA_OK = 0,
+  PASTA_ERR_INVALID_ARG = 1,   /* unknown id, thread listed twice, finished thread in a step, bad pointer or size */
+  PASTA_ERR_OUT_OF_PAGES = 2,  /* the pool has too few free pages for the request */
+  PASTA_ERR_BAD_STATE = 3,     /* e.g. merging a fork that is still decoding, compute call on a host-only pool */
+  PASTA_ERR_CAPACITY = 4,      /* more requests / threads / segments / step entries than the pool was created for */
+  PASTA_ERR_CUDA = 5,          /* a CUDA runtime call failed; pasta_last_cuda_error() gives its code */
+  PASTA_ERR_DEVICE_CHECK = 6,  /* a kernel found an out-of-range page id or offset and skipped the access */
+  PASTA_ERR_TIMEOUT = 7        /* a bounded wait inside a kernel expired; the kernel returned early */
+};
+
+enum {
+  PASTA_FLAG_HOST_ONLY = 1,      /* bookkeeping only: no CUDA call is ever made, compute entry points return BAD_STATE */
+  PASTA_FLAG_NO_TENSOR_PATH = 2  /* route every stream through the warp-shuffle kernel (debugging / comparison) */
+};
+
+/* thread states reported by pasta_pool_dump */
+enum { PASTA_THREAD_ACTIVE = 0, PASTA_THREAD_FINISHED = 1, PASTA_THREAD_MERGED = 2 };
+
+typedef struct {
+  int32_t n_layers;                 /* independent layers stored in the pool (page ids are shared by all layers) */
+  int32_t n_q_heads, n_kv_heads;    /* n_q_heads must be a multiple of n_kv_heads; group = n_q_heads / n_kv_heads in {1,2,4,8} */
+  int32_t head_dim;                 /* 64 or 128 */
+  int32_t page_size;                /* tokens per page; must be 16 */
+  int32_t n_pages;                  /* pages per layer */
+  int32_t max_requests;             /* requests alive at the same time */
+  int32_t max_threads_per_request;  /* main thread + every fork ever spawned by one request (ids are not reused) */
+  int32_t max_segments_per_thread;  /* longest segment list of one thread */
+  int32_t max_step_queries;         /* most (request, thread) entries in one step; 0 = max_requests * 17 */
+  int32_t max_partial_rows;         /* split/segment partial results per layer; 0 = derived from max_step_queries */
+  int32_t max_layers_per_launch;    /* layers whose partials fit the workspace at once; 0 = min(n_layers, 8) */
+  int32_t flags;                    /* PASTA_FLAG_* */
+  int32_t device;                   /* CUDA device ordinal the pool lives on */
+  void *kv_base;                    /* device; pasta_kv_bytes() bytes, 1024-byte aligned, allocated and freed by the caller */
+  size_t kv_bytes;
+  void *workspace;                  /* device; pasta_workspace_bytes() bytes, 256-byte aligned, caller-owned */
+  size_t workspace_bytes;
+  const int32_t *free_order;        /* host; n_pages entries, a permutation: order in which free pages are handed out
+                                       (NULL = 0, 1, 2, …) */
+} pasta_pool_config_t;
+
+/* Sizes of the two device buffers the caller has to provide for this configuration. */
+pasta_status_t pasta_kv_bytes(const pasta_pool_config_t *cfg, size_t *out);
+pasta_status_t pasta_workspace_bytes(const pasta_pool_config_t *cfg, size_t *out);
+
+/*
+ * The single pre-allocated KV pool of Section 3 "Efficiency" (here paged: 16 tokens per page, one
+ * page list per stream, where a stream is the main thread's tokens or one fork's chunk).  The
+ * layout inside a page is private to the library; results do not depend on which pages a stream
+ * receives.  The KV memory itself is not touched by create/destroy.
+ */
+pasta_status_t pasta_pool_create(const pasta_pool_config_t *cfg, pasta_pool_t **out);
+pasta_status_t pasta_pool_destroy(pasta_pool_t *pool);
+
+/* ---- thread lifecycle: host only, integers only (Section 3 "Interpreter") -------------------- */
+
+/* A new response; its main thread has id 0.  The request gets the lowest id not in use. */
+pasta_status_t pasta_request_begin(pasta_pool_t *pool, int32_t *out_req);
+/* Returns every page of the request: stream by stream (ascending id), page by page, each to the
+ * FRONT of the free sequence. */
+pasta_status_t pasta_request_end(pasta_pool_t *pool, int32_t req);
+/* <promise/>: a fork whose view is the main thread's view at this moment (call it after the promise
+ * token was appended), followed by its own chunk.  Forks are numbered 1, 2, 3, … per request. */
+pasta_status_t pasta_thread_spawn(pasta_pool_t *pool, int32_t req, int32_t *out_thread);
+/* </async>: the fork decodes no more; its chunk stays invisible to the main thread until merged. */
+pasta_status_t pasta_thread_finish(pasta_pool_t *pool, int32_t req, int32_t thread);
+
+/*
+ * <sync/> (Section 3: the main thread waits for the forks, then conditions on their chunks; the
+ * paper's pool moves no KV at this point and neither does this call).  The named finished forks
+ * are merged into the main thread's segment list: each chunk goes right after the main-stream
+ * piece that ends at the fork's cut-off (ties: ascending thread id).  n_threads < 0 merges every
+ * finished, unmerged fork.  Naming a fork that is still decoding returns BAD_STATE: waiting is
+ * the caller's job.  Host only; the <sync/> token itself is appended by the next step.
+ */
+pasta_status_t pasta_sync_merge(pasta_pool_t *pool, int32_t req, int32_t n_threads, const int32_t *thread_ids);
+
+/* ---- one decode step (Section 3: every active thread decodes one token in the same step) ----- */
+
+/*
+ * Reserves the pool slot of every token appended in this step and plans the attention of the
+ * step.  Entry i is thread thread_ids[i] of request req_ids[i] (host arrays, n entries, each
+ * thread at most once, ACTIVE threads only) and appends n_new[i] tokens (0 or 1; NULL = all 1).
+ * Pages are taken in list order, one whenever a stream's token index is a multiple of 16.
+ * An entry that would see nothing (no visible token and n_new == 0) is INVALID_ARG.
+ * The plan is uploaded on `stream`; it is used by the pasta_kv_append and pasta_decode_attn calls
+ * that follow, for every layer, until the next pasta_step_begin.
+ */
+pasta_status_t pasta_step_begin(pasta_pool_t *pool, int32_t n, const int32_t *req_ids,
+                                const int32_t *thread_ids, const int32_t *n_new, void *stream);
+
+/* (page, offset) reserved by the last pasta_step_begin for each of its entries, two int32 per
+ * entry, (-1, -1) for entries with n_new == 0.  Host array of 2 * n entries. */
+pasta_status_t pasta_step_slots(pasta_pool_t *pool, int32_t *out_slots, int32_t capacity_entries);
+
+/*
+ * Copies the new tokens' K and V into their reserved slots for layers
+ * [layer_begin, layer_begin + layer_count).  k_new, v_new: device bf16
+ * [layer_count, n_app, n_kv_heads, head_dim], where n_app is the number of step entries with
+ * n_new == 1, in entry order.  A pure bit copy.
+ */
+pasta_status_t pasta_kv_append(pasta_pool_t *pool, int32_t layer_begin, int32_t layer_count,
+                               const void *k_new, const void *v_new, void *stream);
+
+/*
+ * Decode attention of the planned step.  For entry i and query head h (kv head h / group):
+ *     out[l, i, h, :] = softmax(q[l, i, h, :] . K_vis^T * scale) V_vis
+ * over the tokens visible to that thread (its segment list; the token appended in this step
+ * included).  q: device bf16 [layer_count, n, n_q_heads, head_dim]; out: device fp32 of the same
+ * shape; lse: optional device fp32 [layer_count, n, n_q_heads] (natural-log sum of exponentials of
+ * the scaled scores), may be NULL; scale 0 means 1/sqrt(head_dim).
+ * Streams seen by two or more threads of the step are staged into shared memory once per kv head
+ * and scored against all those threads' queries on tensor cores; streams seen by one thread take
+ * a warp-shuffle kernel; a merge kernel combines the partial results (fp32 throughout).
+ */
+pasta_status_t pasta_decode_attn(pasta_pool_t *pool, int32_t layer_begin, int32_t layer_count,
+                                 const void *q, void *out, float *lse, float scale, void *stream);
+
+/*
+ * Appends m tokens to one thread outside a decode step (prompt prefill, benchmark set-up):
+ * reserves slots like m steps of that thread alone would, then copies k, v
+ * (device bf16 [layer_count, m, n_kv_heads, head_dim]).  With layer_count == 0 only the
+ * bookkeeping is done.  Invalidates the current step plan.
+ */
+pasta_status_t pasta_kv_append_run(pasta_pool_t *pool, int32_t req, int32_t thread, int32_t m,
+                                   int32_t layer_begin, int32_t layer_count,
+                                   const void *k, const void *v, void *stream);
+
+/*
+ * One whole step with HOST tensors: step_begin, copy k_new / v_new / q to the device, kv_append
+ * and decode_attn for all layers, copy `out` back, synchronise the stream.  k_new, v_new:
+ * host bf16 [n_layers, n_app, n_kv_heads, head_dim]; q: host bf16 [n_layers, n, n_q_heads, head_dim];
+ * out: host fp32 like q.  staging: device scratch of at least pasta_step_host_bytes(pool, n)
+ * bytes, caller-owned.  Pinned host memory makes the copies asynchronous; pageable works too.
+ */
+pasta_status_t pasta_step_host_bytes(pasta_pool_t *pool, int32_t n, size_t *out);
+pasta_status_t pasta_step_host(pasta_pool_t *pool, int32_t n, const int32_t *req_ids,
+                               const int32_t *thread_ids, const int32_t *n_new,
+                               const void *k_new, const void *v_new, const void *q, void *out,
+                               void *staging, size_t staging_bytes, float scale, void *stream);
+
+/* ---- introspection ---------------------------------------------------------------------------- */
+
+/*
+ * Reads tokens [start, start + m) of one stream (stream id = thread id; 0 = main) of one layer back
+ * into dense device bf16 arrays k_out, v_out [m, n_kv_heads, head_dim].
+ */
+pasta_status_t pasta_kv_read(pasta_pool_t *pool, int32_t layer, int32_t req, int32_t stream_id,
+                             int32_t start, int32_t m, void *k_out, void *v_out, void *stream);
+
+/*
+ * Serialises the bookkeeping state into host int32 words:
+ *   n_requests, then per live request (ascending id):
+ *     req, n_streams, per stream (ascending id): stream, len, n_pages, page ids…
+ *     n_threads, per thread (ascending id): thread, state, cutoff, n_segments, (stream, start, len)…
+ *   n_free, free page ids in hand-out order.
+ * *needed receives the number of words; nothing is written when capacity_words is too small
+ * (the call then still returns PASTA_OK so that the size can be queried with host_buf == NULL).
+ */
+pasta_status_t pasta_pool_dump(pasta_pool_t *pool, int32_t *host_buf, size_t capacity_words, size_t *needed);
+
+/*
+ * The current step plan as uploaded to the device (int32 words, layout documented in
+ * pasta_plan.h inside the package).  Same size protocol as pasta_pool_dump.  For tests.
+ */
+pasta_status_t pasta_plan_dump(pasta_pool_t *pool, int32_t *host_buf, size_t capacity_words, size_t *needed);
+
+/* Synchronises `stream`, returns and clears the status word the kernels write
+ * (PASTA_OK, PASTA_ERR_DEVICE_CHECK or PASTA_ERR_TIMEOUT). */
+pasta_status_t pasta_pool_status(pasta_pool_t *pool, void *stream);
+
+/* Number of kernels this pool has launched so far (for launch accounting). */
+pasta_status_t pasta_launch_count(pasta_pool_t *pool, int64_t *out);
+
+/* cudaError_t of the last failed CUDA call made by the library in this process (0 if none). */
+int32_t pasta_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PASTA_H_ */

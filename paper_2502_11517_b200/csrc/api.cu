@@ -1,0 +1,459 @@
+// The C ABI (include/pasta.h): argument checks, the device side of a pool, uploads and launches.
+#include <algorithm>
+#include <cmath>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "device_common.cuh"
+#include "kernels.hpp"
+#include "plan.hpp"
+#include "pool.hpp"
+
+using namespace pasta;
+
+namespace {
+
+constexpr int kStaging = 4;           // pinned upload buffers in rotation
+constexpr int kRunChunk = 8192;       // tokens whose slots are uploaded at once by pasta_kv_append_run
+int32_t g_last_cuda_error = 0;
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+struct Derived {
+  int32_t group, max_queries, max_rows, layers_per_launch;
+  int64_t max_words, staging_words;
+  size_t kv_bytes, layer_stride;
+  size_t off_status, off_plan, off_run, off_ml, off_o, ws_bytes;
+};
+
+pasta_status_t derive(const pasta_pool_config_t &c, Derived *d) {
+  if (c.n_layers < 1 || c.n_kv_heads < 1 || c.n_q_heads < 1 || c.n_q_heads % c.n_kv_heads) return PASTA_ERR_INVALID_ARG;
+  d->group = c.n_q_heads / c.n_kv_heads;
+  if (d->group != 1 && d->group != 2 && d->group != 4 && d->group != 8) return PASTA_ERR_INVALID_ARG;
+  if (c.head_dim != 64 && c.head_dim != 128) return PASTA_ERR_INVALID_ARG;
+  if (c.page_size != PASTA_PAGE || c.n_pages < 1) return PASTA_ERR_INVALID_ARG;
+  if (c.max_requests < 1 || c.max_threads_per_request < 1 || c.max_segments_per_thread < 1) return PASTA_ERR_INVALID_ARG;
+  if (c.max_step_queries < 0 || c.max_partial_rows < 0 || c.max_layers_per_launch < 0) return PASTA_ERR_INVALID_ARG;
+  const int grid = 160;   // upper bound on CTAs of the tensor-core kernel, for sizing only
+  d->max_queries = c.max_step_queries ? c.max_step_queries
+                                      : static_cast<int32_t>(std::min<int64_t>(int64_t(c.max_requests) * 17, 1 << 20));
+  d->max_rows = c.max_partial_rows ? c.max_partial_rows
+                                   : static_cast<int32_t>(std::min<int64_t>(
+                                         int64_t(d->max_queries) * c.n_q_heads * 8 + int64_t(grid) * PASTA_MAX_ROWS, 1 << 28));
+  d->layers_per_launch = c.max_layers_per_launch ? std::min(c.max_layers_per_launch, c.n_layers)
+                                                 : std::min(c.n_layers, 8);
+  const int64_t nq = d->max_queries, nr = c.max_requests;
+  d->max_words = PH_WORDS + 2 * nq + PQ_WORDS * nq + PT_WORDS * nr + 2 * nr * c.n_kv_heads +
+                 PU_WORDS * (nr * c.n_kv_heads + grid) + 2 * grid + PW_WORDS * (int64_t(d->max_rows) / d->group + 1) +
+                 2 * int64_t(c.n_pages) + nq * std::min(255, c.max_threads_per_request) + nq + 64;
+  d->staging_words = std::max<int64_t>(d->max_words, 2 * kRunChunk);
+  d->layer_stride = size_t(c.n_pages) * c.n_kv_heads * kv_block_bytes(c.head_dim);
+  d->kv_bytes = d->layer_stride * c.n_layers;
+  size_t off = 0;
+  d->off_status = off; off += 256;
+  d->off_plan = off;   off = align_up(off + size_t(d->max_words) * 4, 256);
+  d->off_run = off;    off = align_up(off + size_t(2 * kRunChunk) * 4, 256);
+  const size_t rows = size_t(d->max_rows) * d->layers_per_launch;
+  d->off_ml = off;     off = align_up(off + rows * sizeof(float2), 256);
+  d->off_o = off;      off = align_up(off + rows * c.head_dim * sizeof(float), 256);
+  d->ws_bytes = off;
+  return PASTA_OK;
+}
+
+}  // namespace
+
+struct pasta_pool {
+  pasta_pool_config_t cfg;
+  Derived d;
+  HostPool host;
+  bool host_only;
+  int sm_count = 148;
+  PoolView pv{};
+  int32_t *run_slots_dev = nullptr;
+  int32_t *pinned[kStaging] = {nullptr, nullptr, nullptr, nullptr};
+  cudaEvent_t pinned_free[kStaging] = {nullptr, nullptr, nullptr, nullptr};
+  int next_pinned = 0;
+  int32_t *status_host = nullptr;     // pinned, one word
+  std::vector<StepEntry> entries;
+  std::vector<Slot> slots;
+  std::vector<int32_t> plan;
+  PlanHeader hdr{};
+  bool plan_valid = false;
+  int64_t launches = 0;
+
+  pasta_pool(const pasta_pool_config_t &c, const Derived &dd)
+      : cfg(c), d(dd),
+        host(c.n_pages, c.page_size, c.free_order, c.max_requests, c.max_threads_per_request,
+             c.max_segments_per_thread),
+        host_only((c.flags & PASTA_FLAG_HOST_ONLY) != 0) {}
+};
+
+namespace {
+
+pasta_status_t cuda_fail(cudaError_t e) {
+  g_last_cuda_error = static_cast<int32_t>(e);
+  return PASTA_ERR_CUDA;
+}
+#define PASTA_CUDA(call)                                  \
+  do {                                                    \
+    cudaError_t e__ = (call);                             \
+    if (e__ != cudaSuccess) return cuda_fail(e__);        \
+  } while (0)
+
+// Copies `words` int32 from host memory to `dst` on the stream through a pinned buffer of the ring.
+pasta_status_t upload(pasta_pool *p, const int32_t *src, size_t words, int32_t *dst, cudaStream_t st) {
+  const int b = p->next_pinned;
+  p->next_pinned = (b + 1) % kStaging;
+  PASTA_CUDA(cudaEventSynchronize(p->pinned_free[b]));   // the copy that last used this buffer is done
+  std::memcpy(p->pinned[b], src, words * 4);
+  PASTA_CUDA(cudaMemcpyAsync(dst, p->pinned[b], words * 4, cudaMemcpyHostToDevice, st));
+  PASTA_CUDA(cudaEventRecord(p->pinned_free[b], st));
+  return PASTA_OK;
+}
+
+PlanLimits limits_of(const pasta_pool *p) {
+  PlanLimits l;
+  l.n_q_heads = p->cfg.n_q_heads;
+  l.n_kv_heads = p->cfg.n_kv_heads;
+  l.head_dim = p->cfg.head_dim;
+  l.max_queries = p->d.max_queries;
+  l.max_rows = p->d.max_rows;
+  l.max_words = p->d.max_words;
+  l.grid = p->sm_count;
+  l.tensor_path = p->cfg.head_dim == 128 && !(p->cfg.flags & PASTA_FLAG_NO_TENSOR_PATH) && tensor_path_available();
+  return l;
+}
+
+}  // namespace
+
+extern "C" {
+
+int32_t pasta_last_cuda_error(void) { return g_last_cuda_error; }
+
+pasta_status_t pasta_kv_bytes(const pasta_pool_config_t *cfg, size_t *out) {
+  if (!cfg || !out) return PASTA_ERR_INVALID_ARG;
+  Derived d;
+  pasta_status_t s = derive(*cfg, &d);
+  if (s != PASTA_OK) return s;
+  *out = d.kv_bytes;
+  return PASTA_OK;
+}
+
+pasta_status_t pasta_workspace_bytes(const pasta_pool_config_t *cfg, size_t *out) {
+  if (!cfg || !out) return PASTA_ERR_INVALID_ARG;
+  Derived d;
+  pasta_status_t s = derive(*cfg, &d);
+  if (s != PASTA_OK) return s;
+  *out = d.ws_bytes;
+  return PASTA_OK;
+}
+
+pasta_status_t pasta_pool_create(const pasta_pool_config_t *cfg, pasta_pool_t **out) {
+  if (!cfg || !out) return PASTA_ERR_INVALID_ARG;
+  Derived d;
+  pasta_status_t s = derive(*cfg, &d);
+  if (s != PASTA_OK) return s;
+  if (!HostPool::valid_free_order(cfg->n_pages, cfg->free_order)) return PASTA_ERR_INVALID_ARG;
+  const bool host_only = (cfg->flags & PASTA_FLAG_HOST_ONLY) != 0;
+  if (!host_only) {
+    if (!cfg->kv_base || cfg->kv_bytes < d.kv_bytes || (reinterpret_cast<uintptr_t>(cfg->kv_base) & 1023))
+      return PASTA_ERR_INVALID_ARG;
+    if (!cfg->workspace || cfg->workspace_bytes < d.ws_bytes || (reinterpret_cast<uintptr_t>(cfg->workspace) & 255))
+      return PASTA_ERR_INVALID_ARG;
+  }
+  pasta_pool *p = new (std::nothrow) pasta_pool(*cfg, d);
+  if (!p) return PASTA_ERR_CAPACITY;
+  p->cfg.free_order = nullptr;   // read during this call only
+  if (!host_only) {
+    cudaError_t e = cudaSetDevice(cfg->device);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&p->sm_count, cudaDevAttrMultiProcessorCount, cfg->device);
+    for (int i = 0; i < kStaging && e == cudaSuccess; ++i) {
+      e = cudaMallocHost(reinterpret_cast<void **>(&p->pinned[i]), size_t(d.staging_words) * 4);
+      if (e == cudaSuccess) e = cudaEventCreateWithFlags(&p->pinned_free[i], cudaEventDisableTiming);
+    }
+    if (e == cudaSuccess) e = cudaMallocHost(reinterpret_cast<void **>(&p->status_host), 64);
+    uint8_t *ws = static_cast<uint8_t *>(cfg->workspace);
+    if (e == cudaSuccess) e = cudaMemset(ws, 0, 256);
+    // stale bytes of a page's unused tail are multiplied by zero weights, so they must be finite
+    if (e == cudaSuccess) e = cudaMemset(cfg->kv_base, 0, d.kv_bytes);
+    if (e == cudaSuccess) e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) {
+      pasta_pool_destroy(p);
+      return cuda_fail(e);
+    }
+    p->pv.kv_base = static_cast<uint8_t *>(cfg->kv_base);
+    p->pv.layer_stride = static_cast<int64_t>(d.layer_stride);
+    p->pv.n_pages = cfg->n_pages;
+    p->pv.n_q_heads = cfg->n_q_heads;
+    p->pv.n_kv_heads = cfg->n_kv_heads;
+    p->pv.head_dim = cfg->head_dim;
+    p->pv.status = reinterpret_cast<int32_t *>(ws + d.off_status);
+    p->pv.plan = reinterpret_cast<const int32_t *>(ws + d.off_plan);
+    p->run_slots_dev = reinterpret_cast<int32_t *>(ws + d.off_run);
+    p->pv.part_ml = reinterpret_cast<float2 *>(ws + d.off_ml);
+    p->pv.part_o = reinterpret_cast<float *>(ws + d.off_o);
+    p->pv.rows_per_layer = d.max_rows;
+  }
+  *out = p;
+  return PASTA_OK;
+}
+
+pasta_status_t pasta_pool_destroy(pasta_pool_t *p) {
+  if (!p) return PASTA_ERR_INVALID_ARG;
+  for (int i = 0; i < kStaging; ++i) {
+    if (p->pinned_free[i]) { cudaEventSynchronize(p->pinned_free[i]); cudaEventDestroy(p->pinned_free[i]); }
+    if (p->pinned[i]) cudaFreeHost(p->pinned[i]);
+  }
+  if (p->status_host) cudaFreeHost(p->status_host);
+  delete p;
+  return PASTA_OK;
+}
+
+pasta_status_t pasta_request_begin(pasta_pool_t *p, int32_t *out_req) {
+  if (!p || !out_req) return PASTA_ERR_INVALID_ARG;
+  return p->host.request_begin(out_req);
+}
+
+pasta_status_t pasta_request_end(pasta_pool_t *p, int32_t req) {
+  if (!p) return PASTA_ERR_INVALID_ARG;
+  pasta_status_t s = p->host.request_end(req);
+  if (s == PASTA_OK) p->plan_valid = false;
+  return s;
+}
+
+pasta_status_t pasta_thread_spawn(pasta_pool_t *p, int32_t req, int32_t *out_thread) {
+  if (!p || !out_thread) return PASTA_ERR_INVALID_ARG;
+  return p->host.thread_spawn(req, out_thread);
+}
+
+pasta_status_t pasta_thread_finish(pasta_pool_t *p, int32_t req, int32_t thread) {
+  if (!p) return PASTA_ERR_INVALID_ARG;
+  return p->host.thread_finish(req, thread);
+}
+
+pasta_status_t pasta_sync_merge(pasta_pool_t *p, int32_t req, int32_t n_threads, const int32_t *thread_ids) {
+  if (!p) return PASTA_ERR_INVALID_ARG;
+  return p->host.sync_merge(req, n_threads, thread_ids);
+}
+
+pasta_status_t pasta_step_begin(pasta_pool_t *p, int32_t n, const int32_t *req_ids, const int32_t *thread_ids,
+                                const int32_t *n_new, void *stream) {
+  if (!p || n < 0 || (n > 0 && (!req_ids || !thread_ids))) return PASTA_ERR_INVALID_ARG;
+  if (n > p->d.max_queries) return PASTA_ERR_CAPACITY;
+  std::vector<StepEntry> entries(n);
+  for (int32_t i = 0; i < n; ++i) entries[i] = StepEntry{req_ids[i], thread_ids[i], n_new ? n_new[i] : 1};
+  std::vector<Slot> slots;
+  pasta_status_t s = p->host.reserve_step(entries, &slots);
+  if (s != PASTA_OK) return s;
+  p->plan_valid = false;
+  p->entries.swap(entries);
+  p->slots.swap(slots);
+  s = build_plan(p->host, p->entries, p->slots, limits_of(p), &p->plan);
+  if (s != PASTA_OK) return s;   // the tokens stay reserved; only the attention of this step cannot be planned
+  std::memcpy(p->hdr.w, p->plan.data(), sizeof(p->hdr.w));
+  if (!p->host_only) {
+    s = upload(p, p->plan.data(), p->plan.size(), const_cast<int32_t *>(p->pv.plan), static_cast<cudaStream_t>(stream));
+    if (s != PASTA_OK) return s;
+  }
+  p->plan_valid = true;
+  return PASTA_OK;
+}
+
+pasta_status_t pasta_step_slots(pasta_pool_t *p, int32_t *out_slots, int32_t capacity_entries) {
+  if (!p || !out_slots) return PASTA_ERR_INVALID_ARG;
+  if (capacity_entries < static_cast<int32_t>(p->slots.size())) return PASTA_ERR_CAPACITY;
+  for (size_t i = 0; i < p->slots.size(); ++i) {
+    out_slots[2 * i] = p->slots[i].page;
+    out_slots[2 * i + 1] = p->slots[i].offset;
+  }
+  return PASTA_OK;
+}
+
+pasta_status_t pasta_kv_append(pasta_pool_t *p, int32_t layer_begin, int32_t layer_count, const void *k_new,
+                               const void *v_new, void *stream) {
+  if (!p) return PASTA_ERR_INVALID_ARG;
+  if (p->host_only || !p->plan_valid) return PASTA_ERR_BAD_STATE;
+  if (layer_begin < 0 || layer_count < 0 || layer_begin + layer_count > p->cfg.n_layers) return PASTA_ERR_INVALID_ARG;
+  const int32_t n_app = p->hdr.w[PH_N_APPEND];
+  if (n_app == 0 || layer_count == 0) return PASTA_OK;
+  if (!k_new || !v_new) return PASTA_ERR_INVALID_ARG;
+  PASTA_CUDA(launch_kv_append(p->pv, p->pv.plan + p->hdr.w[PH_OFF_APPEND], n_app, layer_begin, layer_count, k_new, v_new,
+                              static_cast<cudaStream_t>(stream)));
+  p->launches += 1;
+  return PASTA_OK;
+}
+
+pasta_status_t pasta_decode_attn(pasta_pool_t *p, int32_t layer_begin, int32_t layer_count, const void *q, void *out,
+                                 float *lse, float scale, void *stream) {
+  if (!p) return PASTA_ERR_INVALID_ARG;
+  if (p->host_only || !p->plan_valid) return PASTA_ERR_BAD_STATE;
+  if (layer_begin < 0 || layer_count < 0 || layer_begin + layer_count > p->cfg.n_layers) return PASTA_ERR_INVALID_ARG;
+  const int32_t n = p->hdr.w[PH_N_QUERIES];
+  if (n == 0 || layer_count == 0) return PASTA_OK;
+  if (!q || !out || !(scale >= 0.f)) return PASTA_ERR_INVALID_ARG;
+  const float sc = (scale == 0.f ? 1.0f / std::sqrt(static_cast<float>(p->cfg.head_dim)) : scale) * 1.4426950408889634f;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const size_t q_layer = size_t(n) * p->cfg.n_q_heads * p->cfg.head_dim;
+  for (int32_t done = 0; done < layer_count; done += p->d.layers_per_launch) {
+    const int32_t cnt = std::min(p->d.layers_per_launch, layer_count - done);
+    const uint16_t *qg = static_cast<const uint16_t *>(q) + size_t(done) * q_layer;
+    float *og = static_cast<float *>(out) + size_t(done) * q_layer;
+    float *lg = lse ? lse + size_t(done) * n * p->cfg.n_q_heads : nullptr;
+    if (p->hdr.w[PH_N_TUNITS] > 0) {
+      PASTA_CUDA(launch_attn_tensor(p->pv, p->hdr, layer_begin + done, cnt, qg, sc, st));
+      p->launches += 1;
+    }
+    if (p->hdr.w[PH_N_WUNITS] > 0) {
+      PASTA_CUDA(launch_attn_warp(p->pv, p->hdr, layer_begin + done, cnt, qg, sc, st));
+      p->launches += 1;
+    }
+    PASTA_CUDA(launch_merge(p->pv, p->hdr, cnt, og, lg, st));
+    p->launches += 1;
+  }
+  return PASTA_OK;
+}
+
+pasta_status_t pasta_kv_append_run(pasta_pool_t *p, int32_t req, int32_t thread, int32_t m, int32_t layer_begin,
+                                   int32_t layer_count, const void *k, const void *v, void *stream) {
+  if (!p) return PASTA_ERR_INVALID_ARG;
+  if (layer_begin < 0 || layer_count < 0 || layer_begin + layer_count > p->cfg.n_layers) return PASTA_ERR_INVALID_ARG;
+  if (layer_count > 0 && p->host_only) return PASTA_ERR_BAD_STATE;
+  if (layer_count > 0 && m > 0 && (!k || !v)) return PASTA_ERR_INVALID_ARG;
+  std::vector<Slot> slots;
+  pasta_status_t s = p->host.reserve_run(req, thread, m, &slots);
+  if (s != PASTA_OK) return s;
+  p->plan_valid = false;
+  if (layer_count == 0 || m == 0) return PASTA_OK;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const size_t tok = size_t(p->cfg.n_kv_heads) * p->cfg.head_dim;      // elements per token
+  std::vector<int32_t> words;
+  for (int32_t begin = 0; begin < m; begin += kRunChunk) {
+    const int32_t cnt = std::min(kRunChunk, m - begin);
+    words.resize(size_t(cnt) * 2);
+    for (int32_t i = 0; i < cnt; ++i) { words[2 * i] = slots[begin + i].page; words[2 * i + 1] = slots[begin + i].offset; }
+    s = upload(p, words.data(), words.size(), p->run_slots_dev, st);
+    if (s != PASTA_OK) return s;
+    for (int32_t l = 0; l < layer_count; ++l) {     // the run's layers are [layer_count, m, …]: one launch per layer and chunk
+      const uint16_t *kl = static_cast<const uint16_t *>(k) + (size_t(l) * m + begin) * tok;
+      const uint16_t *vl = static_cast<const uint16_t *>(v) + (size_t(l) * m + begin) * tok;
+      PASTA_CUDA(launch_kv_append(p->pv, p->run_slots_dev, cnt, layer_begin + l, 1, kl, vl, st));
+      p->launches += 1;
+    }
+  }
+  return PASTA_OK;
+}
+
+pasta_status_t pasta_step_host_bytes(pasta_pool_t *p, int32_t n, size_t *out) {
+  if (!p || !out || n < 0) return PASTA_ERR_INVALID_ARG;
+  const size_t L = p->cfg.n_layers, d = p->cfg.head_dim;
+  const size_t kv = align_up(L * n * p->cfg.n_kv_heads * d * 2, 256);
+  const size_t qb = align_up(L * n * p->cfg.n_q_heads * d * 2, 256);
+  const size_t ob = align_up(L * n * p->cfg.n_q_heads * d * 4, 256);
+  *out = 2 * kv + qb + ob;
+  return PASTA_OK;
+}
+
+pasta_status_t pasta_step_host(pasta_pool_t *p, int32_t n, const int32_t *req_ids, const int32_t *thread_ids,
+                               const int32_t *n_new, const void *k_new, const void *v_new, const void *q, void *out,
+                               void *staging, size_t staging_bytes, float scale, void *stream) {
+  if (!p || !q || !out || !staging) return PASTA_ERR_INVALID_ARG;
+  if (p->host_only) return PASTA_ERR_BAD_STATE;
+  size_t need = 0;
+  pasta_status_t s = pasta_step_host_bytes(p, n, &need);
+  if (s != PASTA_OK) return s;
+  if (staging_bytes < need || (reinterpret_cast<uintptr_t>(staging) & 255)) return PASTA_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  s = pasta_step_begin(p, n, req_ids, thread_ids, n_new, stream);
+  if (s != PASTA_OK) return s;
+  const size_t L = p->cfg.n_layers, d = p->cfg.head_dim;
+  const size_t n_app = p->hdr.w[PH_N_APPEND];
+  const size_t kv_full = align_up(L * n * p->cfg.n_kv_heads * d * 2, 256);
+  const size_t kv_bytes = L * n_app * p->cfg.n_kv_heads * d * 2;
+  const size_t q_bytes = L * n * p->cfg.n_q_heads * d * 2;
+  uint8_t *base = static_cast<uint8_t *>(staging);
+  uint8_t *k_dev = base, *v_dev = base + kv_full, *q_dev = base + 2 * kv_full;
+  uint8_t *o_dev = q_dev + align_up(q_bytes, 256);
+  if (n_app > 0) {
+    if (!k_new || !v_new) return PASTA_ERR_INVALID_ARG;
+    PASTA_CUDA(cudaMemcpyAsync(k_dev, k_new, kv_bytes, cudaMemcpyHostToDevice, st));
+    PASTA_CUDA(cudaMemcpyAsync(v_dev, v_new, kv_bytes, cudaMemcpyHostToDevice, st));
+  }
+  PASTA_CUDA(cudaMemcpyAsync(q_dev, q, q_bytes, cudaMemcpyHostToDevice, st));
+  s = pasta_kv_append(p, 0, p->cfg.n_layers, k_dev, v_dev, stream);
+  if (s != PASTA_OK) return s;
+  s = pasta_decode_attn(p, 0, p->cfg.n_layers, q_dev, o_dev, nullptr, scale, stream);
+  if (s != PASTA_OK) return s;
+  PASTA_CUDA(cudaMemcpyAsync(out, o_dev, q_bytes * 2, cudaMemcpyDeviceToHost, st));
+  PASTA_CUDA(cudaStreamSynchronize(st));
+  return PASTA_OK;
+}
+
+pasta_status_t pasta_kv_read(pasta_pool_t *p, int32_t layer, int32_t req, int32_t stream_id, int32_t start, int32_t m,
+                             void *k_out, void *v_out, void *stream) {
+  if (!p) return PASTA_ERR_INVALID_ARG;
+  if (p->host_only) return PASTA_ERR_BAD_STATE;
+  const Request *r = p->host.request(req);
+  if (!r || layer < 0 || layer >= p->cfg.n_layers || stream_id < 0 || stream_id >= static_cast<int32_t>(r->streams.size()))
+    return PASTA_ERR_INVALID_ARG;
+  const Stream &sm = r->streams[stream_id];
+  if (start < 0 || m < 0 || start + m > sm.len) return PASTA_ERR_INVALID_ARG;
+  if (m == 0) return PASTA_OK;
+  if (!k_out || !v_out) return PASTA_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const size_t tok = size_t(p->cfg.n_kv_heads) * p->cfg.head_dim;
+  std::vector<int32_t> words;
+  for (int32_t begin = 0; begin < m; begin += kRunChunk) {
+    const int32_t cnt = std::min(kRunChunk, m - begin);
+    words.resize(size_t(cnt) * 2);
+    for (int32_t i = 0; i < cnt; ++i) {
+      const int32_t t = start + begin + i;
+      words[2 * i] = sm.pages[t / PASTA_PAGE];
+      words[2 * i + 1] = t % PASTA_PAGE;
+    }
+    pasta_status_t s = upload(p, words.data(), words.size(), p->run_slots_dev, st);
+    if (s != PASTA_OK) return s;
+    PASTA_CUDA(launch_kv_read(p->pv, p->run_slots_dev, cnt, layer, static_cast<uint16_t *>(k_out) + size_t(begin) * tok,
+                              static_cast<uint16_t *>(v_out) + size_t(begin) * tok, st));
+    p->launches += 1;
+  }
+  return PASTA_OK;
+}
+
+static pasta_status_t copy_words(const std::vector<int32_t> &w, int32_t *host_buf, size_t capacity, size_t *needed) {
+  if (!needed) return PASTA_ERR_INVALID_ARG;
+  *needed = w.size();
+  if (host_buf && capacity >= w.size()) std::memcpy(host_buf, w.data(), w.size() * 4);
+  return PASTA_OK;
+}
+
+pasta_status_t pasta_pool_dump(pasta_pool_t *p, int32_t *host_buf, size_t capacity_words, size_t *needed) {
+  if (!p) return PASTA_ERR_INVALID_ARG;
+  std::vector<int32_t> w;
+  p->host.dump(&w);
+  return copy_words(w, host_buf, capacity_words, needed);
+}
+
+pasta_status_t pasta_plan_dump(pasta_pool_t *p, int32_t *host_buf, size_t capacity_words, size_t *needed) {
+  if (!p) return PASTA_ERR_INVALID_ARG;
+  if (!p->plan_valid) return PASTA_ERR_BAD_STATE;
+  return copy_words(p->plan, host_buf, capacity_words, needed);
+}
+
+pasta_status_t pasta_pool_status(pasta_pool_t *p, void *stream) {
+  if (!p) return PASTA_ERR_INVALID_ARG;
+  if (p->host_only) return PASTA_OK;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  PASTA_CUDA(cudaMemcpyAsync(p->status_host, p->pv.status, 4, cudaMemcpyDeviceToHost, st));
+  PASTA_CUDA(cudaMemsetAsync(p->pv.status, 0, 4, st));
+  PASTA_CUDA(cudaStreamSynchronize(st));
+  return *p->status_host;
+}
+
+pasta_status_t pasta_launch_count(pasta_pool_t *p, int64_t *out) {
+  if (!p || !out) return PASTA_ERR_INVALID_ARG;
+  *out = p->launches;
+  return PASTA_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,366 @@
+// K1 (KV append), its inverse (read-back), K3 (warp-shuffle attention pass) and K4 (log-sum-exp merge).
+#include "device_common.cuh"
+#include "kernels.hpp"
+
+namespace pasta {
+
+// =============================================================================================
+// K1: KV append.  One thread moves one 16-byte chunk (8 bf16) of K or V of one token.
+// =============================================================================================
+__global__ void kv_append_kernel(PoolView pv, const int32_t *__restrict__ slots, int32_t n_tok,
+                                 int32_t layer_begin, int32_t layer_count,
+                                 const uint4 *__restrict__ k_new, const uint4 *__restrict__ v_new) {
+  const int chunks = pv.head_dim >> 3;
+  const int64_t total = static_cast<int64_t>(layer_count) * n_tok * pv.n_kv_heads * 2 * chunks;
+  const int64_t idx = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (idx >= total) return;
+  const int c = static_cast<int>(idx % chunks);
+  int64_t rest = idx / chunks;
+  const int kv = static_cast<int>(rest & 1);
+  rest >>= 1;
+  const int g = static_cast<int>(rest % pv.n_kv_heads);
+  rest /= pv.n_kv_heads;
+  const int a = static_cast<int>(rest % n_tok);
+  const int ll = static_cast<int>(rest / n_tok);
+  const int page = slots[2 * a], off = slots[2 * a + 1];
+  if (page < 0 || page >= pv.n_pages || off < 0 || off >= PASTA_PAGE) {
+    report(pv.status, PASTA_ERR_DEVICE_CHECK);
+    return;
+  }
+  const uint4 *src = (kv ? v_new : k_new) + ((static_cast<int64_t>(ll) * n_tok + a) * pv.n_kv_heads + g) * chunks + c;
+  uint8_t *block = pv.kv_base + (layer_begin + ll) * pv.layer_stride +
+                   (static_cast<int64_t>(page) * pv.n_kv_heads + g) * kv_block_bytes(pv.head_dim);
+  *reinterpret_cast<uint4 *>(block + kv_chunk_offset(pv.head_dim >> 6, kv, off, c)) = __ldg(src);
+}
+
+__global__ void kv_read_kernel(PoolView pv, const int32_t *__restrict__ slots, int32_t n_tok, int32_t layer,
+                               uint4 *__restrict__ k_out, uint4 *__restrict__ v_out) {
+  const int chunks = pv.head_dim >> 3;
+  const int64_t total = static_cast<int64_t>(n_tok) * pv.n_kv_heads * 2 * chunks;
+  const int64_t idx = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (idx >= total) return;
+  const int c = static_cast<int>(idx % chunks);
+  int64_t rest = idx / chunks;
+  const int kv = static_cast<int>(rest & 1);
+  rest >>= 1;
+  const int g = static_cast<int>(rest % pv.n_kv_heads);
+  const int a = static_cast<int>(rest / pv.n_kv_heads);
+  const int page = slots[2 * a], off = slots[2 * a + 1];
+  if (page < 0 || page >= pv.n_pages || off < 0 || off >= PASTA_PAGE) {
+    report(pv.status, PASTA_ERR_DEVICE_CHECK);
+    return;
+  }
+  const uint8_t *block = pv.kv_base + layer * pv.layer_stride +
+                         (static_cast<int64_t>(page) * pv.n_kv_heads + g) * kv_block_bytes(pv.head_dim);
+  uint4 *dst = (kv ? v_out : k_out) + (static_cast<int64_t>(a) * pv.n_kv_heads + g) * chunks + c;
+  *dst = *reinterpret_cast<const uint4 *>(block + kv_chunk_offset(pv.head_dim >> 6, kv, off, c));
+}
+
+cudaError_t launch_kv_append(const PoolView &pv, const int32_t *slots, int32_t n_tok, int32_t layer_begin,
+                             int32_t layer_count, const void *k_new, const void *v_new, cudaStream_t st) {
+  const int64_t total = static_cast<int64_t>(layer_count) * n_tok * pv.n_kv_heads * 2 * (pv.head_dim >> 3);
+  if (total == 0) return cudaSuccess;
+  const int threads = 256;
+  const int64_t blocks = (total + threads - 1) / threads;
+  kv_append_kernel<<<static_cast<unsigned>(blocks), threads, 0, st>>>(
+      pv, slots, n_tok, layer_begin, layer_count, static_cast<const uint4 *>(k_new),
+      static_cast<const uint4 *>(v_new));
+  return cudaGetLastError();
+}
+
+cudaError_t launch_kv_read(const PoolView &pv, const int32_t *slots, int32_t n_tok, int32_t layer,
+                           void *k_out, void *v_out, cudaStream_t st) {
+  const int64_t total = static_cast<int64_t>(n_tok) * pv.n_kv_heads * 2 * (pv.head_dim >> 3);
+  if (total == 0) return cudaSuccess;
+  const int threads = 256;
+  const int64_t blocks = (total + threads - 1) / threads;
+  kv_read_kernel<<<static_cast<unsigned>(blocks), threads, 0, st>>>(
+      pv, slots, n_tok, layer, static_cast<uint4 *>(k_out), static_cast<uint4 *>(v_out));
+  return cudaGetLastError();
+}
+
+// =============================================================================================
+// K3: warp-shuffle pass.  One warp = one w-unit = (query, kv head, <= chunk tokens of one stream).
+// Pages are bulk-copied into a per-warp ring of shared-memory stages.  Scores: lane (r, s) holds
+// token r of the page and half s of the head dim, halves are combined with one shuffle; the
+// running maximum is a shuffle reduction over the 16 tokens.  P.V: every lane owns D/32 output
+// elements for each of the G heads.
+// =============================================================================================
+constexpr int W_WARPS = 8;
+constexpr int W_STAGES = 3;
+
+template <int D, int G>
+struct WarpSmem {
+  static constexpr int BLOCK = D * 64;
+  static constexpr int Q_BYTES = G * D * 4;
+  static constexpr int P_BYTES = 16 * G * 4;
+  static constexpr int BAR_BYTES = 64;
+  static constexpr int PER_WARP = W_STAGES * BLOCK + Q_BYTES + P_BYTES + BAR_BYTES;
+  static constexpr int TOTAL = PER_WARP * W_WARPS;
+};
+
+template <int D, int G>
+__global__ void __launch_bounds__(W_WARPS * 32)
+attn_warp_kernel(PoolView pv, int32_t off_wunit, int32_t off_pages, int32_t n_wunits, int32_t t_rows,
+                 int32_t n_queries, int32_t layer_begin, int32_t layer_count,
+                 const __nv_bfloat16 *__restrict__ q, float scale_log2) {
+  using S = WarpSmem<D, G>;
+  constexpr int NH = D / 64;
+  constexpr int E = D / 32;            // output elements per lane
+  constexpr int CH = D / 16;           // 16-byte chunks of a K row handled by one lane
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int64_t gw = static_cast<int64_t>(blockIdx.x) * W_WARPS + warp;
+  if (gw >= static_cast<int64_t>(n_wunits) * layer_count) return;
+  const int ll = static_cast<int>(gw / n_wunits);
+  const int u = static_cast<int>(gw % n_wunits);
+
+  uint8_t *base = smem_raw + warp * S::PER_WARP;
+  uint8_t *stages = base;
+  float *q_s = reinterpret_cast<float *>(base + W_STAGES * S::BLOCK);
+  float *p_s = reinterpret_cast<float *>(base + W_STAGES * S::BLOCK + S::Q_BYTES);
+  const uint32_t bar0 = smem_u32(base + W_STAGES * S::BLOCK + S::Q_BYTES + S::P_BYTES);
+
+  const int32_t *U = pv.plan + off_wunit + u * PW_WORDS;
+  const int qi = U[PW_QUERY], g = U[PW_KV_HEAD], n_tok = U[PW_N_TOKENS];
+  const int32_t *pg = pv.plan + off_pages + U[PW_PAGE_OFF];
+  const int n_pg = (n_tok + PASTA_PAGE - 1) / PASTA_PAGE;
+  const uint8_t *kv_layer = pv.kv_base + (layer_begin + ll) * pv.layer_stride;
+
+  if (lane == 0) {
+    for (int s = 0; s < W_STAGES; ++s) mbar_init(bar0 + 8 * s, 1);
+    mbar_init_fence();
+    fence_proxy_async();
+  }
+  // the G query rows of this kv head, pre-multiplied by scale * log2(e)
+  {
+    const __nv_bfloat162 *qsrc = reinterpret_cast<const __nv_bfloat162 *>(
+        q + ((static_cast<int64_t>(ll) * n_queries + qi) * pv.n_q_heads + g * G) * D);
+    for (int i = lane; i < G * D / 2; i += 32) {
+      const float2 f = __bfloat1622float2(qsrc[i]);
+      q_s[2 * i] = f.x * scale_log2;
+      q_s[2 * i + 1] = f.y * scale_log2;
+    }
+  }
+  __syncwarp();
+
+  auto issue = [&](int i) {
+    if (lane == 0) {
+      int page = pg[i];
+      if (page < 0 || page >= pv.n_pages) { report(pv.status, PASTA_ERR_DEVICE_CHECK); page = 0; }
+      const int s = i % W_STAGES;
+      fence_proxy_async();            // the lanes' reads of this stage (ordered by __syncwarp) precede the refill
+      mbar_expect_tx(bar0 + 8 * s, S::BLOCK);
+      bulk_g2s(smem_u32(stages + s * S::BLOCK),
+               kv_layer + (static_cast<int64_t>(page) * pv.n_kv_heads + g) * S::BLOCK, S::BLOCK, bar0 + 8 * s);
+    }
+  };
+  for (int i = 0; i < W_STAGES && i < n_pg; ++i) issue(i);
+
+  float m[G], l[G], o[G][E];
+#pragma unroll
+  for (int h = 0; h < G; ++h) {
+    m[h] = -INFINITY; l[h] = 0.f;
+#pragma unroll
+    for (int e = 0; e < E; ++e) o[h][e] = 0.f;
+  }
+  const int r = lane & 15, sub = lane >> 4;
+  int issued = min(W_STAGES, n_pg), consumed = 0;
+  bool ok = true;
+
+  for (int i = 0; i < n_pg; ++i) {
+    const int s = i % W_STAGES;
+    if (!mbar_wait_bounded(bar0 + 8 * s, (i / W_STAGES) & 1)) { ok = false; consumed = i; break; }
+    const uint8_t *sp = stages + s * S::BLOCK;
+    const int nv = min(PASTA_PAGE, n_tok - i * PASTA_PAGE);
+
+    float acc[G];
+#pragma unroll
+    for (int h = 0; h < G; ++h) acc[h] = 0.f;
+#pragma unroll
+    for (int cc = 0; cc < CH; ++cc) {
+      const int c = sub * CH + cc;
+      const uint4 kk = *reinterpret_cast<const uint4 *>(sp + kv_chunk_offset(NH, 0, r, c));
+      const float k0 = bf16_lo(kk.x), k1 = bf16_hi(kk.x), k2 = bf16_lo(kk.y), k3 = bf16_hi(kk.y);
+      const float k4 = bf16_lo(kk.z), k5 = bf16_hi(kk.z), k6 = bf16_lo(kk.w), k7 = bf16_hi(kk.w);
+#pragma unroll
+      for (int h = 0; h < G; ++h) {
+        const float4 qa = *reinterpret_cast<const float4 *>(q_s + h * D + c * 8);
+        const float4 qb = *reinterpret_cast<const float4 *>(q_s + h * D + c * 8 + 4);
+        acc[h] = fmaf(k0, qa.x, acc[h]); acc[h] = fmaf(k1, qa.y, acc[h]);
+        acc[h] = fmaf(k2, qa.z, acc[h]); acc[h] = fmaf(k3, qa.w, acc[h]);
+        acc[h] = fmaf(k4, qb.x, acc[h]); acc[h] = fmaf(k5, qb.y, acc[h]);
+        acc[h] = fmaf(k6, qb.z, acc[h]); acc[h] = fmaf(k7, qb.w, acc[h]);
+      }
+    }
+#pragma unroll
+    for (int h = 0; h < G; ++h) {
+      float sc = acc[h] + __shfl_xor_sync(0xffffffffu, acc[h], 16);
+      if (r >= nv) sc = -INFINITY;
+      float mx = sc;
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 8));
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 4));
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+      const float m_new = fmaxf(m[h], mx);          // finite: nv >= 1
+      const float corr = fast_exp2(m[h] - m_new);   // 0 on the first page
+      const float pj = fast_exp2(sc - m_new);       // 0 for masked rows
+      l[h] = l[h] * corr + (sub == 0 ? pj : 0.f);
+      m[h] = m_new;
+#pragma unroll
+      for (int e = 0; e < E; ++e) o[h][e] *= corr;
+      if (sub == 0) p_s[r * G + h] = pj;
+    }
+    __syncwarp();
+    {
+      const int c = (lane * E) >> 3;                // chunk that holds this lane's elements
+      const int within = ((lane * E) & 7) * 2;      // byte offset inside the chunk
+      for (int r2 = 0; r2 < nv; ++r2) {
+        const uint8_t *vp = sp + kv_chunk_offset(NH, 1, r2, c) + within;
+        float v[E];
+        if constexpr (E == 4) {
+          const uint2 vv = *reinterpret_cast<const uint2 *>(vp);
+          v[0] = bf16_lo(vv.x); v[1] = bf16_hi(vv.x); v[2] = bf16_lo(vv.y); v[3] = bf16_hi(vv.y);
+        } else {
+          const uint32_t vv = *reinterpret_cast<const uint32_t *>(vp);
+          v[0] = bf16_lo(vv); v[1] = bf16_hi(vv);
+        }
+#pragma unroll
+        for (int h = 0; h < G; ++h) {
+          const float ph = p_s[r2 * G + h];
+#pragma unroll
+          for (int e = 0; e < E; ++e) o[h][e] = fmaf(ph, v[e], o[h][e]);
+        }
+      }
+    }
+    __syncwarp();                                   // every lane is done with stage s and with p_s
+    if (i + W_STAGES < n_pg) { issue(i + W_STAGES); ++issued; }
+  }
+
+  if (!ok) {
+    // give up: report, then wait (bounded) for the copies still in flight before leaving
+    if (lane == 0) report(pv.status, PASTA_ERR_TIMEOUT);
+    for (int j = consumed; j < issued; ++j) mbar_wait_bounded(bar0 + 8 * (j % W_STAGES), (j / W_STAGES) & 1);
+    return;
+  }
+
+  const int64_t row0 = static_cast<int64_t>(ll) * pv.rows_per_layer + t_rows + static_cast<int64_t>(u) * G;
+#pragma unroll
+  for (int h = 0; h < G; ++h) {
+    float lt = l[h];
+    lt += __shfl_xor_sync(0xffffffffu, lt, 16);
+    lt += __shfl_xor_sync(0xffffffffu, lt, 8);
+    lt += __shfl_xor_sync(0xffffffffu, lt, 4);
+    lt += __shfl_xor_sync(0xffffffffu, lt, 2);
+    lt += __shfl_xor_sync(0xffffffffu, lt, 1);
+    if (lane == 0) pv.part_ml[row0 + h] = make_float2(m[h], lt);
+    float *dst = pv.part_o + (row0 + h) * D + lane * E;
+    if constexpr (E == 4) *reinterpret_cast<float4 *>(dst) = make_float4(o[h][0], o[h][1], o[h][2], o[h][3]);
+    else *reinterpret_cast<float2 *>(dst) = make_float2(o[h][0], o[h][1]);
+  }
+}
+
+template <int D, int G>
+static cudaError_t launch_warp_t(const PoolView &pv, const PlanHeader &h, int32_t layer_begin, int32_t layer_count,
+                                 const void *q, float scale_log2, cudaStream_t st) {
+  using S = WarpSmem<D, G>;
+  static bool prepared = false;
+  if (!prepared) {
+    cudaError_t e = cudaFuncSetAttribute(attn_warp_kernel<D, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, S::TOTAL);
+    if (e != cudaSuccess) return e;
+    prepared = true;
+  }
+  const int64_t warps = static_cast<int64_t>(h.w[PH_N_WUNITS]) * layer_count;
+  if (warps == 0) return cudaSuccess;
+  const int64_t blocks = (warps + W_WARPS - 1) / W_WARPS;
+  attn_warp_kernel<D, G><<<static_cast<unsigned>(blocks), W_WARPS * 32, S::TOTAL, st>>>(
+      pv, h.w[PH_OFF_WUNIT], h.w[PH_OFF_PAGES], h.w[PH_N_WUNITS], h.w[PH_T_ROWS], h.w[PH_N_QUERIES], layer_begin,
+      layer_count, static_cast<const __nv_bfloat16 *>(q), scale_log2);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_attn_warp(const PoolView &pv, const PlanHeader &h, int32_t layer_begin, int32_t layer_count,
+                             const void *q, float scale_log2, cudaStream_t st) {
+  const int G = pv.n_q_heads / pv.n_kv_heads;
+#define PASTA_W(DD, GG) \
+  if (pv.head_dim == DD && G == GG) return launch_warp_t<DD, GG>(pv, h, layer_begin, layer_count, q, scale_log2, st);
+  PASTA_W(128, 1) PASTA_W(128, 2) PASTA_W(128, 4) PASTA_W(128, 8)
+  PASTA_W(64, 1) PASTA_W(64, 2) PASTA_W(64, 4) PASTA_W(64, 8)
+#undef PASTA_W
+  return cudaErrorInvalidValue;
+}
+
+// =============================================================================================
+// K4: log-sum-exp merge.  One warp per (layer, query, head): m* = max m_i,
+// out = sum_i 2^(m_i - m*) O_i / sum_i 2^(m_i - m*) l_i,  lse = ln2 * (m* + log2 of that sum).
+// =============================================================================================
+__global__ void __launch_bounds__(256)
+merge_kernel(PoolView pv, int32_t n_queries, int32_t layer_count, int32_t off_query, int32_t off_trange,
+             int32_t off_tunit, int32_t t_rows, float *__restrict__ out, float *__restrict__ lse) {
+  const int D = pv.head_dim, Hq = pv.n_q_heads, G = Hq / pv.n_kv_heads;
+  const int64_t gw = (static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x) >> 5;
+  const int lane = threadIdx.x & 31;
+  if (gw >= static_cast<int64_t>(layer_count) * n_queries * Hq) return;
+  const int h = static_cast<int>(gw % Hq);
+  const int n = static_cast<int>((gw / Hq) % n_queries);
+  const int ll = static_cast<int>(gw / (static_cast<int64_t>(Hq) * n_queries));
+  const int g = h / G, hl = h % G;
+  const int32_t *Q = pv.plan + off_query + n * PQ_WORDS;
+  const int treq = Q[PQ_TREQ], tidx = Q[PQ_TIDX], w0 = Q[PQ_WUNIT0], nw = Q[PQ_NW];
+  int tb = 0, nt = 0;
+  if (treq >= 0) {
+    tb = pv.plan[off_trange + (treq * pv.n_kv_heads + g) * 2];
+    nt = pv.plan[off_trange + (treq * pv.n_kv_heads + g) * 2 + 1] - tb;
+  }
+  const int total = nt + nw;
+  const int64_t lbase = static_cast<int64_t>(ll) * pv.rows_per_layer;
+  auto row_of = [&](int i) -> int64_t {
+    if (i < nt) return lbase + pv.plan[off_tunit + (tb + i) * PU_WORDS + PU_ROW_BASE] + tidx * G + hl;
+    return lbase + t_rows + static_cast<int64_t>(w0 + g * nw + (i - nt)) * G + hl;
+  };
+  float mstar = -INFINITY;
+  for (int i = lane; i < total; i += 32) {
+    const float2 ml = pv.part_ml[row_of(i)];
+    if (ml.y > 0.f) mstar = fmaxf(mstar, ml.x);
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) mstar = fmaxf(mstar, __shfl_xor_sync(0xffffffffu, mstar, o));
+  const int E = D >> 5;                    // 4 or 2 elements per lane
+  float acc[4] = {0.f, 0.f, 0.f, 0.f};
+  float L = 0.f;
+  for (int i = 0; i < total; ++i) {
+    const int64_t row = row_of(i);
+    const float2 ml = pv.part_ml[row];
+    if (!(ml.y > 0.f)) continue;           // nothing visible in that piece
+    const float w = fast_exp2(ml.x - mstar);
+    L = fmaf(w, ml.y, L);
+    const float *src = pv.part_o + row * D + lane * E;
+    if (E == 4) {
+      const float4 v = *reinterpret_cast<const float4 *>(src);
+      acc[0] = fmaf(w, v.x, acc[0]); acc[1] = fmaf(w, v.y, acc[1]);
+      acc[2] = fmaf(w, v.z, acc[2]); acc[3] = fmaf(w, v.w, acc[3]);
+    } else {
+      const float2 v = *reinterpret_cast<const float2 *>(src);
+      acc[0] = fmaf(w, v.x, acc[0]); acc[1] = fmaf(w, v.y, acc[1]);
+    }
+  }
+  const float inv = L > 0.f ? 1.f / L : 0.f;
+  float *dst = out + ((static_cast<int64_t>(ll) * n_queries + n) * Hq + h) * D + lane * E;
+  if (E == 4) *reinterpret_cast<float4 *>(dst) = make_float4(acc[0] * inv, acc[1] * inv, acc[2] * inv, acc[3] * inv);
+  else *reinterpret_cast<float2 *>(dst) = make_float2(acc[0] * inv, acc[1] * inv);
+  if (lse && lane == 0)
+    lse[(static_cast<int64_t>(ll) * n_queries + n) * Hq + h] = (mstar + log2f(L)) * 0.6931471805599453f;
+}
+
+cudaError_t launch_merge(const PoolView &pv, const PlanHeader &h, int32_t layer_count, float *out, float *lse,
+                         cudaStream_t st) {
+  const int64_t warps = static_cast<int64_t>(layer_count) * h.w[PH_N_QUERIES] * pv.n_q_heads;
+  if (warps == 0) return cudaSuccess;
+  const int64_t blocks = (warps * 32 + 255) / 256;
+  merge_kernel<<<static_cast<unsigned>(blocks), 256, 0, st>>>(pv, h.w[PH_N_QUERIES], layer_count, h.w[PH_OFF_QUERY],
+                                                              h.w[PH_OFF_TRANGE], h.w[PH_OFF_TUNIT], h.w[PH_T_ROWS],
+                                                              out, lse);
+  return cudaGetLastError();
+}
+
+}  // namespace pasta

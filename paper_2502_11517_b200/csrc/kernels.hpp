@@ -1,0 +1,32 @@
+// Host-callable launchers of the CUDA kernels.  Each returns the cudaError_t of its launch.
+#pragma once
+#include <cuda_runtime.h>
+
+#include <cstdint>
+
+namespace pasta {
+
+struct PoolView;   // device_common.cuh
+
+struct PlanHeader {            // host copy of the plan's header words
+  int32_t w[32];
+};
+
+// K1: copies the new tokens of `layer_count` layers into their slots.  slots: device, 2 words per token.
+cudaError_t launch_kv_append(const PoolView &pv, const int32_t *slots, int32_t n_tok, int32_t layer_begin,
+                             int32_t layer_count, const void *k_new, const void *v_new, cudaStream_t st);
+// inverse of K1 for one layer: gathers the listed slots into dense [n_tok, Hkv, D] arrays
+cudaError_t launch_kv_read(const PoolView &pv, const int32_t *slots, int32_t n_tok, int32_t layer,
+                           void *k_out, void *v_out, cudaStream_t st);
+// K3: warp-shuffle pass over streams seen by one query
+cudaError_t launch_attn_warp(const PoolView &pv, const PlanHeader &h, int32_t layer_begin, int32_t layer_count,
+                             const void *q, float scale_log2, cudaStream_t st);
+// K2: tensor-core pass over streams shared by several queries (head_dim 128 only)
+cudaError_t launch_attn_tensor(const PoolView &pv, const PlanHeader &h, int32_t layer_begin, int32_t layer_count,
+                               const void *q, float scale_log2, cudaStream_t st);
+bool tensor_path_available();       // false while the tensor-core kernel is compiled out
+// K4: log-sum-exp merge of all partial rows of every (query, head)
+cudaError_t launch_merge(const PoolView &pv, const PlanHeader &h, int32_t layer_count, float *out, float *lse,
+                         cudaStream_t st);
+
+}  // namespace pasta

@@ -1,0 +1,90 @@
+// The step plan: what pasta_step_begin builds on the host and uploads, and what the kernels read.
+// One array of int32 words; a header of word offsets followed by tables.  Page ids are shared by
+// all layers, so one plan serves every layer of the step.
+//
+// Terms
+//   query      one (request, thread) entry of the step, index n in entry order
+//   stream     one page list: a request's main-thread tokens (id 0) or one fork's chunk (id = fork id).
+//              Every thread sees a PREFIX [0, vis) of every stream (vis may be 0).
+//   t-request  a request with at least one stream seen by >= 2 queries of the step ("shared").
+//              Its shared streams' pages are concatenated into one page list that is cut into
+//              tiles of PASTA_TILE_PAGES pages; rows of the score matrix are the request's queries
+//              times the `group` query heads of one kv head: row = t_idx * group + h_local.
+//   t-unit     (t-request, kv head, tile range): one CTA-sized piece of the tensor-core kernel; it
+//              writes one partial result (m, l, O[d]) per row.
+//   w-unit     (query, kv head, token range of one stream seen by that query alone): one warp of
+//              the warp-shuffle kernel; it writes `group` partial rows.
+//   partial rows are numbered per layer: t-unit rows first (row_base + row), then
+//              t_rows + w_unit * group + h_local.
+#pragma once
+#include <cstdint>
+
+#define PASTA_PLAN_MAGIC 0x50415354
+#define PASTA_TILE_PAGES 4          // pages per tensor-core tile (64 tokens)
+#define PASTA_PAGE 16               // tokens per page
+#define PASTA_MAX_ROWS 128          // rows of the stacked-query matrix (threads * group)
+
+// header words
+enum {
+  PH_MAGIC = 0,
+  PH_N_QUERIES,
+  PH_N_APPEND,        // entries with n_new == 1
+  PH_N_TREQ,
+  PH_N_TUNITS,
+  PH_N_WUNITS,
+  PH_T_ROWS,          // partial rows written by t-units
+  PH_ROWS,            // all partial rows of one layer
+  PH_T_GRID,          // CTAs of the tensor-core kernel that have work
+  PH_OFF_APPEND,      // 2 words per appended token: page, offset
+  PH_OFF_QUERY,       // PQ_WORDS per query
+  PH_OFF_TREQ,        // PT_WORDS per t-request
+  PH_OFF_TRANGE,      // per (t-request, kv head): first t-unit, one past the last
+  PH_OFF_TUNIT,       // PU_WORDS per t-unit
+  PH_OFF_TCTA,        // per CTA: first t-unit, one past the last
+  PH_OFF_WUNIT,       // PW_WORDS per w-unit
+  PH_OFF_PAGES,       // page ids
+  PH_OFF_PMETA,       // parallel to pages (t-request lists only): (page index in its stream << 8) | local stream
+  PH_OFF_VIS,         // per t-request: [n_threads][n_streams] visible length of local stream for thread
+  PH_OFF_TQ,          // per t-request: [n_threads] query index of each row-thread
+  PH_TOTAL_WORDS,
+  PH_WORDS = 32
+};
+
+// per query
+enum {
+  PQ_TREQ = 0,        // t-request index or -1
+  PQ_TIDX,            // row-thread index inside the t-request
+  PQ_WUNIT0,          // first w-unit of this query; w-unit of (kv head g, piece k) = WUNIT0 + g * NW + k
+  PQ_NW,              // w-units per kv head
+  PQ_WORDS
+};
+
+// per t-request
+enum {
+  PT_PAGE_OFF = 0,    // index into pages / pmeta
+  PT_N_PAGES,
+  PT_N_THREADS,
+  PT_N_STREAMS,
+  PT_VIS_OFF,         // index into vis
+  PT_TQ_OFF,          // index into tq
+  PT_WORDS
+};
+
+// per t-unit
+enum {
+  PU_TREQ = 0,
+  PU_KV_HEAD,
+  PU_TILE_BEGIN,
+  PU_TILE_END,
+  PU_ROW_BASE,
+  PU_WORDS
+};
+
+// per w-unit
+enum {
+  PW_QUERY = 0,
+  PW_KV_HEAD,
+  PW_PAGE_OFF,        // index into pages of the unit's first page
+  PW_N_TOKENS,        // tokens of the unit, starting at the first token of that page
+  PW_WORDS
+};

@@ -1,0 +1,302 @@
+// Builds the step plan (see pasta_plan.h) from the pool's bookkeeping.  Host only.
+#include "plan.hpp"
+
+#include <algorithm>
+#include <cmath>
+
+namespace pasta {
+
+namespace {
+
+struct StreamUse {
+  int32_t stream;
+  int32_t n_seen;                 // queries of the step that see a non-empty prefix of it
+  int32_t max_vis;
+  int32_t local = -1;             // index among the t-request's shared streams
+  int32_t page_off = -1;          // where its pages were put in the page table (w-units)
+};
+
+struct WPiece {                   // one stream seen by one query alone
+  int32_t query, page_off, vis;
+};
+
+struct TReq {
+  int32_t page_off, n_pages, n_threads, n_streams, vis_off, tq_off;
+};
+
+struct TUnit {
+  int32_t treq, g, tile_begin, tile_end, row_base;
+};
+
+}  // namespace
+
+pasta_status_t build_plan(const HostPool &pool, const std::vector<StepEntry> &entries,
+                          const std::vector<Slot> &slots, const PlanLimits &lim,
+                          std::vector<int32_t> *out) {
+  const int32_t n = static_cast<int32_t>(entries.size());
+  const int32_t G = lim.n_q_heads / lim.n_kv_heads;
+  const int32_t P = PASTA_PAGE;
+  if (n > lim.max_queries) return PASTA_ERR_CAPACITY;
+
+  // ---- group the queries by request, in order of first appearance
+  std::vector<int32_t> req_order;
+  std::vector<std::vector<int32_t>> by_req;
+  {
+    std::vector<std::pair<int32_t, int32_t>> first;   // (req, group index), small linear map would be O(n^2)
+    std::vector<int32_t> slot_of;
+    for (int32_t i = 0; i < n; ++i) {
+      const int32_t r = entries[i].req;
+      if (r >= static_cast<int32_t>(slot_of.size())) slot_of.resize(r + 1, -1);
+      if (slot_of[r] < 0) {
+        slot_of[r] = static_cast<int32_t>(by_req.size());
+        req_order.push_back(r);
+        by_req.emplace_back();
+      }
+      by_req[slot_of[r]].push_back(i);
+    }
+  }
+
+  std::vector<int32_t> pages, pmeta, vis_tab, tq_tab;
+  std::vector<TReq> treqs;
+  std::vector<WPiece> wpieces;
+  std::vector<int32_t> q_treq(n, -1), q_tidx(n, 0);
+  std::vector<int32_t> vis_of;      // scratch: stream -> visible length for the current query
+  std::vector<int32_t> use_index;   // scratch: stream -> index in `uses`
+  int64_t w_tokens = 0;
+
+  for (size_t gi = 0; gi < by_req.size(); ++gi) {
+    const Request *r = pool.request(req_order[gi]);
+    const std::vector<int32_t> &qs = by_req[gi];
+    const int32_t T = static_cast<int32_t>(qs.size());
+    const int32_t n_streams_all = static_cast<int32_t>(r->streams.size());
+    use_index.assign(n_streams_all, -1);
+    std::vector<StreamUse> uses;
+    std::vector<std::vector<int32_t>> q_vis(T);       // per query: visible length per entry of `uses` (grown lazily)
+    for (int32_t ti = 0; ti < T; ++ti) {
+      const Thread &th = r->threads[entries[qs[ti]].thread];
+      vis_of.assign(n_streams_all, 0);
+      for (const Seg &s : th.view) vis_of[s.stream] = std::max(vis_of[s.stream], s.start + s.len);
+      for (const Seg &s : th.view) {
+        if (use_index[s.stream] < 0) {
+          use_index[s.stream] = static_cast<int32_t>(uses.size());
+          uses.push_back(StreamUse{s.stream, 0, 0});
+        }
+      }
+      q_vis[ti].assign(uses.size(), 0);
+      for (size_t u = 0; u < uses.size(); ++u) {
+        const int32_t v = vis_of[uses[u].stream];
+        q_vis[ti][u] = v;
+        if (v > 0) {
+          // count each (query, stream) once: views list a stream several times only for the main stream pieces
+          uses[u].n_seen += 1;
+          uses[u].max_vis = std::max(uses[u].max_vis, v);
+        }
+      }
+    }
+    for (int32_t ti = 0; ti < T; ++ti) q_vis[ti].resize(uses.size(), 0);
+
+    bool tensor = lim.tensor_path && T >= 2 && T * G <= PASTA_MAX_ROWS;
+    int32_t n_shared = 0;
+    if (tensor) {
+      for (StreamUse &u : uses)
+        if (u.n_seen >= 2) u.local = n_shared++;
+      if (n_shared == 0 || n_shared > 255) {
+        tensor = false;
+        for (StreamUse &u : uses) u.local = -1;
+      }
+    }
+    if (tensor) {
+      TReq t;
+      t.page_off = static_cast<int32_t>(pages.size());
+      t.n_threads = T;
+      t.n_streams = n_shared;
+      t.vis_off = static_cast<int32_t>(vis_tab.size());
+      t.tq_off = static_cast<int32_t>(tq_tab.size());
+      for (const StreamUse &u : uses) {
+        if (u.local < 0) continue;
+        const std::vector<int32_t> &sp = r->streams[u.stream].pages;
+        const int32_t np = (u.max_vis + P - 1) / P;
+        for (int32_t k = 0; k < np; ++k) {
+          pages.push_back(sp[k]);
+          pmeta.push_back((k << 8) | u.local);
+        }
+      }
+      t.n_pages = static_cast<int32_t>(pages.size()) - t.page_off;
+      for (int32_t ti = 0; ti < T; ++ti) {
+        for (size_t u = 0; u < uses.size(); ++u)
+          if (uses[u].local >= 0) vis_tab.push_back(q_vis[ti][u]);   // uses are in local order
+        tq_tab.push_back(qs[ti]);
+        q_treq[qs[ti]] = static_cast<int32_t>(treqs.size());
+        q_tidx[qs[ti]] = ti;
+      }
+      treqs.push_back(t);
+    }
+    // streams that stay on the warp path: their pages are stored once per request
+    for (int32_t ti = 0; ti < T; ++ti) {
+      for (size_t u = 0; u < uses.size(); ++u) {
+        if (uses[u].local >= 0 || q_vis[ti][u] == 0) continue;
+        if (uses[u].page_off < 0) {
+          uses[u].page_off = static_cast<int32_t>(pages.size());
+          const std::vector<int32_t> &sp = r->streams[uses[u].stream].pages;
+          const int32_t np = (uses[u].max_vis + P - 1) / P;
+          pages.insert(pages.end(), sp.begin(), sp.begin() + np);
+          pmeta.insert(pmeta.end(), np, 0);
+        }
+        wpieces.push_back(WPiece{qs[ti], uses[u].page_off, q_vis[ti][u]});
+        w_tokens += q_vis[ti][u];
+      }
+    }
+  }
+
+  // ---- t-units: cut the sequence of (t-request, kv head) tile runs into one contiguous range per CTA
+  std::vector<TUnit> tunits;
+  std::vector<int32_t> trange(treqs.size() * lim.n_kv_heads * 2, 0);
+  std::vector<int32_t> tcta;
+  int32_t t_rows = 0;
+  if (!treqs.empty()) {
+    const double overhead = 2.0;           // cost of starting a unit, in tiles
+    const int32_t min_piece = 4;           // do not leave fragments smaller than this many tiles
+    double total = 0;
+    for (const TReq &t : treqs)
+      total += lim.n_kv_heads * ((t.n_pages + PASTA_TILE_PAGES - 1) / PASTA_TILE_PAGES + overhead);
+    const int32_t grid = std::max(1, lim.grid);
+    const double target = total / grid;
+    int32_t cta = 0;
+    double acc = 0;
+    tcta.assign(2 * grid, 0);
+    auto close_cta = [&]() {
+      tcta[2 * cta + 1] = static_cast<int32_t>(tunits.size());
+      if (cta + 1 < grid) {
+        ++cta;
+        tcta[2 * cta] = tcta[2 * cta + 1] = static_cast<int32_t>(tunits.size());
+        acc = 0;
+      }
+    };
+    for (size_t ti = 0; ti < treqs.size(); ++ti) {
+      const int32_t n_tiles = (treqs[ti].n_pages + PASTA_TILE_PAGES - 1) / PASTA_TILE_PAGES;
+      const int32_t rows = treqs[ti].n_threads * G;
+      for (int32_t g = 0; g < lim.n_kv_heads; ++g) {
+        trange[(ti * lim.n_kv_heads + g) * 2] = static_cast<int32_t>(tunits.size());
+        int32_t begin = 0;
+        while (begin < n_tiles) {
+          const int32_t remaining = n_tiles - begin;
+          int32_t take = remaining;
+          if (cta + 1 < grid) {
+            const double room = target - acc - overhead;
+            if (room < std::min(remaining, min_piece)) {
+              if (acc > 0) { close_cta(); continue; }
+            } else if (room < remaining) {
+              take = static_cast<int32_t>(room);
+              if (remaining - take < min_piece) take = remaining;   // no tiny tail
+            }
+          }
+          tunits.push_back(TUnit{static_cast<int32_t>(ti), g, begin, begin + take, t_rows});
+          t_rows += rows;
+          begin += take;
+          acc += take + overhead;
+          if (cta + 1 < grid && acc >= target - 0.5) close_cta();
+        }
+        trange[(ti * lim.n_kv_heads + g) * 2 + 1] = static_cast<int32_t>(tunits.size());
+      }
+    }
+    tcta[2 * cta + 1] = static_cast<int32_t>(tunits.size());
+    int32_t used = cta + 1;
+    while (used > 0 && tcta[2 * (used - 1)] == tcta[2 * (used - 1) + 1]) --used;
+    tcta.resize(2 * used);
+  }
+
+  // ---- w-units: pieces of at most `chunk` tokens, ordered (query, kv head, piece)
+  int32_t chunk;
+  {
+    const double want_warps = 16.0 * std::max(1, lim.grid);
+    double c = std::ceil(static_cast<double>(w_tokens) * lim.n_kv_heads / want_warps / P) * P;
+    chunk = static_cast<int32_t>(std::min(1024.0, std::max(64.0, c)));
+  }
+  std::vector<int32_t> q_nw(n, 0), q_w0(n, 0);
+  int64_t n_wunits = 0;
+  for (;;) {
+    std::fill(q_nw.begin(), q_nw.end(), 0);
+    for (const WPiece &w : wpieces) q_nw[w.query] += (w.vis + chunk - 1) / chunk;
+    n_wunits = 0;
+    for (int32_t i = 0; i < n; ++i) n_wunits += static_cast<int64_t>(q_nw[i]) * lim.n_kv_heads;
+    if (t_rows + n_wunits * G <= lim.max_rows) break;
+    if (chunk >= (1 << 24)) return PASTA_ERR_CAPACITY;
+    chunk *= 2;
+  }
+  {
+    int32_t w0 = 0;
+    for (int32_t i = 0; i < n; ++i) { q_w0[i] = w0; w0 += q_nw[i] * lim.n_kv_heads; }
+  }
+  std::vector<int32_t> wunits(static_cast<size_t>(n_wunits) * PW_WORDS);
+  {
+    std::vector<int32_t> next(n, 0);       // next piece index k of each query
+    // pieces of one query are contiguous in wpieces only per request group; index by query instead
+    for (const WPiece &w : wpieces) {
+      for (int32_t begin = 0; begin < w.vis; begin += chunk) {
+        const int32_t k = next[w.query]++;
+        for (int32_t g = 0; g < lim.n_kv_heads; ++g) {
+          int32_t *u = &wunits[static_cast<size_t>(q_w0[w.query] + g * q_nw[w.query] + k) * PW_WORDS];
+          u[PW_QUERY] = w.query;
+          u[PW_KV_HEAD] = g;
+          u[PW_PAGE_OFF] = w.page_off + begin / P;
+          u[PW_N_TOKENS] = std::min(chunk, w.vis - begin);
+        }
+      }
+    }
+  }
+
+  // ---- assemble
+  int32_t n_app = 0;
+  for (const StepEntry &e : entries) n_app += e.n_new;
+  std::vector<int32_t> &w = *out;
+  w.assign(PH_WORDS, 0);
+  auto put = [&](int off_field, const std::vector<int32_t> &v) {
+    w[off_field] = static_cast<int32_t>(w.size());
+    w.insert(w.end(), v.begin(), v.end());
+    while (w.size() % 4) w.push_back(0);   // keep every table 16-byte aligned
+  };
+  std::vector<int32_t> app;
+  for (int32_t i = 0; i < n; ++i)
+    if (entries[i].n_new) { app.push_back(slots[i].page); app.push_back(slots[i].offset); }
+  std::vector<int32_t> qtab(static_cast<size_t>(n) * PQ_WORDS);
+  for (int32_t i = 0; i < n; ++i) {
+    qtab[i * PQ_WORDS + PQ_TREQ] = q_treq[i];
+    qtab[i * PQ_WORDS + PQ_TIDX] = q_tidx[i];
+    qtab[i * PQ_WORDS + PQ_WUNIT0] = q_w0[i];
+    qtab[i * PQ_WORDS + PQ_NW] = q_nw[i];
+  }
+  std::vector<int32_t> ttab, utab;
+  for (const TReq &t : treqs) {
+    const int32_t rec[PT_WORDS] = {t.page_off, t.n_pages, t.n_threads, t.n_streams, t.vis_off, t.tq_off};
+    ttab.insert(ttab.end(), rec, rec + PT_WORDS);
+  }
+  for (const TUnit &u : tunits) {
+    const int32_t rec[PU_WORDS] = {u.treq, u.g, u.tile_begin, u.tile_end, u.row_base};
+    utab.insert(utab.end(), rec, rec + PU_WORDS);
+  }
+  w[PH_MAGIC] = PASTA_PLAN_MAGIC;
+  w[PH_N_QUERIES] = n;
+  w[PH_N_APPEND] = n_app;
+  w[PH_N_TREQ] = static_cast<int32_t>(treqs.size());
+  w[PH_N_TUNITS] = static_cast<int32_t>(tunits.size());
+  w[PH_N_WUNITS] = static_cast<int32_t>(n_wunits);
+  w[PH_T_ROWS] = t_rows;
+  w[PH_ROWS] = t_rows + static_cast<int32_t>(n_wunits) * G;
+  w[PH_T_GRID] = static_cast<int32_t>(tcta.size() / 2);
+  put(PH_OFF_APPEND, app);
+  put(PH_OFF_QUERY, qtab);
+  put(PH_OFF_TREQ, ttab);
+  put(PH_OFF_TRANGE, trange);
+  put(PH_OFF_TUNIT, utab);
+  put(PH_OFF_TCTA, tcta);
+  put(PH_OFF_WUNIT, wunits);
+  put(PH_OFF_PAGES, pages);
+  put(PH_OFF_PMETA, pmeta);
+  put(PH_OFF_VIS, vis_tab);
+  put(PH_OFF_TQ, tq_tab);
+  w[PH_TOTAL_WORDS] = static_cast<int32_t>(w.size());
+  if (static_cast<int64_t>(w.size()) > lim.max_words) return PASTA_ERR_CAPACITY;
+  return PASTA_OK;
+}
+
+}  // namespace pasta

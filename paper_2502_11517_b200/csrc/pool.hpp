@@ -1,0 +1,83 @@
+// Host-side bookkeeping of the KV pool: pages, streams, threads and their segment lists.
+// Pure C++ (no CUDA): everything here is integers.
+//
+// Rules (Section 3 "Efficiency" of the paper for what a thread may see; paging and canonical
+// forms are this library's own):
+//  * a stream (main thread's tokens = stream 0, a fork's chunk = stream <fork id>) takes a page
+//    from the front of the free sequence whenever it appends a token whose index is a multiple of
+//    the page size;
+//  * a fork's view = copy of the main thread's view at spawn time + its own chunk;
+//  * merging puts a chunk right after the main-stream piece ending at the fork's cut-off,
+//    behind chunks with the same cut-off and a smaller id.
+#pragma once
+#include <cstdint>
+#include <deque>
+#include <vector>
+
+#include "../../include/pasta.h"
+
+namespace pasta {
+
+struct Seg {
+  int32_t stream, start, len;
+  int32_t anchor;  // cut-off of a merged chunk; -1 for pieces of the main stream and a fork's own chunk
+};
+
+struct Stream {
+  int32_t len = 0;
+  std::vector<int32_t> pages;
+};
+
+struct Thread {
+  int32_t state = PASTA_THREAD_ACTIVE;
+  int32_t cutoff = 0;
+  std::vector<Seg> view;
+};
+
+struct Request {
+  bool live = false;
+  std::vector<Stream> streams;   // index = stream id = thread id
+  std::vector<Thread> threads;   // index = thread id; 0 = main
+};
+
+struct StepEntry {
+  int32_t req, thread, n_new;
+};
+
+struct Slot {
+  int32_t page, offset;
+};
+
+class HostPool {
+ public:
+  HostPool(int32_t n_pages, int32_t page_size, const int32_t *free_order, int32_t max_requests,
+           int32_t max_threads, int32_t max_segments);
+
+  static bool valid_free_order(int32_t n_pages, const int32_t *free_order);
+
+  pasta_status_t request_begin(int32_t *out_req);
+  pasta_status_t request_end(int32_t req);
+  pasta_status_t thread_spawn(int32_t req, int32_t *out_thread);
+  pasta_status_t thread_finish(int32_t req, int32_t thread);
+  pasta_status_t sync_merge(int32_t req, int32_t n_threads, const int32_t *thread_ids);
+
+  // Validates the whole step first, then reserves; slots[i] = {-1,-1} when n_new == 0.
+  pasta_status_t reserve_step(const std::vector<StepEntry> &entries, std::vector<Slot> *slots);
+  pasta_status_t reserve_run(int32_t req, int32_t thread, int32_t m, std::vector<Slot> *slots);
+
+  const Request *request(int32_t req) const;
+  int32_t page_size() const { return page_size_; }
+  int32_t n_pages() const { return n_pages_; }
+  void dump(std::vector<int32_t> *words) const;
+
+ private:
+  bool can_extend(const Request &r, int32_t thread) const;
+  Slot append_one(Request &r, int32_t thread);
+  Request *live(int32_t req);
+
+  int32_t n_pages_, page_size_, max_requests_, max_threads_, max_segments_;
+  std::deque<int32_t> free_;
+  std::vector<Request> requests_;
+};
+
+}  // namespace pasta

@@ -1,0 +1,86 @@
+"""Executes a step plan (the int32 words pasta_step_begin uploads) with NumPy, unit by unit, the way
+the kernels are meant to: every t-unit and w-unit yields partial (m, l, O) rows, the merge combines
+them.  It lets the planner be checked against the oracle without a GPU.  Tests only."""
+import numpy as np
+
+# header word indices (pasta_plan.h)
+(PH_MAGIC, PH_N_QUERIES, PH_N_APPEND, PH_N_TREQ, PH_N_TUNITS, PH_N_WUNITS, PH_T_ROWS, PH_ROWS, PH_T_GRID,
+ PH_OFF_APPEND, PH_OFF_QUERY, PH_OFF_TREQ, PH_OFF_TRANGE, PH_OFF_TUNIT, PH_OFF_TCTA, PH_OFF_WUNIT, PH_OFF_PAGES,
+ PH_OFF_PMETA, PH_OFF_VIS, PH_OFF_TQ, PH_TOTAL_WORDS) = range(21)
+PQ, PT, PU, PW = 4, 6, 5, 4
+TILE_PAGES, PAGE = 4, 16
+
+
+def run_plan(w, K, V, q, n_kv_heads):
+    """w: plan words; K, V: [n_pages, 16, Hkv, d] float64; q: [n, Hq, d] float64 -> out [n, Hq, d], lse [n, Hq]."""
+    assert w[PH_MAGIC] == 0x50415354 and w[PH_TOTAL_WORDS] == len(w)
+    n, Hq, d = q.shape
+    G = Hq // n_kv_heads
+    scale = 1.0 / np.sqrt(d)
+    rows = int(w[PH_ROWS]); t_rows = int(w[PH_T_ROWS])
+    m = np.full(rows, np.nan); l = np.full(rows, np.nan); O = np.full((rows, d), np.nan)
+    pages, pmeta = w[w[PH_OFF_PAGES]:], w[w[PH_OFF_PMETA]:]
+    written = np.zeros(rows, dtype=int)
+
+    # every t-unit belongs to exactly one CTA range, ranges are contiguous and cover all units
+    cta = w[w[PH_OFF_TCTA]: w[PH_OFF_TCTA] + 2 * w[PH_T_GRID]].reshape(-1, 2)
+    if w[PH_N_TUNITS]:
+        assert cta[0, 0] == 0 and cta[-1, 1] == w[PH_N_TUNITS]
+        assert np.all(cta[1:, 0] == cta[:-1, 1]) and np.all(cta[:, 1] > cta[:, 0])
+
+    for u in range(w[PH_N_TUNITS]):
+        treq, g, tb, te, row_base = w[w[PH_OFF_TUNIT] + u * PU: w[PH_OFF_TUNIT] + (u + 1) * PU]
+        T = w[PH_OFF_TREQ] + treq * PT
+        page_off, n_pages, n_thr, n_str, vis_off, tq_off = w[T:T + PT]
+        assert 0 <= tb < te <= -(-n_pages // TILE_PAGES)
+        vis = w[w[PH_OFF_VIS] + vis_off: w[PH_OFF_VIS] + vis_off + n_thr * n_str].reshape(n_thr, n_str)
+        tq = w[w[PH_OFF_TQ] + tq_off: w[PH_OFF_TQ] + tq_off + n_thr]
+        for ti in range(n_thr):
+            for hl in range(G):
+                h = g * G + hl
+                s_all, v_all = [], []
+                for pi in range(tb * TILE_PAGES, min(te * TILE_PAGES, n_pages)):
+                    page, meta = pages[page_off + pi], pmeta[page_off + pi]
+                    thr = vis[ti, meta & 255] - (meta >> 8) * PAGE
+                    cnt = int(np.clip(thr, 0, PAGE))
+                    s_all.append(K[page, :cnt, g] @ q[tq[ti], h] * scale)
+                    v_all.append(V[page, :cnt, g])
+                s = np.concatenate(s_all); v = np.concatenate(v_all)
+                row = row_base + ti * G + hl
+                written[row] += 1
+                if len(s) == 0:
+                    m[row], l[row], O[row] = -np.inf, 0.0, 0.0
+                else:
+                    m[row] = s.max(); e = np.exp(s - m[row]); l[row] = e.sum(); O[row] = e @ v
+
+    for u in range(w[PH_N_WUNITS]):
+        qi, g, page_off, n_tok = w[w[PH_OFF_WUNIT] + u * PW: w[PH_OFF_WUNIT] + (u + 1) * PW]
+        assert n_tok > 0
+        for hl in range(G):
+            h = g * G + hl
+            ks = np.concatenate([K[pages[page_off + k], :, g] for k in range(-(-n_tok // PAGE))])[:n_tok]
+            vs = np.concatenate([V[pages[page_off + k], :, g] for k in range(-(-n_tok // PAGE))])[:n_tok]
+            s = ks @ q[qi, h] * scale
+            row = t_rows + u * G + hl
+            written[row] += 1
+            m[row] = s.max(); e = np.exp(s - m[row]); l[row] = e.sum(); O[row] = e @ vs
+    assert np.all(written == 1), "every partial row is written exactly once"
+
+    out = np.zeros((n, Hq, d)); lse = np.zeros((n, Hq))
+    tr = w[w[PH_OFF_TRANGE]:]
+    for i in range(n):
+        treq, tidx, w0, nw = w[w[PH_OFF_QUERY] + i * PQ: w[PH_OFF_QUERY] + (i + 1) * PQ]
+        for h in range(Hq):
+            g, hl = divmod(h, G)
+            rows_i = []
+            if treq >= 0:
+                for u in range(tr[(treq * n_kv_heads + g) * 2], tr[(treq * n_kv_heads + g) * 2 + 1]):
+                    assert w[w[PH_OFF_TUNIT] + u * PU] == treq and w[w[PH_OFF_TUNIT] + u * PU + 1] == g
+                    rows_i.append(w[w[PH_OFF_TUNIT] + u * PU + 4] + tidx * G + hl)
+            rows_i += [t_rows + (w0 + g * nw + k) * G + hl for k in range(nw)]
+            rows_i = [r for r in rows_i if l[r] > 0]
+            ms = max(m[r] for r in rows_i)
+            L = sum(np.exp(m[r] - ms) * l[r] for r in rows_i)
+            out[i, h] = sum(np.exp(m[r] - ms) * O[r] for r in rows_i) / L
+            lse[i, h] = ms + np.log(L)
+    return out, lse

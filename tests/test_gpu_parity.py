@@ -1,0 +1,181 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the fp64 oracle on the same seeded inputs.
+
+Indexing (slots, page tables, segment lists, the appended bits) must be bit-exact.  Attention must be
+within max-abs 1e-2 and mean-abs 1e-3 of the oracle (the stated target; bf16 inputs, bf16 softmax
+weights on the tensor-core path, fp32 accumulation)."""
+import numpy as np
+import pytest
+
+from oracle import OracleReplay
+from pasta_workloads import (Geometry, cfg1_tiny, cfg2_single_request, cfg3_batched, cfg4_long_prefix, cfg5_trace,
+                             random_script, run_tensors, step_tensors)
+
+pytestmark = pytest.mark.gpu
+
+MAX_ABS, MEAN_ABS = 1e-2, 1e-3
+
+
+@pytest.fixture(scope="module")
+def lib():
+    import torch
+    assert torch.cuda.is_available(), "GPU tests need a CUDA device"
+    from paper_2502_11517_b200 import binding, build
+    build()
+    return binding
+
+
+def compare(got, got_lse, want, want_lse, what=""):
+    got = got.double().cpu().numpy(); got_lse = got_lse.double().cpu().numpy()
+    assert np.all(np.isfinite(got)), what
+    err = np.abs(got - want)
+    assert err.max() <= MAX_ABS and err.mean() <= MEAN_ABS, (what, err.max(), err.mean())
+    assert np.abs(got_lse - want_lse).max() <= 1e-2, (what, np.abs(got_lse - want_lse).max())
+    return err.max(), err.mean()
+
+
+def run_script(lib, script, flags=0, layers=None, check_steps=None, **kw):
+    """Replays on both sides; compares bookkeeping after every op and attention at every (chosen) step."""
+    from lib_replay import LibReplay, make_pool
+    layers = list(range(script.geometry.n_layers)) if layers is None else layers
+    pool = make_pool(script, flags=flags, **kw)
+    rep = LibReplay(script, pool)
+    ora = OracleReplay(script, layers=layers)
+    worst = (0.0, 0.0)
+    for i, op in enumerate(script.ops):
+        if op[0] == "step":
+            attend = check_steps is None or i in check_steps
+            res = rep.apply(i, attend=attend)
+            want = ora.apply(i, attend=attend)
+            slots = [None if s[0] < 0 else (int(s[0]), int(s[1])) for s in rep.last_slots]
+            assert slots == [s for s in _oracle_slots(ora, op)], (i, "slots")
+            if attend:
+                out, lse = res
+                for l in layers:
+                    e = compare(out[l], lse[l], want[l][0], want[l][1], f"op {i} layer {l}")
+                    worst = (max(worst[0], e[0]), max(worst[1], e[1]))
+        else:
+            rep.apply(i); ora.apply(i)
+    assert pool.dump() == ora.model.dump()
+    assert pool.status() == 0
+    pool.close()
+    return worst
+
+
+def _oracle_slots(ora, op):
+    """Slots of the step's entries as the oracle's model placed them (last token of each appended stream)."""
+    out = []
+    for req, t, n_new in op[1]:
+        if not n_new:
+            out.append(None); continue
+        r = ora.model.requests[req]
+        k = r.stream_len[t] - 1
+        out.append((r.stream_pages[t][k // 16], k % 16))
+    return out
+
+
+# ------------------------------------------------------------------------------------------------ K1
+@pytest.mark.parametrize("geo", [Geometry(2, 4, 2, 64, 16), Geometry(2, 8, 2, 128, 16)])
+def test_append_is_a_bit_copy_into_the_right_slots(lib, geo):
+    import torch
+    from lib_replay import LibReplay, make_pool
+    script = random_script(5, n_ops=60, geo=geo)
+    pool = make_pool(script)
+    rep = LibReplay(script, pool)
+    ora = OracleReplay(script, layers=[0, 1])
+    for i in range(len(script.ops)):
+        rep.apply(i, attend=False); ora.apply(i, attend=False)
+    dump = pool.dump()
+    assert dump == ora.model.dump()
+    checked = 0
+    for req, r in dump["requests"].items():
+        for sid, s in r["streams"].items():
+            if s["len"] == 0:
+                continue
+            slots = [(s["pages"][k // 16], k % 16) for k in range(s["len"])]
+            for layer in (0, 1):
+                k, v = pool.kv_read(layer, req, sid, 0, s["len"])
+                wk, wv = ora.stores[layer].gather(slots)
+                assert np.array_equal(k.float().cpu().numpy().astype(np.float64), wk)
+                assert np.array_equal(v.float().cpu().numpy().astype(np.float64), wv)
+                checked += 1
+    assert checked > 4 and pool.status() == 0
+    pool.close()
+
+
+# ------------------------------------------------------------------------------------------------ attention
+@pytest.mark.parametrize("variant", ["base", "cutoffs", "chunk16", "chunk33", "append"])
+def test_config1_tiny(lib, variant):
+    run_script(lib, cfg1_tiny(variant))
+
+
+@pytest.mark.parametrize("variant", ["a", "b"])
+@pytest.mark.parametrize("tensor", [True, False])
+def test_config2_single_request(lib, variant, tensor):
+    run_script(lib, cfg2_single_request(variant), flags=0 if tensor else lib.FLAG_NO_TENSOR_PATH)
+
+
+@pytest.mark.parametrize("tensor", [True, False])
+def test_config3_batched_reduced(lib, tensor):
+    # 16 requests, 3 layers, two launches of <= 2 layers
+    run_script(lib, cfg3_batched(16, 3), flags=0 if tensor else lib.FLAG_NO_TENSOR_PATH, max_layers_per_launch=2)
+
+
+@pytest.mark.parametrize("tensor", [True, False])
+def test_config4_long_prefix_reduced(lib, tensor):
+    # 2 requests x 4111-token prefix (ragged: not a multiple of the tile) x 16 forks
+    run_script(lib, cfg4_long_prefix(2, 4111, 16), flags=0 if tensor else lib.FLAG_NO_TENSOR_PATH)
+
+
+def test_config4_appending_step(lib):
+    run_script(lib, cfg4_long_prefix(2, 2048, 16, n_new=1))
+
+
+def test_config5_trace_reduced(lib):
+    script = cfg5_trace(8, 96, 2, prompt_range=(32, 300), p_promise=0.08, mean_chunk=20.0)
+    steps = [i for i, op in enumerate(script.ops) if op[0] == "step"]
+    run_script(lib, script, check_steps=set(steps[::8] + steps[-2:]))
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_random_scripts(lib, seed):
+    geo = Geometry(1, 8, 2, 128, 16) if seed % 2 else Geometry(1, 4, 2, 64, 16)
+    run_script(lib, random_script(40 + seed, n_ops=70, geo=geo))
+
+
+def test_page_placement_does_not_change_the_result(lib):
+    import torch
+    from lib_replay import LibReplay, make_pool
+    outs = []
+    for order_seed in (0, 1):
+        script = cfg2_single_request("b")
+        script.free_order = np.random.default_rng(order_seed).permutation(script.n_pages).astype(np.int32)
+        pool = make_pool(script); rep = LibReplay(script, pool)
+        res = [rep.apply(i) for i in range(len(script.ops))]
+        outs.append([r[0].cpu() for r in res if r is not None])
+        pool.close()
+    for a, b in zip(*outs):
+        assert torch.equal(a, b)
+
+
+def test_step_host_entry_point(lib):
+    """The host-buffer entry point (copies inside the call) gives the same numbers as the device one."""
+    import torch
+    from lib_replay import LibReplay, make_pool
+    script = cfg2_single_request("a")
+    pool = make_pool(script); rep = LibReplay(script, pool)
+    ora = OracleReplay(script)
+    last = len(script.ops) - 1
+    for i in range(last):
+        rep.apply(i, attend=False); ora.apply(i, attend=False)
+    op = script.ops[last]
+    k, v, q = step_tensors(script, last, 0)
+    want = ora.apply(last)[0]
+    out = torch.empty(q.unsqueeze(0).shape, dtype=torch.float32).pin_memory()
+    staging = torch.empty(pool.step_host_bytes(len(op[1])), dtype=torch.uint8, device="cuda")
+    pool.step_host([e[0] for e in op[1]], [e[1] for e in op[1]], [e[2] for e in op[1]],
+                   k.unsqueeze(0).contiguous().pin_memory(), v.unsqueeze(0).contiguous().pin_memory(),
+                   q.unsqueeze(0).contiguous().pin_memory(), out, staging)
+    err = np.abs(out[0].double().numpy() - want[0])
+    assert err.max() <= MAX_ABS and err.mean() <= MEAN_ABS
+    assert pool.dump() == ora.model.dump() and pool.status() == 0
+    pool.close()

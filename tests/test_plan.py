@@ -1,0 +1,93 @@
+"""The step plan, executed on the CPU by tests/plan_interpreter.py, must reproduce the oracle."""
+import numpy as np
+import pytest
+
+from oracle import OracleReplay
+from paper_2502_11517_b200 import binding, build
+from pasta_workloads import (Geometry, cfg1_tiny, cfg2_single_request, cfg3_batched, cfg4_long_prefix, cfg5_trace,
+                             random_script, run_tensors, step_tensors)
+from lib_replay import LibReplay, make_pool
+from plan_interpreter import run_plan
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    build()
+
+
+def _f64(t):
+    import torch
+    return t.to(torch.float32).numpy().astype(np.float64)
+
+
+def check_script(script, flags=0, steps=None, **kw):
+    geo = script.geometry
+    pool = make_pool(script, host_only=True, flags=flags, **kw)
+    lib = LibReplay(script, pool)
+    ora = OracleReplay(script)
+    K = np.zeros((script.n_pages, 16, geo.n_kv_heads, geo.head_dim)); V = np.zeros_like(K)
+    n_checked = 0
+    stats = {"tunits": 0, "wunits": 0}
+    for i, op in enumerate(script.ops):
+        if op[0] == "run":
+            before = pool.dump()["requests"][op[1]]["streams"][op[2]]["len"]
+            lib.apply(i); ora.apply(i)
+            pages = pool.dump()["requests"][op[1]]["streams"][op[2]]["pages"]
+            k, v = run_tensors(script, i, 0)
+            for j in range(op[3]):
+                t = before + j
+                K[pages[t // 16], t % 16] = _f64(k[j]); V[pages[t // 16], t % 16] = _f64(v[j])
+        elif op[0] == "step":
+            lib.apply(i)
+            k, v, q = step_tensors(script, i, 0)
+            j = 0
+            for e, s in zip(op[1], lib.last_slots):
+                if e[2]:
+                    K[s[0], s[1]] = _f64(k[j]); V[s[0], s[1]] = _f64(v[j]); j += 1
+            if steps is not None and i not in steps:
+                ora.apply(i, attend=False)
+                continue
+            want, want_lse = ora.apply(i)[0]
+            w = pool.plan_words()
+            stats["tunits"] += int(w[4]); stats["wunits"] += int(w[5])
+            got, got_lse = run_plan(w, K, V, _f64(q), geo.n_kv_heads)
+            np.testing.assert_allclose(got, want, rtol=0, atol=1e-11)
+            np.testing.assert_allclose(got_lse, want_lse, rtol=0, atol=1e-11)
+            n_checked += 1
+        else:
+            lib.apply(i); ora.apply(i)
+    pool.close()
+    assert n_checked
+    return stats
+
+
+@pytest.mark.parametrize("seed", range(10))
+def test_plan_on_random_scripts_d64(seed):
+    check_script(random_script(seed, n_ops=70, geo=Geometry(1, 4, 2, 64, 16)))
+
+
+@pytest.mark.parametrize("seed", range(10, 18))
+@pytest.mark.parametrize("flags", [0, binding.FLAG_NO_TENSOR_PATH])
+def test_plan_on_random_scripts_d128(seed, flags):
+    check_script(random_script(seed, n_ops=70, geo=Geometry(1, 8, 2, 128, 16)), flags=flags)
+
+
+@pytest.mark.parametrize("maker", [cfg1_tiny, lambda: cfg1_tiny("cutoffs"), lambda: cfg1_tiny("append"),
+                                   lambda: cfg2_single_request("a"), lambda: cfg2_single_request("b"),
+                                   lambda: cfg3_batched(6, 1, prefix_range=(64, 400)),
+                                   lambda: cfg4_long_prefix(2, 1100, 5)])
+def test_plan_on_configs(maker):
+    check_script(maker())
+
+
+def test_plan_on_a_trace():
+    script = cfg5_trace(5, 60, 1, prompt_range=(16, 120), p_promise=0.1, mean_chunk=12.0)
+    steps = [i for i, op in enumerate(script.ops) if op[0] == "step"][::6]
+    check_script(script, steps=set(steps))
+
+
+def test_small_partial_budget_still_plans():
+    # few partial rows allowed: the planner must use longer pieces instead of failing
+    script = cfg3_batched(4, 1, prefix_range=(300, 600))
+    n = len(script.ops[-1][1])
+    check_script(script, max_partial_rows=n * 32 * 2 + 160 * 128)
