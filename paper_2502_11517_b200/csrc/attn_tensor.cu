@@ -1,11 +1,449 @@
-// K2 placeholder until the tensor-core kernel is in place.
+// K2: tensor-core pass over streams shared by several queries of a request (head_dim 128).
+//
+// One persistent CTA per SM walks its contiguous range of t-units.  A t-unit is a range of 64-token
+// tiles (4 pages) of one request's shared page list, for one kv head.  Rows of the score matrix are
+// the request's queries times the `group` query heads of that kv head (<= 128 rows, zero padded):
+//
+//   S[128 x 64]  = Q[128 x 128] . K_tile^T            tcgen05.mma, A and B from shared memory, D in TMEM
+//   P            = 2^(S * scale*log2e - m_ref)         one thread per row, masked by the row's visible lengths
+//   O[128 x 128] += P[128 x 64] . V_tile               tcgen05.mma, P written to shared memory as bf16
+//
+// m_ref is a per-row reference that is raised only when a tile's maximum exceeds it by more than 2^8
+// (then O and l are rescaled in TMEM); partial (m_ref, l, O) rows go to the merge kernel.
+//
+// Warp roles: warp 0 producer (bulk copies of whole (page, kv head) blocks into a 5-stage ring),
+// warp 1 MMA issue (one thread), warps 2-3 build the stacked, swizzled Q operand of each unit,
+// warps 4-7 softmax and epilogue (thread i owns row i = TMEM lane i).
+// Every wait is bounded; on expiry the CTA reports PASTA_ERR_TIMEOUT, drains and leaves.
 #include "device_common.cuh"
 #include "kernels.hpp"
 
 namespace pasta {
-cudaError_t launch_attn_tensor(const PoolView &, const PlanHeader &, int32_t, int32_t, const void *, float,
-                               cudaStream_t) {
-  return cudaErrorNotSupported;
+
+namespace {
+
+constexpr int T_THREADS = 256;
+constexpr int T_STAGES = 5;
+constexpr int T_TILE = PASTA_TILE_PAGES * PASTA_PAGE;          // 64 tokens
+constexpr int T_BLOCK = 8192;                                  // bytes of one (page, kv head) block, d = 128
+constexpr int T_STAGE_BYTES = PASTA_TILE_PAGES * T_BLOCK;      // 32 KB
+constexpr int T_Q_BYTES = 128 * 128 * 2;                       // 32 KB
+constexpr int T_P_BYTES = 128 * T_TILE * 2;                    // 16 KB
+constexpr int OFF_Q = 0;
+constexpr int OFF_P = OFF_Q + T_Q_BYTES;
+constexpr int OFF_STAGE = OFF_P + 2 * T_P_BYTES;
+constexpr int OFF_BAR = OFF_STAGE + T_STAGES * T_STAGE_BYTES;
+// barriers (8 bytes each)
+constexpr int B_FULL = 0, B_EMPTY = B_FULL + T_STAGES, B_SFULL = B_EMPTY + T_STAGES, B_PFULL = B_SFULL + 2,
+              B_PVDONE = B_PFULL + 2, B_QFULL = B_PVDONE + 2, B_QFREE = B_QFULL + 1, B_OFULL = B_QFREE + 1,
+              B_OFREE = B_OFULL + 1, B_COUNT = B_OFREE + 1;
+constexpr int OFF_META = OFF_BAR + 8 * ((B_COUNT + 1) & ~1);   // per stage: 4 page metas
+constexpr int OFF_MISC = OFF_META + T_STAGES * 16;             // tmem base, abort flag
+constexpr int T_SMEM_USED = OFF_MISC + 16;
+constexpr int T_SMEM_BYTES = T_SMEM_USED + 1024;               // slack to align the base to 1024
+static_assert(T_SMEM_BYTES <= 232448, "shared memory budget");
+
+constexpr uint32_t TMEM_COLS = 256;
+constexpr uint32_t COL_S = 0, COL_O = 128;                     // S buffers at columns 0 and 64, O at 128..255
+
+// instruction descriptors: D fp32, A/B bf16, M = 128
+constexpr uint32_t IDESC_BASE = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 4) << 24);
+constexpr uint32_t IDESC_QK = IDESC_BASE | ((64u >> 3) << 17);                 // N = 64, both operands K-major
+constexpr uint32_t IDESC_PV = IDESC_BASE | ((128u >> 3) << 17) | (1u << 16);   // N = 128, B (= V) MN-major
+
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  return static_cast<uint64_t>((addr & 0x3FFFFu) >> 4) | (static_cast<uint64_t>(lbo_bytes >> 4) << 16) |
+         (static_cast<uint64_t>(sbo_bytes >> 4) << 32) | (1ull << 46) | (2ull << 61);   // version 1, 128-byte swizzle
 }
-bool tensor_path_available() { return false; }
+
+__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a, uint64_t b, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a), "l"(b), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void mma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+#define PASTA_R32(v) \
+  v[0], v[1], v[2], v[3], v[4], v[5], v[6], v[7], v[8], v[9], v[10], v[11], v[12], v[13], v[14], v[15], v[16], v[17], \
+  v[18], v[19], v[20], v[21], v[22], v[23], v[24], v[25], v[26], v[27], v[28], v[29], v[30], v[31]
+
+// 32 consecutive fp32 columns of this thread's TMEM lane
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float *v) {
+  uint32_t r[32];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,"
+      "%29,%30,%31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const float *v) {
+  uint32_t r[32];
+#pragma unroll
+  for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(v[i]);
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%32], "
+      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,"
+      "%29,%30,%31};"
+      ::"r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]),
+        "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]), "r"(r[18]),
+        "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]),
+        "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31]), "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  uint32_t r;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+  return r;
+}
+
+// Bounded wait that also gives up when another role of the CTA has already given up.
+__device__ __forceinline__ bool wait_or_abort(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const uint64_t t0 = global_timer_ns();
+  for (;;) {
+#pragma unroll 1
+    for (int i = 0; i < 128; ++i)
+      if (mbar_try_wait(bar, parity)) return true;
+    if (*abort_flag) return false;
+    if (global_timer_ns() - t0 > 1000000000ull) { *abort_flag = 1; return false; }
+  }
+}
+
+struct UnitInfo {
+  int treq, g, tile_begin, tile_end, row_base;
+  int page_off, n_pages, n_threads, n_streams, vis_off, tq_off;
+};
+
+__device__ __forceinline__ UnitInfo load_unit(const int32_t *plan, int off_tunit, int off_treq, int u) {
+  const int32_t *U = plan + off_tunit + u * PU_WORDS;
+  UnitInfo x;
+  x.treq = U[PU_TREQ]; x.g = U[PU_KV_HEAD]; x.tile_begin = U[PU_TILE_BEGIN]; x.tile_end = U[PU_TILE_END];
+  x.row_base = U[PU_ROW_BASE];
+  const int32_t *T = plan + off_treq + x.treq * PT_WORDS;
+  x.page_off = T[PT_PAGE_OFF]; x.n_pages = T[PT_N_PAGES]; x.n_threads = T[PT_N_THREADS];
+  x.n_streams = T[PT_N_STREAMS]; x.vis_off = T[PT_VIS_OFF]; x.tq_off = T[PT_TQ_OFF];
+  return x;
+}
+
+struct TensorArgs {
+  int32_t off_tunit, off_treq, off_tcta, off_pages, off_pmeta, off_vis, off_tq;
+  int32_t n_queries, layer_begin, layer_count;
+  float scale_log2;
+};
+
+__global__ void __launch_bounds__(T_THREADS, 1)
+attn_tensor_kernel(PoolView pv, TensorArgs a, const __nv_bfloat16 *__restrict__ q) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  uint8_t *sm = smem_raw + (base - raw);
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int G = pv.n_q_heads / pv.n_kv_heads;
+  const uint32_t bar = base + OFF_BAR;
+  int32_t *meta_s = reinterpret_cast<int32_t *>(sm + OFF_META);
+  uint32_t *misc = reinterpret_cast<uint32_t *>(sm + OFF_MISC);
+  volatile int *abort_flag = reinterpret_cast<volatile int *>(misc + 1);
+  const int32_t *plan = pv.plan;
+  const int u0 = plan[a.off_tcta + 2 * blockIdx.x], u1 = plan[a.off_tcta + 2 * blockIdx.x + 1];
+
+  // ---- set-up: zero the operand buffers (stale bytes meet zero weights, so they must be finite)
+  for (int i = tid; i < OFF_BAR / 16; i += T_THREADS) reinterpret_cast<uint4 *>(sm)[i] = make_uint4(0, 0, 0, 0);
+  if (tid == 0) {
+    for (int s = 0; s < T_STAGES; ++s) { mbar_init(bar + 8 * (B_FULL + s), 1); mbar_init(bar + 8 * (B_EMPTY + s), 1); }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(bar + 8 * (B_SFULL + b), 1);
+      mbar_init(bar + 8 * (B_PFULL + b), 128);
+      mbar_init(bar + 8 * (B_PVDONE + b), 1);
+    }
+    mbar_init(bar + 8 * B_QFULL, 64);
+    mbar_init(bar + 8 * B_QFREE, 1);
+    mbar_init(bar + 8 * B_OFULL, 1);
+    mbar_init(bar + 8 * B_OFREE, 128);
+    misc[1] = 0;
+    mbar_init_fence();
+  }
+  fence_proxy_async();
+  if (warp == 2) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(base + OFF_MISC), "r"(TMEM_COLS)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = misc[0];
+
+  if (warp == 0) {
+    // ================================================================ producer
+    uint32_t it = 0;
+    bool ok = true;
+    for (int ll = 0; ll < a.layer_count && ok; ++ll) {
+      const uint8_t *kv_layer = pv.kv_base + (a.layer_begin + ll) * pv.layer_stride;
+      for (int u = u0; u < u1 && ok; ++u) {
+        const UnitInfo x = load_unit(plan, a.off_tunit, a.off_treq, u);
+        for (int tile = x.tile_begin; tile < x.tile_end; ++tile, ++it) {
+          const int s = it % T_STAGES;
+          if (!wait_or_abort(bar + 8 * (B_EMPTY + s), ((it / T_STAGES) & 1) ^ 1, abort_flag)) { ok = false; break; }
+          const int n_valid = min(PASTA_TILE_PAGES, x.n_pages - tile * PASTA_TILE_PAGES);
+          int page = 0;
+          if (lane < PASTA_TILE_PAGES) {
+            int meta = -1;
+            if (lane < n_valid) {
+              page = plan[a.off_pages + x.page_off + tile * PASTA_TILE_PAGES + lane];
+              meta = plan[a.off_pmeta + x.page_off + tile * PASTA_TILE_PAGES + lane];
+              if (page < 0 || page >= pv.n_pages) { report(pv.status, PASTA_ERR_DEVICE_CHECK); page = 0; meta = -1; }
+            }
+            meta_s[s * 4 + lane] = meta;
+          }
+          if (lane == 0) mbar_expect_tx(bar + 8 * (B_FULL + s), n_valid * T_BLOCK);
+          __syncwarp();
+          if (lane < n_valid)
+            bulk_g2s(base + OFF_STAGE + s * T_STAGE_BYTES + lane * T_BLOCK,
+                     kv_layer + (static_cast<int64_t>(page) * pv.n_kv_heads + x.g) * T_BLOCK, T_BLOCK,
+                     bar + 8 * (B_FULL + s));
+        }
+      }
+    }
+    if (!ok && lane == 0) {
+      // copies still in flight must land before the CTA leaves: bounded waits on the last stages issued
+      for (uint32_t j = (it > T_STAGES ? it - T_STAGES : 0); j < it; ++j)
+        mbar_wait_bounded(bar + 8 * (B_FULL + j % T_STAGES), (j / T_STAGES) & 1);
+    }
+  } else if (warp == 1) {
+    // ================================================================ MMA issue (one thread)
+    if (lane == 0) {
+      uint32_t it = 0, uc = 0;
+      bool ok = true;
+      const uint32_t q_addr = base + OFF_Q;
+      for (int ll = 0; ll < a.layer_count && ok; ++ll) {
+        for (int u = u0; u < u1 && ok; ++u, ++uc) {
+          const UnitInfo x = load_unit(plan, a.off_tunit, a.off_treq, u);
+          const int nt = x.tile_end - x.tile_begin;
+          if (!wait_or_abort(bar + 8 * B_QFULL, uc & 1, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          for (int k = 0; k <= nt && ok; ++k) {
+            if (k < nt) {
+              // ---- S[b] = Q . K^T for tile `it`
+              const uint32_t s = it % T_STAGES, b = it & 1;
+              if (!wait_or_abort(bar + 8 * (B_FULL + s), (it / T_STAGES) & 1, abort_flag)) { ok = false; break; }
+              tc_fence_after();
+              const uint32_t k_addr = base + OFF_STAGE + s * T_STAGE_BYTES;
+#pragma unroll
+              for (int ks = 0; ks < 8; ++ks) {
+                const uint32_t half = ks >> 2, kk = ks & 3;
+                mma_ss(tmem + COL_S + b * 64, smem_desc(q_addr + half * 16384 + kk * 32, 16, 1024),
+                       smem_desc(k_addr + half * 1024 + kk * 32, 16, 4096), IDESC_QK, ks > 0);
+              }
+              mma_commit(bar + 8 * (B_SFULL + b));
+              if (k == nt - 1) mma_commit(bar + 8 * B_QFREE);   // the Q operand may be replaced once these finish
+            }
+            if (k > 0) {
+              // ---- O += P . V for tile `it - 1` (it has not been advanced for this k yet when k == nt)
+              const uint32_t j = (k < nt) ? it - 1 : it - 1;
+              const uint32_t s = j % T_STAGES, b = j & 1;
+              if (k == 1 && uc > 0) {   // first P.V of the unit overwrites O: the previous unit's rows must be read out
+                if (!wait_or_abort(bar + 8 * B_OFREE, (uc - 1) & 1, abort_flag)) { ok = false; break; }
+              }
+              if (!wait_or_abort(bar + 8 * (B_PFULL + b), (j >> 1) & 1, abort_flag)) { ok = false; break; }
+              tc_fence_after();
+              const uint32_t p_addr = base + OFF_P + b * T_P_BYTES;
+              const uint32_t v_addr = base + OFF_STAGE + s * T_STAGE_BYTES + 2048;
+#pragma unroll
+              for (int pg = 0; pg < PASTA_TILE_PAGES; ++pg)
+                mma_ss(tmem + COL_O, smem_desc(p_addr + pg * 32, 16, 1024),
+                       smem_desc(v_addr + pg * T_BLOCK, 1024, 4096), IDESC_PV, (k > 1) || (pg > 0));
+              mma_commit(bar + 8 * (B_EMPTY + s));
+              mma_commit(bar + 8 * (B_PVDONE + b));
+              if (k == nt) mma_commit(bar + 8 * B_OFULL);
+            }
+            if (k < nt) ++it;
+          }
+        }
+      }
+    }
+  } else if (warp < 4) {
+    // ================================================================ stacked Q operand (64 threads)
+    const int t64 = tid - 64;
+    uint32_t uc = 0;
+    bool ok = true;
+    for (int ll = 0; ll < a.layer_count && ok; ++ll) {
+      for (int u = u0; u < u1; ++u, ++uc) {
+        const UnitInfo x = load_unit(plan, a.off_tunit, a.off_treq, u);
+        if (uc > 0 && !wait_or_abort(bar + 8 * B_QFREE, (uc - 1) & 1, abort_flag)) { ok = false; break; }
+        const int rows = x.n_threads * G;
+        for (int idx = t64; idx < 128 * 16; idx += 64) {
+          const int row = idx >> 4, c = idx & 15;
+          uint4 val = make_uint4(0, 0, 0, 0);
+          if (row < rows) {
+            const int t = row / G, hl = row - t * G;
+            const int qn = plan[a.off_tq + x.tq_off + t];
+            val = __ldg(reinterpret_cast<const uint4 *>(
+                q + ((static_cast<int64_t>(ll) * a.n_queries + qn) * pv.n_q_heads + x.g * G + hl) * 128 + c * 8));
+          }
+          const int r8 = row & 7;
+          *reinterpret_cast<uint4 *>(sm + OFF_Q + (c >> 3) * 16384 + (row >> 3) * 1024 + r8 * 128 + (((c & 7) ^ r8) << 4)) = val;
+        }
+        fence_proxy_async();
+        mbar_arrive(bar + 8 * B_QFULL);
+      }
+    }
+  } else {
+    // ================================================================ softmax + epilogue (128 threads)
+    const int row = tid - 128;                      // = TMEM lane
+    const uint32_t lane_addr = static_cast<uint32_t>((warp & 3) * 32) << 16;
+    uint32_t it = 0, uc = 0;
+    bool ok = true;
+    for (int ll = 0; ll < a.layer_count && ok; ++ll) {
+      for (int u = u0; u < u1 && ok; ++u, ++uc) {
+        const UnitInfo x = load_unit(plan, a.off_tunit, a.off_treq, u);
+        const int nt = x.tile_end - x.tile_begin;
+        const int rows = x.n_threads * G;
+        const bool active = row < rows;
+        const bool warp_active = (warp - 4) * 32 < rows;
+        const int32_t *visrow = plan + a.off_vis + x.vis_off + (active ? row / G : 0) * x.n_streams;
+        float m_ref = -INFINITY, l = 0.f;
+        for (int k = 0; k < nt; ++k, ++it) {
+          const uint32_t s = it % T_STAGES, b = it & 1;
+          if (!wait_or_abort(bar + 8 * (B_SFULL + b), (it >> 1) & 1, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          if (warp_active) {
+            float sc[T_TILE];
+            tmem_ld32(tmem + lane_addr + COL_S + b * 64, sc);
+            tmem_ld32(tmem + lane_addr + COL_S + b * 64 + 32, sc + 32);
+            int thr[PASTA_TILE_PAGES];
+            bool full = true;
+#pragma unroll
+            for (int pg = 0; pg < PASTA_TILE_PAGES; ++pg) {
+              const int meta = meta_s[s * 4 + pg];
+              int t = 0;
+              if (active && meta >= 0) t = min(max(visrow[meta & 255] - (meta >> 8) * PASTA_PAGE, 0), PASTA_PAGE);
+              thr[pg] = t;
+              full = full && (t == PASTA_PAGE);
+            }
+            if (!full) {
+#pragma unroll
+              for (int j = 0; j < T_TILE; ++j)
+                if ((j & 15) >= thr[j >> 4]) sc[j] = -INFINITY;
+            }
+            float mt = sc[0];
+#pragma unroll
+            for (int j = 1; j < T_TILE; ++j) mt = fmaxf(mt, sc[j]);
+            mt *= a.scale_log2;
+            const bool need = mt > m_ref + 8.f;       // also true for the first visible tile (m_ref = -inf)
+            const bool rescale = need && l > 0.f;
+            if (__any_sync(0xffffffffu, rescale)) {
+              // O and l are relative to m_ref: move them to the new reference.  P.V of the previous tile must be done.
+              if (!wait_or_abort(bar + 8 * (B_PVDONE + (b ^ 1)), ((it - 1) >> 1) & 1, abort_flag)) { ok = false; break; }
+              tc_fence_after();
+              const float f = rescale ? fast_exp2(m_ref - mt) : 1.f;
+#pragma unroll 1
+              for (int cb = 0; cb < 4; ++cb) {
+                float ov[32];
+                tmem_ld32(tmem + lane_addr + COL_O + cb * 32, ov);
+#pragma unroll
+                for (int j = 0; j < 32; ++j) ov[j] *= f;
+                tmem_st32(tmem + lane_addr + COL_O + cb * 32, ov);
+              }
+              tmem_st_wait();
+              l *= f;
+            }
+            if (need) m_ref = mt;
+            const float ref = (m_ref == -INFINITY) ? 0.f : m_ref;
+            float lsum = 0.f;
+            uint32_t pk[T_TILE / 2];
+#pragma unroll
+            for (int j = 0; j < T_TILE; j += 2) {
+              const float p0 = fast_exp2(fmaf(sc[j], a.scale_log2, -ref));
+              const float p1 = fast_exp2(fmaf(sc[j + 1], a.scale_log2, -ref));
+              lsum += p0 + p1;
+              pk[j >> 1] = pack_bf16(p0, p1);
+            }
+            l += lsum;
+            // P[b] may be overwritten once P.V of tile it-2 has finished
+            if (it >= 2 && !wait_or_abort(bar + 8 * (B_PVDONE + b), ((it - 2) >> 1) & 1, abort_flag)) { ok = false; break; }
+            uint8_t *prow = sm + OFF_P + b * T_P_BYTES + (row >> 3) * 1024 + (row & 7) * 128;
+#pragma unroll
+            for (int c = 0; c < 8; ++c)
+              *reinterpret_cast<uint4 *>(prow + ((c ^ (row & 7)) << 4)) =
+                  make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
+            fence_proxy_async();
+          }
+          tc_fence_before();
+          mbar_arrive(bar + 8 * (B_PFULL + b));
+        }
+        if (!ok) break;
+        // ---- epilogue: this unit's rows leave TMEM
+        if (!wait_or_abort(bar + 8 * B_OFULL, uc & 1, abort_flag)) { ok = false; break; }
+        tc_fence_after();
+        if (warp_active) {
+          const int64_t prow = static_cast<int64_t>(ll) * pv.rows_per_layer + x.row_base + row;
+          if (active) pv.part_ml[prow] = make_float2(m_ref, l);
+#pragma unroll 1
+          for (int cb = 0; cb < 4; ++cb) {
+            float ov[32];
+            tmem_ld32(tmem + lane_addr + COL_O + cb * 32, ov);
+            if (active && l > 0.f) {
+              float4 *dst = reinterpret_cast<float4 *>(pv.part_o + prow * 128 + cb * 32);
+#pragma unroll
+              for (int j = 0; j < 8; ++j) dst[j] = make_float4(ov[4 * j], ov[4 * j + 1], ov[4 * j + 2], ov[4 * j + 3]);
+            }
+          }
+        }
+        tc_fence_before();
+        mbar_arrive(bar + 8 * B_OFREE);
+      }
+    }
+  }
+
+  // ---- tear-down
+  if (*abort_flag && tid == 0) report(pv.status, PASTA_ERR_TIMEOUT);
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 2) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(TMEM_COLS) : "memory");
+  }
+}
+
+}  // namespace
+
+bool tensor_path_available() { return true; }
+
+cudaError_t launch_attn_tensor(const PoolView &pv, const PlanHeader &h, int32_t layer_begin, int32_t layer_count,
+                               const void *q, float scale_log2, cudaStream_t st) {
+  if (pv.head_dim != 128) return cudaErrorInvalidValue;
+  static bool prepared = false;
+  if (!prepared) {
+    cudaError_t e = cudaFuncSetAttribute(attn_tensor_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, T_SMEM_BYTES);
+    if (e != cudaSuccess) return e;
+    prepared = true;
+  }
+  const int grid = h.w[PH_T_GRID];
+  if (grid == 0 || layer_count == 0) return cudaSuccess;
+  TensorArgs a;
+  a.off_tunit = h.w[PH_OFF_TUNIT]; a.off_treq = h.w[PH_OFF_TREQ]; a.off_tcta = h.w[PH_OFF_TCTA];
+  a.off_pages = h.w[PH_OFF_PAGES]; a.off_pmeta = h.w[PH_OFF_PMETA]; a.off_vis = h.w[PH_OFF_VIS];
+  a.off_tq = h.w[PH_OFF_TQ];
+  a.n_queries = h.w[PH_N_QUERIES]; a.layer_begin = layer_begin; a.layer_count = layer_count;
+  a.scale_log2 = scale_log2;
+  attn_tensor_kernel<<<grid, T_THREADS, T_SMEM_BYTES, st>>>(pv, a, static_cast<const __nv_bfloat16 *>(q));
+  return cudaGetLastError();
+}
+
 }  // namespace pasta
