@@ -1,0 +1,435 @@
+#!/usr/bin/env python
+"""Benchmark of the decode-attention hot path: step plan + KV append + attention, per decode step.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+
+Prints ONE JSON line.  A step is one decode step of the whole batch: every active thread appends
+one token (pasta_step_begin + pasta_kv_append) and attends (pasta_decode_attn: tensor-core pass over
+shared streams, warp-shuffle pass over private ones, merge).  Metric: thread-tokens per second
+(one thread-token = one (request, thread) query through attention in every layer of the workload).
+
+Workloads (synthetic, seeded; shapes of the five configurations):
+  long_shared_prefix  8 requests x 32768-token prefix x 16 forks (chunks U[50,400]), 1 layer      [default]
+  batched             64 requests, prefix U[256,2048], forks geometric, chunks U[10,300], 32 layers
+  single_request      1 request, 768-token prefix, 4 forks, 1 layer (cache resident: a latency case)
+With N > 1 (torchrun) every rank runs its own copy of the workload on its own GPU: requests are
+independent, there is no exchange between ranks ("weak" scaling).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "decode-attn thread-tokens/s"
+UNIT = "thread-tokens/s"
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+# dram bytes (read + write) of one launch of the dominant kernel from an ncu capture of this workload,
+# or None when no capture matches the current kernel
+NCU_TRAFFIC_BYTES = {"long_shared_prefix": None, "batched": None, "single_request": None}
+
+
+def make_script(workload: str):
+    from pasta_workloads import cfg2_single_request, cfg3_batched, cfg4_long_prefix
+    if workload == "long_shared_prefix":
+        return cfg4_long_prefix()
+    if workload == "batched":
+        return cfg3_batched()
+    if workload == "single_request":
+        return cfg2_single_request("a")
+    raise SystemExit(f"unknown workload {workload}")
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        try:
+            return float(json.load(open(path))["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return FALLBACK_HBM_GBS, "fallback"
+
+
+# ------------------------------------------------------------------------------------------------ clocks
+class ClockSampler:
+    QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, device_index: int):
+        self.file = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(device_index), f"--query-gpu=timestamp,{self.QUERY}",
+                 "--format=csv,noheader,nounits", "-lms", "20"], stdout=self.file, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self, t0: float, t1: float):
+        """Samples whose wall-clock time lies in [t0, t1] (the timed region); falls back to all samples."""
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        time.sleep(0.05)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.file.flush()
+        rows = []
+        import datetime
+        for line in open(self.file.name):
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 9:
+                continue
+            try:
+                ts = datetime.datetime.strptime(parts[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+                rows.append((ts, float(parts[1]), float(parts[2]), parts[4:9]))
+            except Exception:
+                continue
+        os.unlink(self.file.name)
+        inside = [r for r in rows if t0 <= r[0] <= t1]
+        out["window"] = "timed region" if inside else "whole run (timed region shorter than the sampling period)"
+        use = inside or rows
+        if not use:
+            return out
+        out["samples"] = len(use)
+        out["sm_mhz"] = float(np.median([r[1] for r in use]))
+        out["sm_max_mhz"] = float(max(r[2] for r in use))
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        seen = set()
+        for r in use:
+            for name, flag in zip(names, r[3][1:]):
+                if flag.lower().startswith("active"):
+                    seen.add(name)
+        out["reasons"] = sorted(seen)
+        return out
+
+
+# ------------------------------------------------------------------------------------------------ our arm
+def build_state(script, device, seed_offset=0, grow_tokens=640):
+    """Replays the set-up part of the script (everything before its final step) with device-generated
+    bf16 N(0,1) tensors.  Returns the pool and the final step's entries."""
+    import torch
+    from paper_2502_11517_b200 import binding
+    geo = script.geometry
+    # room for the tokens the benchmark appends: every entry may grow by up to `grow` tokens
+    entries = list(script.ops[-1][1])
+    grow_pages = len(entries) * (grow_tokens // 16 + 2)
+    order = np.concatenate([script.free_order, np.arange(script.n_pages, script.n_pages + grow_pages, dtype=np.int32)])
+    pool = binding.Pool(geo.n_layers, geo.n_q_heads, geo.n_kv_heads, geo.head_dim, script.n_pages + grow_pages,
+                        script.max_requests, script.max_threads_per_request, script.max_segments_per_thread,
+                        free_order=order, max_step_queries=len(entries), max_layers_per_launch=geo.n_layers,
+                        device=device.index or 0)
+    gen = torch.Generator(device=device)
+    gen.manual_seed(script.seed + 977 * seed_offset)
+
+    def randn(shape):
+        return torch.randn(shape, generator=gen, device=device, dtype=torch.float32).to(torch.bfloat16)
+
+    for op in script.ops[:-1]:
+        kind = op[0]
+        if kind == "begin":
+            assert pool.request_begin() == op[1]
+        elif kind == "spawn":
+            assert pool.thread_spawn(op[1]) == op[2]
+        elif kind == "finish":
+            pool.thread_finish(op[1], op[2])
+        elif kind == "merge":
+            pool.sync_merge(op[1], None if op[2] is None else list(op[2]))
+        elif kind == "run":
+            m = op[3]
+            done = 0
+            while done < m:                      # bounded transient memory for many-layer pools
+                cnt = min(m - done, 4096)
+                shape = (geo.n_layers, cnt, geo.n_kv_heads, geo.head_dim)
+                pool.kv_append_run(op[1], op[2], cnt, randn(shape), randn(shape))
+                done += cnt
+        else:
+            raise ValueError(kind)
+    torch.cuda.synchronize(device)
+    return pool, entries, randn
+
+
+def unique_tokens(pool, entries):
+    """Per request, the union of what the step's threads see (a shared prefix counts once); and the part of
+    it that is seen by two or more threads (what the tensor-core kernel reads)."""
+    dump = pool.dump()
+    by_req = {}
+    for req, t, _ in entries:
+        by_req.setdefault(req, []).append(t)
+    total = shared = 0
+    for req, threads in by_req.items():
+        seen = {}
+        for t in threads:
+            vis = {}
+            for s, a, n in dump["requests"][req]["threads"][t]["view"]:
+                vis[s] = max(vis.get(s, 0), a + n)
+            for s, v in vis.items():
+                seen.setdefault(s, []).append(v)
+        for s, vs in seen.items():
+            total += max(vs)
+            if len(vs) >= 2:
+                shared += max(vs)
+    return total, shared
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2502_11517_b200.build import build
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    if rank == 0:
+        build()
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+        dist.barrier()
+    device = torch.device("cuda", local)
+    torch.cuda.set_device(device)
+    script = make_script(args.workload)
+    geo = script.geometry
+    e2e_steps = max(3, min(args.steps, 50))
+    pool, entries, randn = build_state(script, device, seed_offset=rank,
+                                       grow_tokens=args.steps + max(args.warmup, 3) + e2e_steps + 3)
+    n = len(entries)
+    reqs = [e[0] for e in entries]; thr = [e[1] for e in entries]
+    ones = [1] * n
+    L = geo.n_layers
+    k_new = randn((L, n, geo.n_kv_heads, geo.head_dim)); v_new = randn((L, n, geo.n_kv_heads, geo.head_dim))
+    q = randn((L, n, geo.n_q_heads, geo.head_dim))
+    out = torch.empty(q.shape, dtype=torch.float32, device=device)
+    stream = torch.cuda.current_stream(device)
+
+    def step():
+        pool.step_begin(reqs, thr, ones)
+        pool.kv_append(k_new, v_new)
+        pool.decode_attn(q, out)
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize(device)
+    tok0, shared0 = unique_tokens(pool, entries)
+    launches0 = pool.launch_count()
+    pool.profile_enable(True)
+    sampler = ClockSampler(local) if rank == 0 else None
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize(device)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t_wall0 = time.time()
+    ev0.record(stream)
+    for _ in range(args.steps):
+        step()
+    ev1.record(stream)
+    torch.cuda.synchronize(device)
+    t_wall1 = time.time()
+    if world > 1:
+        dist.barrier()
+    ms = ev0.elapsed_time(ev1)
+    clocks = sampler.stop(t_wall0, t_wall1) if sampler else None
+    kernel_ms, kernel_launches = pool.profile_read()
+    pool.profile_enable(False)
+    launches = pool.launch_count() - launches0
+    tok1, shared1 = unique_tokens(pool, entries)
+    assert pool.status() == 0, "a kernel reported an error"
+    if world > 1:
+        t = torch.tensor([ms], device=device, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+
+    # ---- end to end: the same step through the host-buffer entry point (copies inside the timed region)
+    k_h = k_new.cpu().pin_memory(); v_h = v_new.cpu().pin_memory(); q_h = q.cpu().pin_memory()
+    out_h = torch.empty(q.shape, dtype=torch.float32).pin_memory()
+    staging = torch.empty(pool.step_host_bytes(n), dtype=torch.uint8, device=device)
+    for _ in range(3):
+        pool.step_host(reqs, thr, ones, k_h, v_h, q_h, out_h, staging)
+    torch.cuda.synchronize(device)
+    if world > 1:
+        dist.barrier()
+    t0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        pool.step_host(reqs, thr, ones, k_h, v_h, q_h, out_h, staging)
+    torch.cuda.synchronize(device)
+    e2e_s = time.perf_counter() - t0
+    if world > 1:
+        t = torch.tensor([e2e_s], device=device, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_s = float(t.item())
+    h2d = k_h.numel() * 2 * 2 + q_h.numel() * 2
+    d2h = out_h.numel() * 4
+
+    # ---- host-only cost of a <sync/> merge (no kernel, no copy): a scratch pool with 16 finished forks
+    merge_us = time_sync_merge()
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+    B_tok = geo.kv_bytes_per_token
+    # unique KV bytes of the average step (every step adds one token per entry); all layers
+    avg_tokens = (tok0 + tok1) / 2.0 + n / 2.0
+    step_bytes = avg_tokens * B_tok * L
+    shared_bytes = (shared0 + shared1) / 2.0 * B_tok * L      # what one tensor-core launch... per step
+    peak, peak_kind = measured_peak()
+    timed_steps = max(1, max(kernel_launches))                 # one launch of each kernel per step
+    dom = 0 if kernel_launches[0] else 1                       # tensor-core kernel when the workload has shared streams
+    dom_name = ["attn_tensor_kernel", "attn_warp_kernel"][dom]
+    dom_bytes_per_launch = shared_bytes if dom == 0 else step_bytes - shared_bytes
+    dom_ms = kernel_ms[dom] / max(1, kernel_launches[dom])
+    achieved = dom_bytes_per_launch / (dom_ms * 1e-3) / 1e9 if dom_ms > 0 else 0.0
+    value = world * n * args.steps / (ms * 1e-3)
+    step_gbs = step_bytes / (ms / args.steps * 1e-3) / 1e9
+    result = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {
+            "workload": args.workload, "script": script.name, "requests": len(set(reqs)), "thread_tokens_per_step": n,
+            "layers": L, "n_q_heads": geo.n_q_heads, "n_kv_heads": geo.n_kv_heads, "head_dim": geo.head_dim,
+            "page_size": geo.page_size, "unique_kv_tokens_per_layer": avg_tokens,
+            "unique_kv_bytes_per_step": step_bytes, "l2": "inputs larger than L2" if step_bytes / L > 126e6 * 1.5 else
+            "working set fits L2 (latency case)",
+            "step_hbm_gbs": step_gbs, "step_frac_of_measured_peak": step_gbs / peak,
+            "step_frac_of_nominal_8TBs": step_gbs / NOMINAL_HBM_GBS,
+            "kernel_ms_per_step": {"tensor": kernel_ms[0] / timed_steps, "warp": kernel_ms[1] / timed_steps,
+                                   "merge": kernel_ms[2] / timed_steps, "steps_timed": timed_steps},
+            "sync_merge_host_us": merge_us,
+        },
+        "clocks": clocks,
+        "e2e": {"value": world * n * e2e_steps / e2e_s, "unit": UNIT, "h2d_bytes_per_step": h2d,
+                "d2h_bytes_per_step": d2h, "steps": e2e_steps},
+        "gpu_launches": launches,
+        "roofline": {"bound": "hbm", "kernel": dom_name, "achieved": achieved, "peak": peak, "peak_kind": peak_kind,
+                     "unit": "GB/s", "frac": achieved / peak, "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
+                     "traffic": NCU_TRAFFIC_BYTES.get(args.workload), "bytes_per_launch": dom_bytes_per_launch,
+                     "ms_per_launch": dom_ms},
+        "cpu_baseline": oracle_sample(args.workload, budget_s=20.0) if world == 1 and not args.no_cpu_baseline else None,
+    }
+    print(json.dumps(result))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def time_sync_merge():
+    from paper_2502_11517_b200 import binding
+    best = None
+    for _ in range(5):
+        pool = binding.Pool(1, 32, 8, 128, 4096, 1, 32, 64, flags=binding.FLAG_HOST_ONLY)
+        r = pool.request_begin()
+        pool.kv_append_run(r, 0, 768)
+        forks = [pool.thread_spawn(r) for _ in range(16)]
+        for t in forks:
+            pool.kv_append_run(r, t, 100); pool.thread_finish(r, t)
+        t0 = time.perf_counter()
+        pool.sync_merge(r)
+        dt = (time.perf_counter() - t0) * 1e6
+        best = dt if best is None else min(best, dt)
+        pool.close()
+    return best
+
+
+# ------------------------------------------------------------------------------------------------ oracle arm
+def oracle_sample(workload: str, budget_s: float = 20.0, steps: int = 1):
+    """Times the fp64 CPU oracle, as it stands, on a bounded sample of the workload: the queries of the
+    workload's first request(s), in layer 0.  Returns the cpu_baseline object."""
+    from oracle import OracleReplay
+    from pasta_workloads import cfg2_single_request, cfg3_batched, cfg4_long_prefix
+    if workload == "long_shared_prefix":
+        script = cfg4_long_prefix(n_requests=1); sample = "the 17 thread-tokens of 1 of 8 requests (32768-token prefix, 16 forks), 1 layer"
+    elif workload == "batched":
+        script = cfg3_batched(n_requests=8, n_layers=1); sample = "the thread-tokens of the first 8 of 64 requests, 1 of 32 layers (time scaled by 32 layers)"
+    else:
+        script = cfg2_single_request("a"); script.ops = script.ops[:11]; sample = "step A: 5 thread-tokens of the request, 1 layer"
+    rep = OracleReplay(script)
+    last = len(script.ops) - 1
+    for i in range(last):
+        rep.apply(i, attend=False)
+    # the step's bookkeeping and append happen once; the attention is what is timed
+    from oracle import decode_attention
+    from pasta_workloads import step_tensors
+    op = script.ops[last]
+    k, v, q = step_tensors(script, last, 0)
+    slots = [s for s in rep.model.reserve(op[1]) if s is not None]
+    rep.stores[0].write(slots, k, v)
+    queries = [(e[0], e[1]) for e in op[1]]
+    times = []
+    t_all = time.perf_counter()
+    for _ in range(steps):
+        t0 = time.perf_counter()
+        done = 0
+        for i, qq in enumerate(queries):
+            decode_attention(rep.model, rep.stores[0], [qq], q[i:i + 1])
+            done += 1
+            if time.perf_counter() - t_all > budget_s and steps == 1:
+                break
+        times.append((time.perf_counter() - t0, done))
+    dt = sum(t for t, _ in times); done = sum(d for _, d in times)
+    layers = 32 if workload == "batched" else 1
+    try:
+        from threadpoolctl import threadpool_info
+        cores = max([p.get("num_threads", 1) for p in threadpool_info()] or [1])
+    except Exception:
+        cores = 1
+    return {"value": done / (dt * layers), "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"{done} thread-tokens: {sample}", "seconds": dt}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    t0 = time.perf_counter()
+    per_step = max(2.0, min(20.0, 120.0 / max(1, args.steps + args.warmup)))
+    for _ in range(args.warmup):
+        oracle_sample(args.workload, budget_s=per_step)
+    res = [oracle_sample(args.workload, budget_s=per_step) for _ in range(args.steps)]
+    secs = sum(r["seconds"] for r in res)
+    done = sum(float(r["sample"].split()[0]) for r in res)
+    layers = 32 if args.workload == "batched" else 1
+    value = done / (secs * layers)
+    base = dict(res[-1]); base["value"] = value
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": int(os.environ.get("WORLD_SIZE", "1")),
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": secs / max(1, args.steps) * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": args.workload}, "cpu_baseline": base,
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "wall_s": time.perf_counter() - t0,
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--workload", default="long_shared_prefix")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        if args.steps == 200:
+            args.steps, args.warmup = 3, 1
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

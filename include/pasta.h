@@ -82,7 +82,8 @@ pasta_status_t pasta_workspace_bytes(const pasta_pool_config_t *cfg, size_t *out
  * The single pre-allocated KV pool of Section 3 "Efficiency" (here paged: 16 tokens per page, one
  * page list per stream, where a stream is the main thread's tokens or one fork's chunk).  The
  * layout inside a page is private to the library; results do not depend on which pages a stream
- * receives.  The KV memory itself is not touched by create/destroy.
+ * receives.  Create zero-fills the KV memory once (bytes of a page beyond a stream's end are read
+ * and multiplied by zero weights, so they have to be finite); destroy does not touch it.
  */
 pasta_status_t pasta_pool_create(const pasta_pool_config_t *cfg, pasta_pool_t **out);
 pasta_status_t pasta_pool_destroy(pasta_pool_t *pool);
@@ -118,6 +119,8 @@ pasta_status_t pasta_sync_merge(pasta_pool_t *pool, int32_t req, int32_t n_threa
  * thread at most once, ACTIVE threads only) and appends n_new[i] tokens (0 or 1; NULL = all 1).
  * Pages are taken in list order, one whenever a stream's token index is a multiple of 16.
  * An entry that would see nothing (no visible token and n_new == 0) is INVALID_ARG.
+ * If the bookkeeping succeeds but the step cannot be planned within the pool's capacities, the call
+ * returns CAPACITY with the tokens already reserved (the one exception to "unchanged on failure").
  * The plan is uploaded on `stream`; it is used by the pasta_kv_append and pasta_decode_attn calls
  * that follow, for every layer, until the next pasta_step_begin.
  */
@@ -206,6 +209,16 @@ pasta_status_t pasta_pool_status(pasta_pool_t *pool, void *stream);
 
 /* Number of kernels this pool has launched so far (for launch accounting). */
 pasta_status_t pasta_launch_count(pasta_pool_t *pool, int64_t *out);
+
+/*
+ * Kernel timing for benchmarks.  While enabled, pasta_decode_attn brackets each of its kernels with
+ * CUDA events on the launching stream (at most 512 launches are kept between two reads).
+ * pasta_profile_read waits for the recorded events and returns, accumulated since the previous read:
+ * out_ms[0..2] = device milliseconds of the tensor-core pass, the warp-shuffle pass and the merge,
+ * out_launches[0..2] = how many launches of each were timed.  Both arrays are host memory.
+ */
+pasta_status_t pasta_profile_enable(pasta_pool_t *pool, int32_t on);
+pasta_status_t pasta_profile_read(pasta_pool_t *pool, double *out_ms, int64_t *out_launches);
 
 /* cudaError_t of the last failed CUDA call made by the library in this process (0 if none). */
 int32_t pasta_last_cuda_error(void);

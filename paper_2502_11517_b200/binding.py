@@ -24,6 +24,7 @@ EXPORTS = [
     "pasta_sync_merge", "pasta_step_begin", "pasta_step_slots", "pasta_kv_append", "pasta_decode_attn",
     "pasta_kv_append_run", "pasta_step_host_bytes", "pasta_step_host", "pasta_kv_read",
     "pasta_pool_dump", "pasta_plan_dump", "pasta_pool_status", "pasta_launch_count",
+    "pasta_profile_enable", "pasta_profile_read",
     "pasta_last_cuda_error",
 ]
 
@@ -261,6 +262,16 @@ class Pool:
     def status(self, stream=None) -> int:
         st = C.c_void_p(0) if self.host_only else _stream(stream)
         return lib().pasta_pool_status(self._h, st)
+
+    def profile_enable(self, on: bool = True) -> None:
+        _check(lib().pasta_profile_enable(self._h, int(on)), "pasta_profile_enable")
+
+    def profile_read(self):
+        """(ms, launches): device time and number of timed launches of the tensor, warp and merge kernels."""
+        ms = (C.c_double * 3)()
+        cnt = (C.c_int64 * 3)()
+        _check(lib().pasta_profile_read(self._h, ms, cnt), "pasta_profile_read")
+        return list(ms), list(cnt)
 
     def launch_count(self) -> int:
         out = C.c_int64()

@@ -15,6 +15,7 @@ using namespace pasta;
 namespace {
 
 constexpr int kStaging = 4;           // pinned upload buffers in rotation
+constexpr int kProfCalls = 512;        // timed pasta_decode_attn launches kept between two profile reads
 constexpr int kRunChunk = 8192;       // tokens whose slots are uploaded at once by pasta_kv_append_run
 int32_t g_last_cuda_error = 0;
 
@@ -81,6 +82,11 @@ struct pasta_pool {
   PlanHeader hdr{};
   bool plan_valid = false;
   int64_t launches = 0;
+  // kernel timing (pasta_profile_*): events[4 * i .. 4 * i + 3] bracket the three kernels of call i
+  bool profiling = false;
+  std::vector<cudaEvent_t> prof_events;
+  std::vector<uint8_t> prof_mask;       // per call: bit k set if kernel k was launched
+  int prof_calls = 0;
 
   pasta_pool(const pasta_pool_config_t &c, const Derived &dd)
       : cfg(c), d(dd),
@@ -206,6 +212,7 @@ pasta_status_t pasta_pool_destroy(pasta_pool_t *p) {
     if (p->pinned[i]) cudaFreeHost(p->pinned[i]);
   }
   if (p->status_host) cudaFreeHost(p->status_host);
+  for (cudaEvent_t e : p->prof_events) if (e) cudaEventDestroy(e);
   delete p;
   return PASTA_OK;
 }
@@ -300,16 +307,29 @@ pasta_status_t pasta_decode_attn(pasta_pool_t *p, int32_t layer_begin, int32_t l
     const uint16_t *qg = static_cast<const uint16_t *>(q) + size_t(done) * q_layer;
     float *og = static_cast<float *>(out) + size_t(done) * q_layer;
     float *lg = lse ? lse + size_t(done) * n * p->cfg.n_q_heads : nullptr;
+    const bool timed = p->profiling && p->prof_calls < kProfCalls;
+    cudaEvent_t *ev = timed ? &p->prof_events[4 * p->prof_calls] : nullptr;
+    uint8_t mask = 0;
+    if (timed) PASTA_CUDA(cudaEventRecord(ev[0], st));
     if (p->hdr.w[PH_N_TUNITS] > 0) {
       PASTA_CUDA(launch_attn_tensor(p->pv, p->hdr, layer_begin + done, cnt, qg, sc, st));
       p->launches += 1;
+      mask |= 1;
     }
+    if (timed) PASTA_CUDA(cudaEventRecord(ev[1], st));
     if (p->hdr.w[PH_N_WUNITS] > 0) {
       PASTA_CUDA(launch_attn_warp(p->pv, p->hdr, layer_begin + done, cnt, qg, sc, st));
       p->launches += 1;
+      mask |= 2;
     }
+    if (timed) PASTA_CUDA(cudaEventRecord(ev[2], st));
     PASTA_CUDA(launch_merge(p->pv, p->hdr, cnt, og, lg, st));
     p->launches += 1;
+    mask |= 4;
+    if (timed) {
+      PASTA_CUDA(cudaEventRecord(ev[3], st));
+      p->prof_mask[p->prof_calls++] = mask;
+    }
   }
   return PASTA_OK;
 }
@@ -448,6 +468,37 @@ pasta_status_t pasta_pool_status(pasta_pool_t *p, void *stream) {
   PASTA_CUDA(cudaMemsetAsync(p->pv.status, 0, 4, st));
   PASTA_CUDA(cudaStreamSynchronize(st));
   return *p->status_host;
+}
+
+pasta_status_t pasta_profile_enable(pasta_pool_t *p, int32_t on) {
+  if (!p) return PASTA_ERR_INVALID_ARG;
+  if (p->host_only) return PASTA_ERR_BAD_STATE;
+  if (on && p->prof_events.empty()) {
+    p->prof_events.resize(4 * kProfCalls, nullptr);
+    p->prof_mask.assign(kProfCalls, 0);
+    for (cudaEvent_t &e : p->prof_events) PASTA_CUDA(cudaEventCreate(&e));
+  }
+  p->profiling = on != 0;
+  p->prof_calls = 0;
+  return PASTA_OK;
+}
+
+pasta_status_t pasta_profile_read(pasta_pool_t *p, double *out_ms, int64_t *out_launches) {
+  if (!p || !out_ms || !out_launches) return PASTA_ERR_INVALID_ARG;
+  for (int k = 0; k < 3; ++k) { out_ms[k] = 0; out_launches[k] = 0; }
+  for (int i = 0; i < p->prof_calls; ++i) {
+    cudaEvent_t *ev = &p->prof_events[4 * i];
+    PASTA_CUDA(cudaEventSynchronize(ev[3]));
+    for (int k = 0; k < 3; ++k) {
+      if (!(p->prof_mask[i] & (1 << k))) continue;
+      float ms = 0;
+      PASTA_CUDA(cudaEventElapsedTime(&ms, ev[k], ev[k + 1]));
+      out_ms[k] += ms;
+      out_launches[k] += 1;
+    }
+  }
+  p->prof_calls = 0;
+  return PASTA_OK;
 }
 
 pasta_status_t pasta_launch_count(pasta_pool_t *p, int64_t *out) {
