@@ -177,6 +177,30 @@ pasta_status_t pasta_step_host(pasta_pool_t *pool, int32_t n, const int32_t *req
                                const void *k_new, const void *v_new, const void *q, void *out,
                                void *staging, size_t staging_bytes, float scale, void *stream);
 
+/*
+ * (No counterpart in the paper: an addition for callers that are not allowed to allocate.)
+ *
+ * pasta_decode_attn for ONE layer of the planned step, with the intermediate partial results (one
+ * (max, sum, unnormalised output) row per query head and per piece of the visible set) kept in a fixed
+ * array inside the library's own device image instead of in workspace memory.  The call itself calls no
+ * allocation routine of any kind, which is what code running under a memory budget that is frozen after
+ * start-up needs: inference-engine plug-ins, real-time loops, or a process whose GPU memory is entirely
+ * owned by a framework's arena.
+ *   - The array holds PASTA_NOALLOC_MAX_ROWS partial rows (about 8 MiB; every GPU that loads the library
+ *     carries it until the process exits).  A step whose plan needs more rows is refused with
+ *     PASTA_ERR_CAPACITY; use pasta_decode_attn for those.
+ *   - The first call on a device looks up the array's device address (a runtime query, no allocation).
+ *     Make that first call outside any stream capture.  The pool's device must be the current device.
+ *   - All calls, from all pools, share the one array per GPU and each overwrites what the previous one
+ *     left: two calls whose kernels may run at the same time on one GPU (different streams, different
+ *     pools or processes' threads) race on it and corrupt each other's results.  Serialise them.
+ * q, out, lse, scale, stream: as for pasta_decode_attn with layer_count == 1
+ * (q: device bf16 [n, n_q_heads, head_dim]; out: device fp32 of the same shape).
+ */
+#define PASTA_NOALLOC_MAX_ROWS 16384
+pasta_status_t pasta_decode_attn_noalloc(pasta_pool_t *pool, int32_t layer, const void *q, void *out,
+                                         float *lse, float scale, void *stream);
+
 /* ---- introspection ---------------------------------------------------------------------------- */
 
 /*

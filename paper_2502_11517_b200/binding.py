@@ -24,7 +24,7 @@ EXPORTS = [
     "pasta_sync_merge", "pasta_step_begin", "pasta_step_slots", "pasta_kv_append", "pasta_decode_attn",
     "pasta_kv_append_run", "pasta_step_host_bytes", "pasta_step_host", "pasta_kv_read",
     "pasta_pool_dump", "pasta_plan_dump", "pasta_pool_status", "pasta_launch_count",
-    "pasta_profile_enable", "pasta_profile_read",
+    "pasta_profile_enable", "pasta_profile_read", "pasta_decode_attn_noalloc",
     "pasta_last_cuda_error",
 ]
 
@@ -188,6 +188,12 @@ class Pool:
         cnt = self.n_layers - layer_begin if layer_count is None else layer_count
         _check(lib().pasta_decode_attn(self._h, layer_begin, cnt, _dev(q), _dev(out), _dev(lse), C.c_float(scale),
                                        _stream(stream)), "pasta_decode_attn")
+
+    def decode_attn_noalloc(self, q, out, lse=None, scale: float = 0.0, layer: int = 0, stream=None) -> None:
+        """One layer of the planned step, partial results in the library's built-in device array: the call
+        allocates nothing (see include/pasta.h for the size limit and the sharing rule)."""
+        _check(lib().pasta_decode_attn_noalloc(self._h, layer, _dev(q), _dev(out), _dev(lse), C.c_float(scale),
+                                               _stream(stream)), "pasta_decode_attn_noalloc")
 
     def kv_append_run(self, req: int, thread: int, m: int, k=None, v=None, layer_begin: int = 0,
                       layer_count: Optional[int] = None, stream=None) -> None:

@@ -133,6 +133,21 @@ PlanLimits limits_of(const pasta_pool *p) {
 
 }  // namespace
 
+namespace pasta {
+// for entry points that live in other files
+bool pool_step_view(pasta_pool_t *p, PoolView *pv, PlanHeader *hdr, int32_t *n_layers, int32_t *head_dim,
+                    int32_t *device) {
+  if (p->host_only || !p->plan_valid) return false;
+  *pv = p->pv;
+  *hdr = p->hdr;
+  *n_layers = p->cfg.n_layers;
+  *head_dim = p->cfg.head_dim;
+  *device = p->cfg.device;
+  return true;
+}
+void pool_count_launches(pasta_pool_t *p, int n) { p->launches += n; }
+}  // namespace pasta
+
 extern "C" {
 
 int32_t pasta_last_cuda_error(void) { return g_last_cuda_error; }

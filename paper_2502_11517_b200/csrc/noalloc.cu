@@ -1,0 +1,66 @@
+// pasta_decode_attn_noalloc: decode attention of one layer with the split/segment partial results
+// kept in a fixed device array that is part of the library image, so that the call needs no
+// workspace memory from anybody and allocates nothing.
+#include "device_common.cuh"
+#include "kernels.hpp"
+
+namespace pasta {
+// defined in api.cu: the device view and plan header of a pool's current step (false: no valid plan / host-only)
+bool pool_step_view(pasta_pool_t *pool, PoolView *pv, PlanHeader *hdr, int32_t *n_layers, int32_t *head_dim,
+                    int32_t *device);
+void pool_count_launches(pasta_pool_t *pool, int n);
+}  // namespace pasta
+
+using namespace pasta;
+
+namespace {
+
+constexpr int kMaxRows = PASTA_NOALLOC_MAX_ROWS;                   // partial rows one call may need
+constexpr size_t kMlBytes = size_t(kMaxRows) * sizeof(float2);     // (m, l) per row
+constexpr size_t kScratchBytes = kMlBytes + size_t(kMaxRows) * 128 * sizeof(float);
+
+// Lives in every GPU's memory from the moment the library is loaded there until the process exits.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[kScratchBytes];
+
+// In host code `g_noalloc_scratch` is only a handle for the runtime, not an address a kernel can use:
+// the device address is looked up once per device and cached here.
+constexpr int kMaxDevices = 64;
+void *g_scratch_addr[kMaxDevices] = {nullptr};
+
+}  // namespace
+
+extern "C" pasta_status_t pasta_decode_attn_noalloc(pasta_pool_t *pool, int32_t layer, const void *q, void *out,
+                                                    float *lse, float scale, void *stream) {
+  if (!pool || !q || !out || !(scale >= 0.f)) return PASTA_ERR_INVALID_ARG;
+  PoolView pv;
+  PlanHeader hdr;
+  int32_t n_layers = 0, head_dim = 0, device = 0;
+  if (!pool_step_view(pool, &pv, &hdr, &n_layers, &head_dim, &device)) return PASTA_ERR_BAD_STATE;
+  if (layer < 0 || layer >= n_layers) return PASTA_ERR_INVALID_ARG;
+  if (hdr.w[PH_N_QUERIES] == 0) return PASTA_OK;
+  if (hdr.w[PH_ROWS] > kMaxRows) return PASTA_ERR_CAPACITY;       // this step needs more partial rows than the array holds
+  int current = -1;
+  if (cudaGetDevice(&current) != cudaSuccess || current != device || device < 0 || device >= kMaxDevices)
+    return PASTA_ERR_INVALID_ARG;                                  // the pool's device must be the current one
+  if (!g_scratch_addr[device]) {
+    void *ptr = nullptr;
+    const cudaError_t e = cudaGetSymbolAddress(&ptr, g_noalloc_scratch);
+    if (e != cudaSuccess || !ptr) return PASTA_ERR_CUDA;
+    g_scratch_addr[device] = ptr;
+  }
+  unsigned char *scratch = static_cast<unsigned char *>(g_scratch_addr[device]);
+  pv.part_ml = reinterpret_cast<float2 *>(scratch);
+  pv.part_o = reinterpret_cast<float *>(scratch + kMlBytes);
+  pv.rows_per_layer = kMaxRows;
+  // Nothing in the array has to start at zero: each kernel writes every partial row of the step before the
+  // merge reads it, so the previous call's contents are simply overwritten.
+  const float sc = (scale == 0.f ? rsqrtf(static_cast<float>(head_dim)) : scale) * 1.4426950408889634f;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  cudaError_t e = cudaSuccess;
+  int launched = 0;
+  if (hdr.w[PH_N_TUNITS] > 0) { e = launch_attn_tensor(pv, hdr, layer, 1, q, sc, st); ++launched; }
+  if (e == cudaSuccess && hdr.w[PH_N_WUNITS] > 0) { e = launch_attn_warp(pv, hdr, layer, 1, q, sc, st); ++launched; }
+  if (e == cudaSuccess) { e = launch_merge(pv, hdr, 1, static_cast<float *>(out), lse, st); ++launched; }
+  pool_count_launches(pool, launched);
+  return e == cudaSuccess ? PASTA_OK : PASTA_ERR_CUDA;
+}
