@@ -39,12 +39,12 @@ FALLBACK_HBM_GBS = 6650.0
 NCU_TRAFFIC_BYTES = {"long_shared_prefix": None, "batched": None, "single_request": None}
 
 
-def make_script(workload: str):
+def make_script(workload: str, size: str = "full"):
     from pasta_workloads import cfg2_single_request, cfg3_batched, cfg4_long_prefix
     if workload == "long_shared_prefix":
-        return cfg4_long_prefix()
+        return cfg4_long_prefix() if size == "full" else cfg4_long_prefix(prefix=8192)
     if workload == "batched":
-        return cfg3_batched()
+        return cfg3_batched() if size == "full" else cfg3_batched(n_layers=4)
     if workload == "single_request":
         return cfg2_single_request("a")
     raise SystemExit(f"unknown workload {workload}")
@@ -202,7 +202,7 @@ def run_ours(args):
         dist.barrier()
     device = torch.device("cuda", local)
     torch.cuda.set_device(device)
-    script = make_script(args.workload)
+    script = make_script(args.workload, args.size)
     geo = script.geometry
     e2e_steps = max(3, min(args.steps, 50))
     pool, entries, randn = build_state(script, device, seed_offset=rank,
@@ -300,7 +300,7 @@ def run_ours(args):
         "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {
-            "workload": args.workload, "script": script.name, "requests": len(set(reqs)), "thread_tokens_per_step": n,
+            "workload": args.workload, "size": args.size, "script": script.name, "requests": len(set(reqs)), "thread_tokens_per_step": n,
             "layers": L, "n_q_heads": geo.n_q_heads, "n_kv_heads": geo.n_kv_heads, "head_dim": geo.head_dim,
             "page_size": geo.page_size, "unique_kv_tokens_per_layer": avg_tokens,
             "unique_kv_bytes_per_step": step_bytes, "l2": "inputs larger than L2" if step_bytes / L > 126e6 * 1.5 else
@@ -422,6 +422,8 @@ def main():
     ap.add_argument("--workload", default="long_shared_prefix")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--size", default="full", choices=["full", "small"],
+                    help="small: a reduced copy of the workload for profiler captures (prefix 8192 / 4 layers)")
     args = ap.parse_args()
     if args.impl == "reference":
         if args.steps == 200:

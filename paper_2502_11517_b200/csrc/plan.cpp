@@ -154,55 +154,52 @@ pasta_status_t build_plan(const HostPool &pool, const std::vector<StepEntry> &en
   std::vector<int32_t> tcta;
   int32_t t_rows = 0;
   if (!treqs.empty()) {
-    const double overhead = 2.0;           // cost of starting a unit, in tiles
-    const int32_t min_piece = 4;           // do not leave fragments smaller than this many tiles
+    // Every tile has a position on a cost axis (tiles, plus `overhead` at the start of each (t-request, kv head)
+    // run); CTA c owns positions [c, c + 1) * total / grid.  Positions are absolute, so rounding at one cut does
+    // not move the others.  Cuts that would leave fewer than `min_piece` tiles on one side snap to the run's end.
+    const double overhead = 2.0;
+    const int32_t min_piece = 2;
     double total = 0;
     for (const TReq &t : treqs)
       total += lim.n_kv_heads * ((t.n_pages + PASTA_TILE_PAGES - 1) / PASTA_TILE_PAGES + overhead);
     const int32_t grid = std::max(1, lim.grid);
     const double target = total / grid;
-    int32_t cta = 0;
-    double acc = 0;
-    tcta.assign(2 * grid, 0);
-    auto close_cta = [&]() {
-      tcta[2 * cta + 1] = static_cast<int32_t>(tunits.size());
-      if (cta + 1 < grid) {
-        ++cta;
-        tcta[2 * cta] = tcta[2 * cta + 1] = static_cast<int32_t>(tunits.size());
-        acc = 0;
-      }
-    };
+    std::vector<int32_t> unit_cta;
+    double cum = 0;
     for (size_t ti = 0; ti < treqs.size(); ++ti) {
       const int32_t n_tiles = (treqs[ti].n_pages + PASTA_TILE_PAGES - 1) / PASTA_TILE_PAGES;
       const int32_t rows = treqs[ti].n_threads * G;
       for (int32_t g = 0; g < lim.n_kv_heads; ++g) {
         trange[(ti * lim.n_kv_heads + g) * 2] = static_cast<int32_t>(tunits.size());
+        cum += overhead;
         int32_t begin = 0;
         while (begin < n_tiles) {
           const int32_t remaining = n_tiles - begin;
+          int32_t c = std::min<int32_t>(grid - 1, static_cast<int32_t>(cum / target));
+          if (c + 1 < grid && (c + 1) * target - cum < min_piece) ++c;   // too close to the CTA's end: next one
           int32_t take = remaining;
-          if (cta + 1 < grid) {
-            const double room = target - acc - overhead;
-            if (room < std::min(remaining, min_piece)) {
-              if (acc > 0) { close_cta(); continue; }
-            } else if (room < remaining) {
-              take = static_cast<int32_t>(room);
-              if (remaining - take < min_piece) take = remaining;   // no tiny tail
-            }
+          if (c + 1 < grid) {
+            const double room = (c + 1) * target - cum;
+            take = std::min<int32_t>(remaining, std::max<int32_t>(min_piece, static_cast<int32_t>(std::lround(room))));
+            if (remaining - take < min_piece) take = remaining;
           }
           tunits.push_back(TUnit{static_cast<int32_t>(ti), g, begin, begin + take, t_rows});
+          unit_cta.push_back(c);
           t_rows += rows;
           begin += take;
-          acc += take + overhead;
-          if (cta + 1 < grid && acc >= target - 0.5) close_cta();
+          cum += take;
         }
         trange[(ti * lim.n_kv_heads + g) * 2 + 1] = static_cast<int32_t>(tunits.size());
       }
     }
-    tcta[2 * cta + 1] = static_cast<int32_t>(tunits.size());
-    int32_t used = cta + 1;
-    while (used > 0 && tcta[2 * (used - 1)] == tcta[2 * (used - 1) + 1]) --used;
-    tcta.resize(2 * used);
+    for (size_t u = 0; u < tunits.size(); ++u) {
+      if (u == 0 || unit_cta[u] != unit_cta[u - 1]) {
+        if (!tcta.empty()) tcta.back() = static_cast<int32_t>(u);
+        tcta.push_back(static_cast<int32_t>(u));
+        tcta.push_back(static_cast<int32_t>(u));
+      }
+    }
+    tcta.back() = static_cast<int32_t>(tunits.size());
   }
 
   // ---- w-units: pieces of at most `chunk` tokens, ordered (query, kv head, piece)
