@@ -13,7 +13,10 @@
 //
 // Warp roles: warp 0 producer (bulk copies of whole (page, kv head) blocks into a 5-stage ring),
 // warp 1 MMA issue (one thread), warps 2-3 build the stacked, swizzled Q operand of each unit,
-// warps 4-7 softmax and epilogue (thread i owns row i = TMEM lane i).
+// warps 4-7 and 8-11 two softmax groups (thread i of a group owns row i = TMEM lane i).  Even tiles go to
+// group 0, odd tiles to group 1; each group has its own S, P and O buffers and its own (m_ref, l), so the
+// two never exchange anything until the unit's epilogue, where group 0 folds both accumulators into one
+// partial row.
 // Every wait is bounded; on expiry the CTA reports PASTA_ERR_TIMEOUT, drains and leaves.
 #include "device_common.cuh"
 #include "kernels.hpp"
@@ -22,7 +25,7 @@ namespace pasta {
 
 namespace {
 
-constexpr int T_THREADS = 256;
+constexpr int T_THREADS = 384;
 constexpr int T_STAGES = 5;
 constexpr int T_TILE = PASTA_TILE_PAGES * PASTA_PAGE;          // 64 tokens
 constexpr int T_BLOCK = 8192;                                  // bytes of one (page, kv head) block, d = 128
@@ -36,15 +39,16 @@ constexpr int OFF_BAR = OFF_STAGE + T_STAGES * T_STAGE_BYTES;
 // barriers (8 bytes each)
 constexpr int B_FULL = 0, B_EMPTY = B_FULL + T_STAGES, B_SFULL = B_EMPTY + T_STAGES, B_PFULL = B_SFULL + 2,
               B_PVDONE = B_PFULL + 2, B_QFULL = B_PVDONE + 2, B_QFREE = B_QFULL + 1, B_OFULL = B_QFREE + 1,
-              B_OFREE = B_OFULL + 1, B_COUNT = B_OFREE + 1;
+              B_OFREE = B_OFULL + 1, B_MLFULL = B_OFREE + 1, B_COUNT = B_MLFULL + 1;
 constexpr int OFF_META = OFF_BAR + 8 * ((B_COUNT + 1) & ~1);   // per stage: 4 page metas
 constexpr int OFF_MISC = OFF_META + T_STAGES * 16;             // tmem base, abort flag
-constexpr int T_SMEM_USED = OFF_MISC + 16;
+constexpr int OFF_ML1 = OFF_MISC + 16;                         // (m_ref, l) of group 1's rows, for the epilogue
+constexpr int T_SMEM_USED = OFF_ML1 + 128 * 8;
 constexpr int T_SMEM_BYTES = T_SMEM_USED + 1024;               // slack to align the base to 1024
 static_assert(T_SMEM_BYTES <= 232448, "shared memory budget");
 
-constexpr uint32_t TMEM_COLS = 256;
-constexpr uint32_t COL_S = 0, COL_O = 128;                     // S buffers at columns 0 and 64, O at 128..255
+constexpr uint32_t TMEM_COLS = 512;
+constexpr uint32_t COL_S = 0, COL_O = 128;                     // S[b] at column 64 b, O[b] at 128 + 128 b
 
 // instruction descriptors: D fp32, A/B bf16, M = 128
 constexpr uint32_t IDESC_BASE = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 4) << 24);
@@ -87,9 +91,31 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float *v) {
         "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
       : "r"(taddr)
       : "memory");
-  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+  // the wait names the registers so that nothing that uses them can be scheduled above it
+  asm volatile("tcgen05.wait::ld.sync.aligned;"
+      : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]), "+r"(r[8]),
+        "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]), "+r"(r[16]),
+        "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]), "+r"(r[23]), "+r"(r[24]),
+        "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
+      :: "memory");
 #pragma unroll
   for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+// 16 consecutive fp32 columns
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float *v) {
+  uint32_t r[16];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;"
+      : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]), "+r"(r[8]),
+        "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15])
+      :: "memory");
+#pragma unroll
+  for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
 }
 __device__ __forceinline__ void tmem_st32(uint32_t taddr, const float *v) {
   uint32_t r[32];
@@ -176,6 +202,7 @@ attn_tensor_kernel(PoolView pv, TensorArgs a, const __nv_bfloat16 *__restrict__ 
     mbar_init(bar + 8 * B_QFREE, 1);
     mbar_init(bar + 8 * B_OFULL, 1);
     mbar_init(bar + 8 * B_OFREE, 128);
+    mbar_init(bar + 8 * B_MLFULL, 128);
     misc[1] = 0;
     mbar_init_fence();
   }
@@ -258,7 +285,7 @@ attn_tensor_kernel(PoolView pv, TensorArgs a, const __nv_bfloat16 *__restrict__ 
               // ---- O += P . V for tile `it - 1` (it has not been advanced for this k yet when k == nt)
               const uint32_t j = (k < nt) ? it - 1 : it - 1;
               const uint32_t s = j % T_STAGES, b = j & 1;
-              if (k == 1 && uc > 0) {   // first P.V of the unit overwrites O: the previous unit's rows must be read out
+              if (k == 1 && uc > 0) {   // the unit's first P.V overwrites an O buffer: the previous unit's rows must be read out
                 if (!wait_or_abort(bar + 8 * B_OFREE, (uc - 1) & 1, abort_flag)) { ok = false; break; }
               }
               if (!wait_or_abort(bar + 8 * (B_PFULL + b), (j >> 1) & 1, abort_flag)) { ok = false; break; }
@@ -267,8 +294,8 @@ attn_tensor_kernel(PoolView pv, TensorArgs a, const __nv_bfloat16 *__restrict__ 
               const uint32_t v_addr = base + OFF_STAGE + s * T_STAGE_BYTES + 2048;
 #pragma unroll
               for (int pg = 0; pg < PASTA_TILE_PAGES; ++pg)
-                mma_ss(tmem + COL_O, smem_desc(p_addr + pg * 32, 16, 1024),
-                       smem_desc(v_addr + pg * T_BLOCK, 1024, 4096), IDESC_PV, (k > 1) || (pg > 0));
+                mma_ss(tmem + COL_O + b * 128, smem_desc(p_addr + pg * 32, 16, 1024),
+                       smem_desc(v_addr + pg * T_BLOCK, 1024, 4096), IDESC_PV, (k > 2) || (pg > 0));
               mma_commit(bar + 8 * (B_EMPTY + s));
               mma_commit(bar + 8 * (B_PVDONE + b));
               if (k == nt) mma_commit(bar + 8 * B_OFULL);
@@ -305,9 +332,12 @@ attn_tensor_kernel(PoolView pv, TensorArgs a, const __nv_bfloat16 *__restrict__ 
       }
     }
   } else {
-    // ================================================================ softmax + epilogue (128 threads)
-    const int row = tid - 128;                      // = TMEM lane
+    // ================================================================ softmax + epilogue (2 groups of 128 threads)
+    const int grp = (warp - 4) >> 2;                // tiles with (it & 1) == grp belong to this group
+    const int row = (tid - 128) & 127;              // = TMEM lane
     const uint32_t lane_addr = static_cast<uint32_t>((warp & 3) * 32) << 16;
+    const uint32_t col_s = COL_S + grp * 64, col_o = COL_O + grp * 128;
+    float2 *ml1 = reinterpret_cast<float2 *>(sm + OFF_ML1);
     uint32_t it = 0, uc = 0;
     bool ok = true;
     for (int ll = 0; ll < a.layer_count && ok; ++ll) {
@@ -316,19 +346,17 @@ attn_tensor_kernel(PoolView pv, TensorArgs a, const __nv_bfloat16 *__restrict__ 
         const int nt = x.tile_end - x.tile_begin;
         const int rows = x.n_threads * G;
         const bool active = row < rows;
-        const bool warp_active = (warp - 4) * 32 < rows;
+        const bool warp_active = ((warp - 4) & 3) * 32 < rows;
         const int32_t *visrow = plan + a.off_vis + x.vis_off + (active ? row / G : 0) * x.n_streams;
         float m_ref = -INFINITY, l = 0.f;
         for (int k = 0; k < nt; ++k, ++it) {
-          const uint32_t s = it % T_STAGES, b = it & 1;
-          if (!wait_or_abort(bar + 8 * (B_SFULL + b), (it >> 1) & 1, abort_flag)) { ok = false; break; }
-          tc_fence_after();
+          if (static_cast<int>(it & 1) != grp) continue;
+          const uint32_t s = it % T_STAGES, b = grp;
+          // the tile's page metas are in shared memory once its copies have landed: fetch the row's thresholds early
+          if (!wait_or_abort(bar + 8 * (B_FULL + s), (it / T_STAGES) & 1, abort_flag)) { ok = false; break; }
+          int thr[PASTA_TILE_PAGES];
+          bool full = true;
           if (warp_active) {
-            float sc[T_TILE];
-            tmem_ld32(tmem + lane_addr + COL_S + b * 64, sc);
-            tmem_ld32(tmem + lane_addr + COL_S + b * 64 + 32, sc + 32);
-            int thr[PASTA_TILE_PAGES];
-            bool full = true;
 #pragma unroll
             for (int pg = 0; pg < PASTA_TILE_PAGES; ++pg) {
               const int meta = meta_s[s * 4 + pg];
@@ -337,47 +365,59 @@ attn_tensor_kernel(PoolView pv, TensorArgs a, const __nv_bfloat16 *__restrict__ 
               thr[pg] = t;
               full = full && (t == PASTA_PAGE);
             }
+          }
+          if (!wait_or_abort(bar + 8 * (B_SFULL + b), (it >> 1) & 1, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          if (warp_active) {
+            float sc[T_TILE];
+            tmem_ld32(tmem + lane_addr + col_s, sc);
+            tmem_ld32(tmem + lane_addr + col_s + 32, sc + 32);
             if (!full) {
 #pragma unroll
               for (int j = 0; j < T_TILE; ++j)
                 if ((j & 15) >= thr[j >> 4]) sc[j] = -INFINITY;
             }
-            float mt = sc[0];
+            float mx[4] = {sc[0], sc[1], sc[2], sc[3]};
 #pragma unroll
-            for (int j = 1; j < T_TILE; ++j) mt = fmaxf(mt, sc[j]);
-            mt *= a.scale_log2;
+            for (int j = 4; j < T_TILE; j += 4) {
+              mx[0] = fmaxf(mx[0], sc[j]); mx[1] = fmaxf(mx[1], sc[j + 1]);
+              mx[2] = fmaxf(mx[2], sc[j + 2]); mx[3] = fmaxf(mx[3], sc[j + 3]);
+            }
+            const float mt = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * a.scale_log2;
             const bool need = mt > m_ref + 8.f;       // also true for the first visible tile (m_ref = -inf)
             const bool rescale = need && l > 0.f;
+            // this group's previous tile is it - 2: its P.V must be done before P[b] is overwritten or O[b] rescaled
+            if (it >= 2 && !wait_or_abort(bar + 8 * (B_PVDONE + b), ((it - 2) >> 1) & 1, abort_flag)) { ok = false; break; }
             if (__any_sync(0xffffffffu, rescale)) {
-              // O and l are relative to m_ref: move them to the new reference.  P.V of the previous tile must be done.
-              if (!wait_or_abort(bar + 8 * (B_PVDONE + (b ^ 1)), ((it - 1) >> 1) & 1, abort_flag)) { ok = false; break; }
+              // O[b] and l are relative to m_ref: move them to the new reference
               tc_fence_after();
               const float f = rescale ? fast_exp2(m_ref - mt) : 1.f;
 #pragma unroll 1
               for (int cb = 0; cb < 4; ++cb) {
                 float ov[32];
-                tmem_ld32(tmem + lane_addr + COL_O + cb * 32, ov);
+                tmem_ld32(tmem + lane_addr + col_o + cb * 32, ov);
 #pragma unroll
                 for (int j = 0; j < 32; ++j) ov[j] *= f;
-                tmem_st32(tmem + lane_addr + COL_O + cb * 32, ov);
+                tmem_st32(tmem + lane_addr + col_o + cb * 32, ov);
               }
               tmem_st_wait();
               l *= f;
             }
             if (need) m_ref = mt;
             const float ref = (m_ref == -INFINITY) ? 0.f : m_ref;
-            float lsum = 0.f;
+            float ls[4] = {0.f, 0.f, 0.f, 0.f};
             uint32_t pk[T_TILE / 2];
 #pragma unroll
-            for (int j = 0; j < T_TILE; j += 2) {
+            for (int j = 0; j < T_TILE; j += 4) {
               const float p0 = fast_exp2(fmaf(sc[j], a.scale_log2, -ref));
               const float p1 = fast_exp2(fmaf(sc[j + 1], a.scale_log2, -ref));
-              lsum += p0 + p1;
+              const float p2 = fast_exp2(fmaf(sc[j + 2], a.scale_log2, -ref));
+              const float p3 = fast_exp2(fmaf(sc[j + 3], a.scale_log2, -ref));
+              ls[0] += p0; ls[1] += p1; ls[2] += p2; ls[3] += p3;
               pk[j >> 1] = pack_bf16(p0, p1);
+              pk[(j >> 1) + 1] = pack_bf16(p2, p3);
             }
-            l += lsum;
-            // P[b] may be overwritten once P.V of tile it-2 has finished
-            if (it >= 2 && !wait_or_abort(bar + 8 * (B_PVDONE + b), ((it - 2) >> 1) & 1, abort_flag)) { ok = false; break; }
+            l += (ls[0] + ls[1]) + (ls[2] + ls[3]);
             uint8_t *prow = sm + OFF_P + b * T_P_BYTES + (row >> 3) * 1024 + (row & 7) * 128;
 #pragma unroll
             for (int c = 0; c < 8; ++c)
@@ -389,20 +429,41 @@ attn_tensor_kernel(PoolView pv, TensorArgs a, const __nv_bfloat16 *__restrict__ 
           mbar_arrive(bar + 8 * (B_PFULL + b));
         }
         if (!ok) break;
-        // ---- epilogue: this unit's rows leave TMEM
+        // ---- epilogue: the unit's rows leave TMEM; group 0 folds group 1's accumulator into its own
         if (!wait_or_abort(bar + 8 * B_OFULL, uc & 1, abort_flag)) { ok = false; break; }
         tc_fence_after();
+        if (grp == 1) {
+          if (active) ml1[row] = make_float2(m_ref, l);
+          mbar_arrive(bar + 8 * B_MLFULL);
+          continue;
+        }
+        if (!wait_or_abort(bar + 8 * B_MLFULL, uc & 1, abort_flag)) { ok = false; break; }
         if (warp_active) {
+          const float2 other = active ? ml1[row] : make_float2(-INFINITY, 0.f);
+          const float m_all = fmaxf(m_ref, other.x);
+          const float f0 = l > 0.f ? fast_exp2(m_ref - m_all) : 0.f;
+          const float f1 = other.y > 0.f ? fast_exp2(other.x - m_all) : 0.f;
+          const float l_all = f0 * l + f1 * other.y;
+          const bool any0 = __any_sync(0xffffffffu, f0 != 0.f), any1 = __any_sync(0xffffffffu, f1 != 0.f);
           const int64_t prow = static_cast<int64_t>(ll) * pv.rows_per_layer + x.row_base + row;
-          if (active) pv.part_ml[prow] = make_float2(m_ref, l);
+          if (active) pv.part_ml[prow] = make_float2(m_all, l_all);
 #pragma unroll 1
-          for (int cb = 0; cb < 4; ++cb) {
-            float ov[32];
-            tmem_ld32(tmem + lane_addr + COL_O + cb * 32, ov);
-            if (active && l > 0.f) {
-              float4 *dst = reinterpret_cast<float4 *>(pv.part_o + prow * 128 + cb * 32);
+          for (int cb = 0; cb < 8; ++cb) {
+            float o0[16], o1[16];
+            if (any0) tmem_ld16(tmem + lane_addr + COL_O + cb * 16, o0);
+            if (any1) tmem_ld16(tmem + lane_addr + COL_O + 128 + cb * 16, o1);
+            if (active && l_all > 0.f) {
+              float4 *dst = reinterpret_cast<float4 *>(pv.part_o + prow * 128 + cb * 16);
 #pragma unroll
-              for (int j = 0; j < 8; ++j) dst[j] = make_float4(ov[4 * j], ov[4 * j + 1], ov[4 * j + 2], ov[4 * j + 3]);
+              for (int j = 0; j < 4; ++j) {
+                float4 r4;
+                // a factor of exactly 0 means that accumulator was never written for this row: do not touch it
+                r4.x = (f0 != 0.f ? f0 * o0[4 * j] : 0.f) + (f1 != 0.f ? f1 * o1[4 * j] : 0.f);
+                r4.y = (f0 != 0.f ? f0 * o0[4 * j + 1] : 0.f) + (f1 != 0.f ? f1 * o1[4 * j + 1] : 0.f);
+                r4.z = (f0 != 0.f ? f0 * o0[4 * j + 2] : 0.f) + (f1 != 0.f ? f1 * o1[4 * j + 2] : 0.f);
+                r4.w = (f0 != 0.f ? f0 * o0[4 * j + 3] : 0.f) + (f1 != 0.f ? f1 * o1[4 * j + 3] : 0.f);
+                dst[j] = r4;
+              }
             }
           }
         }
