@@ -248,10 +248,9 @@ def run_ours(args):
     launches = pool.launch_count() - launches0
     tok1, shared1 = unique_tokens(pool, entries)
     assert pool.status() == 0, "a kernel reported an error"
-    if world > 1:
-        t = torch.tensor([ms], device=device, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    from paper_2502_11517_b200.sharding import aggregate
+    all_tokens, worst_s = aggregate(float(n * args.steps), ms * 1e-3)    # every rank runs its own requests
+    ms = worst_s * 1e3
 
     # ---- end to end: the same step through the host-buffer entry point (copies inside the timed region)
     k_h = k_new.cpu().pin_memory(); v_h = v_new.cpu().pin_memory(); q_h = q.cpu().pin_memory()
@@ -267,10 +266,7 @@ def run_ours(args):
         pool.step_host(reqs, thr, ones, k_h, v_h, q_h, out_h, staging)
     torch.cuda.synchronize(device)
     e2e_s = time.perf_counter() - t0
-    if world > 1:
-        t = torch.tensor([e2e_s], device=device, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_s = float(t.item())
+    e2e_tokens, e2e_s = aggregate(float(n * e2e_steps), e2e_s)
     h2d = k_h.numel() * 2 * 2 + q_h.numel() * 2
     d2h = out_h.numel() * 4
 
@@ -293,7 +289,7 @@ def run_ours(args):
     dom_bytes_per_launch = shared_bytes if dom == 0 else step_bytes - shared_bytes
     dom_ms = kernel_ms[dom] / max(1, kernel_launches[dom])
     achieved = dom_bytes_per_launch / (dom_ms * 1e-3) / 1e9 if dom_ms > 0 else 0.0
-    value = world * n * args.steps / (ms * 1e-3)
+    value = all_tokens / (ms * 1e-3)
     step_gbs = step_bytes / (ms / args.steps * 1e-3) / 1e9
     result = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -312,7 +308,7 @@ def run_ours(args):
             "sync_merge_host_us": merge_us,
         },
         "clocks": clocks,
-        "e2e": {"value": world * n * e2e_steps / e2e_s, "unit": UNIT, "h2d_bytes_per_step": h2d,
+        "e2e": {"value": e2e_tokens / e2e_s, "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "steps": e2e_steps},
         "gpu_launches": launches,
         "roofline": {"bound": "hbm", "kernel": dom_name, "achieved": achieved, "peak": peak, "peak_kind": peak_kind,
