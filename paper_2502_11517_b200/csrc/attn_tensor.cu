@@ -315,17 +315,27 @@ attn_tensor_kernel(PoolView pv, TensorArgs a, const __nv_bfloat16 *__restrict__ 
         const UnitInfo x = load_unit(plan, a.off_tunit, a.off_treq, u);
         if (uc > 0 && !wait_or_abort(bar + 8 * B_QFREE, (uc - 1) & 1, abort_flag)) { ok = false; break; }
         const int rows = x.n_threads * G;
-        for (int idx = t64; idx < 128 * 16; idx += 64) {
-          const int row = idx >> 4, c = idx & 15;
-          uint4 val = make_uint4(0, 0, 0, 0);
+        // thread t64 builds rows 2 t64 and 2 t64 + 1; the 16 loads of a row are issued together before any store
+#pragma unroll 1
+        for (int rr = 0; rr < 2; ++rr) {
+          const int row = t64 * 2 + rr;
+          uint4 val[16];
           if (row < rows) {
             const int t = row / G, hl = row - t * G;
             const int qn = plan[a.off_tq + x.tq_off + t];
-            val = __ldg(reinterpret_cast<const uint4 *>(
-                q + ((static_cast<int64_t>(ll) * a.n_queries + qn) * pv.n_q_heads + x.g * G + hl) * 128 + c * 8));
+            const uint4 *src = reinterpret_cast<const uint4 *>(
+                q + ((static_cast<int64_t>(ll) * a.n_queries + qn) * pv.n_q_heads + x.g * G + hl) * 128);
+#pragma unroll
+            for (int c = 0; c < 16; ++c) val[c] = __ldg(src + c);
+          } else {
+#pragma unroll
+            for (int c = 0; c < 16; ++c) val[c] = make_uint4(0, 0, 0, 0);
           }
           const int r8 = row & 7;
-          *reinterpret_cast<uint4 *>(sm + OFF_Q + (c >> 3) * 16384 + (row >> 3) * 1024 + r8 * 128 + (((c & 7) ^ r8) << 4)) = val;
+          uint8_t *dst = sm + OFF_Q + (row >> 3) * 1024 + r8 * 128;
+#pragma unroll
+          for (int c = 0; c < 16; ++c)
+            *reinterpret_cast<uint4 *>(dst + (c >> 3) * 16384 + (((c & 7) ^ r8) << 4)) = val[c];
         }
         fence_proxy_async();
         mbar_arrive(bar + 8 * B_QFULL);
