@@ -86,7 +86,7 @@ cudaError_t launch_kv_read(const PoolView &pv, const int32_t *slots, int32_t n_t
 // running maximum is a shuffle reduction over the 16 tokens.  P.V: every lane owns D/32 output
 // elements for each of the G heads.
 // =============================================================================================
-constexpr int W_WARPS = 8;
+constexpr int W_WARPS = 1;            // one warp per block: the block scheduler balances the units
 constexpr int W_STAGES = 3;
 
 template <int D, int G>
@@ -121,9 +121,9 @@ attn_warp_kernel(PoolView pv, int32_t off_wunit, int32_t off_pages, int32_t n_wu
   float *p_s = reinterpret_cast<float *>(base + W_STAGES * S::BLOCK + S::Q_BYTES);
   const uint32_t bar0 = smem_u32(base + W_STAGES * S::BLOCK + S::Q_BYTES + S::P_BYTES);
 
-  const int32_t *U = pv.plan + off_wunit + u * PW_WORDS;
-  const int qi = U[PW_QUERY], g = U[PW_KV_HEAD], n_tok = U[PW_N_TOKENS];
-  const int32_t *pg = pv.plan + off_pages + U[PW_PAGE_OFF];
+  const int4 U = *reinterpret_cast<const int4 *>(pv.plan + off_wunit + u * PW_WORDS);   // query, kv head, page offset, tokens
+  const int qi = U.x, g = U.y, n_tok = U.w;
+  const int32_t *pg = pv.plan + off_pages + U.z;
   const int n_pg = (n_tok + PASTA_PAGE - 1) / PASTA_PAGE;
   const uint8_t *kv_layer = pv.kv_base + (layer_begin + ll) * pv.layer_stride;
 
@@ -132,21 +132,14 @@ attn_warp_kernel(PoolView pv, int32_t off_wunit, int32_t off_pages, int32_t n_wu
     mbar_init_fence();
     fence_proxy_async();
   }
-  // the G query rows of this kv head, pre-multiplied by scale * log2(e)
-  {
-    const __nv_bfloat162 *qsrc = reinterpret_cast<const __nv_bfloat162 *>(
-        q + ((static_cast<int64_t>(ll) * n_queries + qi) * pv.n_q_heads + g * G) * D);
-    for (int i = lane; i < G * D / 2; i += 32) {
-      const float2 f = __bfloat1622float2(qsrc[i]);
-      q_s[2 * i] = f.x * scale_log2;
-      q_s[2 * i + 1] = f.y * scale_log2;
-    }
-  }
+  // page ids of the unit's first 64 pages live in registers (lane i: pages i and i + 32), so that refilling a
+  // stage never waits for global memory
+  const int my_pg0 = lane < n_pg ? pg[lane] : 0;
+  const int my_pg1 = lane + 32 < n_pg ? pg[lane + 32] : 0;
   __syncwarp();
-
   auto issue = [&](int i) {
+    int page = i < 32 ? __shfl_sync(0xffffffffu, my_pg0, i) : i < 64 ? __shfl_sync(0xffffffffu, my_pg1, i - 32) : pg[i];
     if (lane == 0) {
-      int page = pg[i];
       if (page < 0 || page >= pv.n_pages) { report(pv.status, PASTA_ERR_DEVICE_CHECK); page = 0; }
       const int s = i % W_STAGES;
       fence_proxy_async();            // the lanes' reads of this stage (ordered by __syncwarp) precede the refill
@@ -156,6 +149,18 @@ attn_warp_kernel(PoolView pv, int32_t off_wunit, int32_t off_pages, int32_t n_wu
     }
   };
   for (int i = 0; i < W_STAGES && i < n_pg; ++i) issue(i);
+  // the G query rows of this kv head, pre-multiplied by scale * log2(e) (overlaps the first copies)
+  {
+    const __nv_bfloat162 *qsrc = reinterpret_cast<const __nv_bfloat162 *>(
+        q + ((static_cast<int64_t>(ll) * n_queries + qi) * pv.n_q_heads + g * G) * D);
+#pragma unroll
+    for (int i = lane; i < G * D / 2; i += 32) {
+      const float2 f = __bfloat1622float2(qsrc[i]);
+      q_s[2 * i] = f.x * scale_log2;
+      q_s[2 * i + 1] = f.y * scale_log2;
+    }
+  }
+  __syncwarp();
 
   float m[G], l[G], o[G][E];
 #pragma unroll
