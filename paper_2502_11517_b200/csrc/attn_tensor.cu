@@ -6,7 +6,7 @@
 //
 //   S[128 x 64]  = Q[128 x 128] . K_tile^T            tcgen05.mma, A and B from shared memory, D in TMEM
 //   P            = 2^(S * scale*log2e - m_ref)         one thread per row, masked by the row's visible lengths
-//   O[128 x 128] += P[128 x 64] . V_tile               tcgen05.mma, P written to shared memory as bf16
+//   O[128 x 128] += P[128 x 64] . V_tile               tcgen05.mma, P (bf16) read from TMEM as the A operand
 //
 // m_ref is a per-row reference that is raised only when a tile's maximum exceeds it by more than 2^8
 // (then O and l are rescaled in TMEM); partial (m_ref, l, O) rows go to the merge kernel.
@@ -26,15 +26,13 @@ namespace pasta {
 namespace {
 
 constexpr int T_THREADS = 384;
-constexpr int T_STAGES = 5;
+constexpr int T_STAGES = 6;
 constexpr int T_TILE = PASTA_TILE_PAGES * PASTA_PAGE;          // 64 tokens
 constexpr int T_BLOCK = 8192;                                  // bytes of one (page, kv head) block, d = 128
 constexpr int T_STAGE_BYTES = PASTA_TILE_PAGES * T_BLOCK;      // 32 KB
 constexpr int T_Q_BYTES = 128 * 128 * 2;                       // 32 KB
-constexpr int T_P_BYTES = 128 * T_TILE * 2;                    // 16 KB
 constexpr int OFF_Q = 0;
-constexpr int OFF_P = OFF_Q + T_Q_BYTES;
-constexpr int OFF_STAGE = OFF_P + 2 * T_P_BYTES;
+constexpr int OFF_STAGE = OFF_Q + T_Q_BYTES;
 constexpr int OFF_BAR = OFF_STAGE + T_STAGES * T_STAGE_BYTES;
 // barriers (8 bytes each)
 constexpr int B_FULL = 0, B_EMPTY = B_FULL + T_STAGES, B_SFULL = B_EMPTY + T_STAGES, B_PFULL = B_SFULL + 2,
@@ -48,7 +46,7 @@ constexpr int T_SMEM_BYTES = T_SMEM_USED + 1024;               // slack to align
 static_assert(T_SMEM_BYTES <= 232448, "shared memory budget");
 
 constexpr uint32_t TMEM_COLS = 512;
-constexpr uint32_t COL_S = 0, COL_O = 128;                     // S[b] at column 64 b, O[b] at 128 + 128 b
+constexpr uint32_t COL_S = 0, COL_O = 128, COL_P = 384;        // S[b] at 64 b, O[b] at 128 + 128 b, P[b] (bf16 pairs) at 384 + 32 b
 
 // instruction descriptors: D fp32, A/B bf16, M = 128
 constexpr uint32_t IDESC_BASE = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 4) << 24);
@@ -66,6 +64,15 @@ __device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a, uint64_t b, 
       "setp.ne.b32 p, %4, 0;\n\t"
       "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
       ::"r"(d_tmem), "l"(a), "l"(b), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// A operand from TMEM: row m in lane m, two bf16 per 32-bit column (16 K-elements = 8 columns)
+__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_tmem), "l"(b), "r"(idesc), "r"(accumulate)
       : "memory");
 }
 __device__ __forceinline__ void mma_commit(uint32_t bar) {
@@ -121,6 +128,17 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const float *v) {
   uint32_t r[32];
 #pragma unroll
   for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(v[i]);
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%32], "
+      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,"
+      "%29,%30,%31};"
+      ::"r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]),
+        "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]), "r"(r[18]),
+        "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]),
+        "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31]), "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st32_u32(uint32_t taddr, const uint32_t *r) {
   asm volatile(
       "tcgen05.st.sync.aligned.32x32b.x32.b32 [%32], "
       "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,"
@@ -290,11 +308,10 @@ attn_tensor_kernel(PoolView pv, TensorArgs a, const __nv_bfloat16 *__restrict__ 
               }
               if (!wait_or_abort(bar + 8 * (B_PFULL + b), (j >> 1) & 1, abort_flag)) { ok = false; break; }
               tc_fence_after();
-              const uint32_t p_addr = base + OFF_P + b * T_P_BYTES;
               const uint32_t v_addr = base + OFF_STAGE + s * T_STAGE_BYTES + 2048;
 #pragma unroll
               for (int pg = 0; pg < PASTA_TILE_PAGES; ++pg)
-                mma_ss(tmem + COL_O + b * 128, smem_desc(p_addr + pg * 32, 16, 1024),
+                mma_ts(tmem + COL_O + b * 128, tmem + COL_P + b * 32 + pg * 8,
                        smem_desc(v_addr + pg * T_BLOCK, 1024, 4096), IDESC_PV, (k > 2) || (pg > 0));
               mma_commit(bar + 8 * (B_EMPTY + s));
               mma_commit(bar + 8 * (B_PVDONE + b));
@@ -428,12 +445,8 @@ attn_tensor_kernel(PoolView pv, TensorArgs a, const __nv_bfloat16 *__restrict__ 
               pk[(j >> 1) + 1] = pack_bf16(p2, p3);
             }
             l += (ls[0] + ls[1]) + (ls[2] + ls[3]);
-            uint8_t *prow = sm + OFF_P + b * T_P_BYTES + (row >> 3) * 1024 + (row & 7) * 128;
-#pragma unroll
-            for (int c = 0; c < 8; ++c)
-              *reinterpret_cast<uint4 *>(prow + ((c ^ (row & 7)) << 4)) =
-                  make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
-            fence_proxy_async();
+            tmem_st32_u32(tmem + lane_addr + COL_P + b * 32, pk);
+            tmem_st_wait();
           }
           tc_fence_before();
           mbar_arrive(bar + 8 * (B_PFULL + b));
