@@ -160,13 +160,13 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 // Bounded wait that also gives up when another role of the CTA has already given up.
 __device__ __forceinline__ bool wait_or_abort(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
   if (mbar_try_wait(bar, parity)) return true;
-  const uint64_t t0 = global_timer_ns();
+  const long long t0 = clock64();
   for (;;) {
 #pragma unroll 1
     for (int i = 0; i < 128; ++i)
       if (mbar_try_wait(bar, parity)) return true;
     if (*abort_flag) return false;
-    if (global_timer_ns() - t0 > 1000000000ull) { *abort_flag = 1; return false; }
+    if (clock64() - t0 > kWaitLimitCycles) { *abort_flag = 1; return false; }
   }
 }
 

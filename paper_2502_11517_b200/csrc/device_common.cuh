@@ -74,22 +74,19 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-__device__ __forceinline__ uint64_t global_timer_ns() {
-  uint64_t t;
-  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-  return t;
-}
+// Upper bound of every wait inside a kernel, in SM clock cycles (about 1.5 s at 2 GHz).
+constexpr long long kWaitLimitCycles = 3000000000ll;
 
-// Waits for the phase with the given parity to complete, for at most ~1 second of wall time.
+// Waits for the phase with the given parity to complete, for at most kWaitLimitCycles.
 // Returns false when the wait was given up (the caller then reports PASTA_ERR_TIMEOUT and leaves).
 __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
   if (mbar_try_wait(bar, parity)) return true;
-  const uint64_t t0 = global_timer_ns();
+  const long long t0 = clock64();
   for (;;) {
 #pragma unroll 1
     for (int i = 0; i < 256; ++i)
       if (mbar_try_wait(bar, parity)) return true;
-    if (global_timer_ns() - t0 > 1000000000ull) return false;
+    if (clock64() - t0 > kWaitLimitCycles) return false;
   }
 }
 
