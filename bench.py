@@ -36,7 +36,7 @@ NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 # dram bytes (read + write) of one launch of the dominant kernel from an ncu capture of this workload,
 # or None when no capture matches the current kernel
-NCU_TRAFFIC_BYTES = {"long_shared_prefix": None, "batched": None, "single_request": None}
+NCU_TRAFFIC_BYTES = {"long_shared_prefix": 1.092e9, "batched": None, "single_request": None}   # see profiles/
 
 
 def make_script(workload: str, size: str = "full"):
