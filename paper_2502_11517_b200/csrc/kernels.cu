@@ -87,7 +87,7 @@ cudaError_t launch_kv_read(const PoolView &pv, const int32_t *slots, int32_t n_t
 // elements for each of the G heads.
 // =============================================================================================
 constexpr int W_WARPS = 1;            // one warp per block: the block scheduler balances the units
-constexpr int W_STAGES = 3;
+constexpr int W_STAGES = 2;
 
 template <int D, int G>
 struct WarpSmem {
@@ -323,30 +323,43 @@ merge_kernel(PoolView pv, int32_t n_queries, int32_t layer_count, int32_t off_qu
     if (i < nt) return lbase + pv.plan[off_tunit + (tb + i) * PU_WORDS + PU_ROW_BASE] + tidx * G + hl;
     return lbase + t_rows + static_cast<int64_t>(w0 + g * nw + (i - nt)) * G + hl;
   };
-  float mstar = -INFINITY;
-  for (int i = lane; i < total; i += 32) {
-    const float2 ml = pv.part_ml[row_of(i)];
-    if (ml.y > 0.f) mstar = fmaxf(mstar, ml.x);
-  }
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) mstar = fmaxf(mstar, __shfl_xor_sync(0xffffffffu, mstar, o));
   const int E = D >> 5;                    // 4 or 2 elements per lane
   float acc[4] = {0.f, 0.f, 0.f, 0.f};
-  float L = 0.f;
-  for (int i = 0; i < total; ++i) {
-    const int64_t row = row_of(i);
-    const float2 ml = pv.part_ml[row];
-    if (!(ml.y > 0.f)) continue;           // nothing visible in that piece
-    const float w = fast_exp2(ml.x - mstar);
-    L = fmaf(w, ml.y, L);
-    const float *src = pv.part_o + row * D + lane * E;
-    if (E == 4) {
-      const float4 v = *reinterpret_cast<const float4 *>(src);
-      acc[0] = fmaf(w, v.x, acc[0]); acc[1] = fmaf(w, v.y, acc[1]);
-      acc[2] = fmaf(w, v.z, acc[2]); acc[3] = fmaf(w, v.w, acc[3]);
-    } else {
-      const float2 v = *reinterpret_cast<const float2 *>(src);
-      acc[0] = fmaf(w, v.x, acc[0]); acc[1] = fmaf(w, v.y, acc[1]);
+  float L = 0.f, mstar = -INFINITY;
+  // lane i looks up partial row i (and i + 32, ...) once; the weighted sum then takes rows and weights from the
+  // lanes' registers, so that only the loads of the partial outputs are left in the loop
+  for (int base_i = 0; base_i < total; base_i += 32) {
+    const int i = base_i + lane;
+    int64_t my_row = 0;
+    float2 my_ml = make_float2(-INFINITY, 0.f);
+    if (i < total) { my_row = row_of(i); my_ml = pv.part_ml[my_row]; }
+    float m_here = my_ml.y > 0.f ? my_ml.x : -INFINITY;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) m_here = fmaxf(m_here, __shfl_xor_sync(0xffffffffu, m_here, o));
+    if (m_here > mstar) {                  // warp-uniform: move what has been summed so far to the new maximum
+      const float f = fast_exp2(mstar - m_here);    // 0 when nothing has been summed yet
+      L *= f;
+#pragma unroll
+      for (int e = 0; e < 4; ++e) acc[e] *= f;
+      mstar = m_here;
+    }
+    const float my_w = my_ml.y > 0.f ? fast_exp2(my_ml.x - mstar) : 0.f;
+    const int cnt = min(32, total - base_i);
+    for (int k = 0; k < cnt; ++k) {
+      const float w = __shfl_sync(0xffffffffu, my_w, k);
+      const float lk = __shfl_sync(0xffffffffu, my_ml.y, k);
+      const int64_t row = __shfl_sync(0xffffffffu, my_row, k);
+      if (w == 0.f) continue;              // nothing visible in that piece (warp-uniform)
+      L = fmaf(w, lk, L);
+      const float *src = pv.part_o + row * D + lane * E;
+      if (E == 4) {
+        const float4 v = *reinterpret_cast<const float4 *>(src);
+        acc[0] = fmaf(w, v.x, acc[0]); acc[1] = fmaf(w, v.y, acc[1]);
+        acc[2] = fmaf(w, v.z, acc[2]); acc[3] = fmaf(w, v.w, acc[3]);
+      } else {
+        const float2 v = *reinterpret_cast<const float2 *>(src);
+        acc[0] = fmaf(w, v.x, acc[0]); acc[1] = fmaf(w, v.y, acc[1]);
+      }
     }
   }
   const float inv = L > 0.f ? 1.f / L : 0.f;
