@@ -25,7 +25,7 @@ struct Derived {
   int32_t group, max_queries, max_rows, layers_per_launch;
   int64_t max_words, staging_words;
   size_t kv_bytes, layer_stride;
-  size_t off_status, off_plan, off_run, off_ml, off_o, ws_bytes;
+  size_t off_status, off_plan, off_plan2, off_run, off_ml, off_o, ws_bytes;
 };
 
 pasta_status_t derive(const pasta_pool_config_t &c, Derived *d) {
@@ -54,6 +54,7 @@ pasta_status_t derive(const pasta_pool_config_t &c, Derived *d) {
   size_t off = 0;
   d->off_status = off; off += 256;
   d->off_plan = off;   off = align_up(off + size_t(d->max_words) * 4, 256);
+  d->off_plan2 = off;  off = align_up(off + size_t(d->max_words) * 4, 256);   // plans of consecutive steps alternate
   d->off_run = off;    off = align_up(off + size_t(2 * kRunChunk) * 4, 256);
   const size_t rows = size_t(d->max_rows) * d->layers_per_launch;
   d->off_ml = off;     off = align_up(off + rows * sizeof(float2), 256);
@@ -82,6 +83,12 @@ struct pasta_pool {
   PlanHeader hdr{};
   bool plan_valid = false;
   int64_t launches = 0;
+  // the plan of step i is uploaded on a stream of its own into buffer i % 2 while step i - 1 still runs
+  int32_t *plan_dev[2] = {nullptr, nullptr};
+  cudaStream_t copy_stream = nullptr;
+  cudaEvent_t plan_ready[2] = {nullptr, nullptr};   // recorded on copy_stream after the upload of buffer b
+  cudaEvent_t work_mark[2] = {nullptr, nullptr};    // recorded on the caller's stream at the start of step i (slot i % 2)
+  int64_t step_index = 0;
   // kernel timing (pasta_profile_*): events[4 * i .. 4 * i + 3] bracket the three kernels of call i
   bool profiling = false;
   std::vector<cudaEvent_t> prof_events;
@@ -194,6 +201,11 @@ pasta_status_t pasta_pool_create(const pasta_pool_config_t *cfg, pasta_pool_t **
       if (e == cudaSuccess) e = cudaEventCreateWithFlags(&p->pinned_free[i], cudaEventDisableTiming);
     }
     if (e == cudaSuccess) e = cudaMallocHost(reinterpret_cast<void **>(&p->status_host), 64);
+    if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&p->copy_stream, cudaStreamNonBlocking);
+    for (int b = 0; b < 2 && e == cudaSuccess; ++b) {
+      e = cudaEventCreateWithFlags(&p->plan_ready[b], cudaEventDisableTiming);
+      if (e == cudaSuccess) e = cudaEventCreateWithFlags(&p->work_mark[b], cudaEventDisableTiming);
+    }
     uint8_t *ws = static_cast<uint8_t *>(cfg->workspace);
     if (e == cudaSuccess) e = cudaMemset(ws, 0, 256);
     // stale bytes of a page's unused tail are multiplied by zero weights, so they must be finite
@@ -210,7 +222,9 @@ pasta_status_t pasta_pool_create(const pasta_pool_config_t *cfg, pasta_pool_t **
     p->pv.n_kv_heads = cfg->n_kv_heads;
     p->pv.head_dim = cfg->head_dim;
     p->pv.status = reinterpret_cast<int32_t *>(ws + d.off_status);
-    p->pv.plan = reinterpret_cast<const int32_t *>(ws + d.off_plan);
+    p->plan_dev[0] = reinterpret_cast<int32_t *>(ws + d.off_plan);
+    p->plan_dev[1] = reinterpret_cast<int32_t *>(ws + d.off_plan2);
+    p->pv.plan = p->plan_dev[0];
     p->run_slots_dev = reinterpret_cast<int32_t *>(ws + d.off_run);
     p->pv.part_ml = reinterpret_cast<float2 *>(ws + d.off_ml);
     p->pv.part_o = reinterpret_cast<float *>(ws + d.off_o);
@@ -227,6 +241,11 @@ pasta_status_t pasta_pool_destroy(pasta_pool_t *p) {
     if (p->pinned[i]) cudaFreeHost(p->pinned[i]);
   }
   if (p->status_host) cudaFreeHost(p->status_host);
+  if (p->copy_stream) { cudaStreamSynchronize(p->copy_stream); cudaStreamDestroy(p->copy_stream); }
+  for (int b = 0; b < 2; ++b) {
+    if (p->plan_ready[b]) cudaEventDestroy(p->plan_ready[b]);
+    if (p->work_mark[b]) cudaEventDestroy(p->work_mark[b]);
+  }
   for (cudaEvent_t e : p->prof_events) if (e) cudaEventDestroy(e);
   delete p;
   return PASTA_OK;
@@ -275,8 +294,19 @@ pasta_status_t pasta_step_begin(pasta_pool_t *p, int32_t n, const int32_t *req_i
   if (s != PASTA_OK) return s;   // the tokens stay reserved; only the attention of this step cannot be planned
   std::memcpy(p->hdr.w, p->plan.data(), sizeof(p->hdr.w));
   if (!p->host_only) {
-    s = upload(p, p->plan.data(), p->plan.size(), const_cast<int32_t *>(p->pv.plan), static_cast<cudaStream_t>(stream));
+    // Buffer b = i % 2 was last read by the kernels of step i - 2.  Everything the caller had enqueued when step
+    // i - 1 began (that is, up to step i - 2) is covered by work_mark[(i - 1) % 2]; the upload waits for that mark
+    // only, so it runs while step i - 1 is still executing, and the caller's stream waits for the upload.
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int64_t i = p->step_index++;
+    const int b = static_cast<int>(i & 1);
+    PASTA_CUDA(cudaEventRecord(p->work_mark[b], st));
+    if (i >= 1) PASTA_CUDA(cudaStreamWaitEvent(p->copy_stream, p->work_mark[b ^ 1], 0));
+    s = upload(p, p->plan.data(), p->plan.size(), p->plan_dev[b], p->copy_stream);
     if (s != PASTA_OK) return s;
+    PASTA_CUDA(cudaEventRecord(p->plan_ready[b], p->copy_stream));
+    PASTA_CUDA(cudaStreamWaitEvent(st, p->plan_ready[b], 0));
+    p->pv.plan = p->plan_dev[b];
   }
   p->plan_valid = true;
   return PASTA_OK;
