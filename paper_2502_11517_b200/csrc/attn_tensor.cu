@@ -375,6 +375,12 @@ attn_tensor_kernel(PoolView pv, TensorArgs a, const __nv_bfloat16 *__restrict__ 
         const bool active = row < rows;
         const bool warp_active = ((warp - 4) & 3) * 32 < rows;
         const int32_t *visrow = plan + a.off_vis + x.vis_off + (active ? row / G : 0) * x.n_streams;
+        // the row's visible lengths of the first four local streams stay in registers for the whole unit: a global
+        // load per page would otherwise sit between two tiles of this group
+        const int vis0 = visrow[0];
+        const int vis1 = x.n_streams > 1 ? visrow[1] : 0;
+        const int vis2 = x.n_streams > 2 ? visrow[2] : 0;
+        const int vis3 = x.n_streams > 3 ? visrow[3] : 0;
         float m_ref = -INFINITY, l = 0.f;
         for (int k = 0; k < nt; ++k, ++it) {
           if (static_cast<int>(it & 1) != grp) continue;
@@ -388,7 +394,11 @@ attn_tensor_kernel(PoolView pv, TensorArgs a, const __nv_bfloat16 *__restrict__ 
             for (int pg = 0; pg < PASTA_TILE_PAGES; ++pg) {
               const int meta = meta_s[s * 4 + pg];
               int t = 0;
-              if (active && meta >= 0) t = min(max(visrow[meta & 255] - (meta >> 8) * PASTA_PAGE, 0), PASTA_PAGE);
+              if (active && meta >= 0) {
+                const int sl = meta & 255;
+                const int vis = sl == 0 ? vis0 : sl == 1 ? vis1 : sl == 2 ? vis2 : sl == 3 ? vis3 : visrow[sl];
+                t = min(max(vis - (meta >> 8) * PASTA_PAGE, 0), PASTA_PAGE);
+              }
               thr[pg] = t;
               full = full && (t == PASTA_PAGE);
             }
