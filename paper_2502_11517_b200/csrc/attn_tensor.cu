@@ -1,22 +1,22 @@
 // K2: tensor-core pass over streams shared by several queries of a request (head_dim 128).
 //
-// One persistent CTA per SM walks its contiguous range of t-units.  A t-unit is a range of 64-token
-// tiles (4 pages) of one request's shared page list, for one kv head.  Rows of the score matrix are
-// the request's queries times the `group` query heads of that kv head (<= 128 rows, zero padded):
+// One persistent CTA per SM walks its contiguous range of t-units.  A t-unit is a range of 128-token tiles
+// (8 pages) of one request's shared page list, for one kv head.  Rows of the score matrix are the request's
+// queries times the `group` query heads of that kv head (<= 128 rows, zero padded):
 //
-//   S[128 x 64]  = Q[128 x 128] . K_tile^T            tcgen05.mma, A and B from shared memory, D in TMEM
-//   P            = 2^(S * scale*log2e - m_ref)         one thread per row, masked by the row's visible lengths
-//   O[128 x 128] += P[128 x 64] . V_tile               tcgen05.mma, P (bf16) read from TMEM as the A operand
+//   S[128 x 128] = Q[128 x 128] . K_tile^T            tcgen05.mma (N = 128), A and B from shared memory, D in TMEM
+//   P            = 2^(S * scale*log2e - m_ref)         one thread per row and half tile, masked by visible lengths
+//   O_h[128 x 128] += P_h[128 x 64] . V_half           tcgen05.mma, P (bf16) read from TMEM as the A operand
 //
-// m_ref is a per-row reference that is raised only when a tile's maximum exceeds it by more than 2^8
-// (then O and l are rescaled in TMEM); partial (m_ref, l, O) rows go to the merge kernel.
+// The two halves h of a tile (pages 0-3 and 4-7) belong to two softmax groups.  Each group has its own running
+// reference m_ref, sum l and accumulator O_h, so the groups exchange nothing until the unit's epilogue, where
+// group 0 folds both accumulators into one partial row.  m_ref is raised only when a half tile's maximum exceeds
+// it by more than 2^8 (then O_h and l are rescaled in TMEM).  P overwrites the first 32 columns of the scores it
+// was computed from; S is double-buffered so that Q.K^T of the next tile runs during the softmax of this one.
 //
-// Warp roles: warp 0 producer (bulk copies of whole (page, kv head) blocks into a 5-stage ring),
-// warp 1 MMA issue (one thread), warps 2-3 build the stacked, swizzled Q operand of each unit,
-// warps 4-7 and 8-11 two softmax groups (thread i of a group owns row i = TMEM lane i).  Even tiles go to
-// group 0, odd tiles to group 1; each group has its own S, P and O buffers and its own (m_ref, l), so the
-// two never exchange anything until the unit's epilogue, where group 0 folds both accumulators into one
-// partial row.
+// Warp roles: warp 0 producer (eight lanes issue the bulk copies of a tile's (page, kv head) blocks into a
+// 3-stage ring of 64 KB), warp 1 MMA issue (one thread), warps 2-3 build the stacked, swizzled Q operand of each
+// unit, warps 4-7 and 8-11 the two softmax groups (thread i of a group owns row i = TMEM lane i).
 // Every wait is bounded; on expiry the CTA reports PASTA_ERR_TIMEOUT, drains and leaves.
 #include "device_common.cuh"
 #include "kernels.hpp"
@@ -26,31 +26,35 @@ namespace pasta {
 namespace {
 
 constexpr int T_THREADS = 384;
-constexpr int T_STAGES = 6;
-constexpr int T_TILE = PASTA_TILE_PAGES * PASTA_PAGE;          // 64 tokens
+constexpr int T_STAGES = 3;
+constexpr int T_TILE = PASTA_TILE_PAGES * PASTA_PAGE;          // 128 tokens
+constexpr int T_HALF = T_TILE / 2;                              // columns of one softmax group
+constexpr int T_HALF_PAGES = PASTA_TILE_PAGES / 2;
+static_assert(PASTA_TILE_PAGES == 8, "the kernel is written for 8-page tiles");
 constexpr int T_BLOCK = 8192;                                  // bytes of one (page, kv head) block, d = 128
-constexpr int T_STAGE_BYTES = PASTA_TILE_PAGES * T_BLOCK;      // 32 KB
+constexpr int T_STAGE_BYTES = PASTA_TILE_PAGES * T_BLOCK;      // 64 KB
 constexpr int T_Q_BYTES = 128 * 128 * 2;                       // 32 KB
 constexpr int OFF_Q = 0;
 constexpr int OFF_STAGE = OFF_Q + T_Q_BYTES;
 constexpr int OFF_BAR = OFF_STAGE + T_STAGES * T_STAGE_BYTES;
 // barriers (8 bytes each)
 constexpr int B_FULL = 0, B_EMPTY = B_FULL + T_STAGES, B_SFULL = B_EMPTY + T_STAGES, B_PFULL = B_SFULL + 2,
-              B_PVDONE = B_PFULL + 2, B_QFULL = B_PVDONE + 2, B_QFREE = B_QFULL + 1, B_OFULL = B_QFREE + 1,
+              B_QFULL = B_PFULL + 4,   // PFULL[2 * b + group]
+              B_QFREE = B_QFULL + 1, B_OFULL = B_QFREE + 1,
               B_OFREE = B_OFULL + 1, B_MLFULL = B_OFREE + 1, B_COUNT = B_MLFULL + 1;
-constexpr int OFF_META = OFF_BAR + 8 * ((B_COUNT + 1) & ~1);   // per stage: 4 page metas
-constexpr int OFF_MISC = OFF_META + T_STAGES * 16;             // tmem base, abort flag
+constexpr int OFF_META = OFF_BAR + 8 * ((B_COUNT + 1) & ~1);   // per stage: 8 page metas
+constexpr int OFF_MISC = OFF_META + T_STAGES * 32;             // tmem base, abort flag
 constexpr int OFF_ML1 = OFF_MISC + 16;                         // (m_ref, l) of group 1's rows, for the epilogue
 constexpr int T_SMEM_USED = OFF_ML1 + 128 * 8;
 constexpr int T_SMEM_BYTES = T_SMEM_USED + 1024;               // slack to align the base to 1024
 static_assert(T_SMEM_BYTES <= 232448, "shared memory budget");
 
 constexpr uint32_t TMEM_COLS = 512;
-constexpr uint32_t COL_S = 0, COL_O = 128, COL_P = 384;        // S[b] at 64 b, O[b] at 128 + 128 b, P[b] (bf16 pairs) at 384 + 32 b
+constexpr uint32_t COL_S = 0, COL_O = 256;   // S[b] at 128 b (group g: columns 64 g .. 64 g + 63; its P reuses the first 32), O_g at 256 + 128 g
 
 // instruction descriptors: D fp32, A/B bf16, M = 128
 constexpr uint32_t IDESC_BASE = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 4) << 24);
-constexpr uint32_t IDESC_QK = IDESC_BASE | ((64u >> 3) << 17);                 // N = 64, both operands K-major
+constexpr uint32_t IDESC_QK = IDESC_BASE | ((128u >> 3) << 17);                // N = 128, both operands K-major
 constexpr uint32_t IDESC_PV = IDESC_BASE | ((128u >> 3) << 17) | (1u << 16);   // N = 128, B (= V) MN-major
 
 __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
@@ -213,8 +217,8 @@ attn_tensor_kernel(PoolView pv, TensorArgs a, const __nv_bfloat16 *__restrict__ 
     for (int s = 0; s < T_STAGES; ++s) { mbar_init(bar + 8 * (B_FULL + s), 1); mbar_init(bar + 8 * (B_EMPTY + s), 1); }
     for (int b = 0; b < 2; ++b) {
       mbar_init(bar + 8 * (B_SFULL + b), 1);
-      mbar_init(bar + 8 * (B_PFULL + b), 128);
-      mbar_init(bar + 8 * (B_PVDONE + b), 1);
+      mbar_init(bar + 8 * (B_PFULL + 2 * b), 128);
+      mbar_init(bar + 8 * (B_PFULL + 2 * b + 1), 128);
     }
     mbar_init(bar + 8 * B_QFULL, 64);
     mbar_init(bar + 8 * B_QFREE, 1);
@@ -255,7 +259,7 @@ attn_tensor_kernel(PoolView pv, TensorArgs a, const __nv_bfloat16 *__restrict__ 
               meta = plan[a.off_pmeta + x.page_off + tile * PASTA_TILE_PAGES + lane];
               if (page < 0 || page >= pv.n_pages) { report(pv.status, PASTA_ERR_DEVICE_CHECK); page = 0; meta = -1; }
             }
-            meta_s[s * 4 + lane] = meta;
+            meta_s[s * PASTA_TILE_PAGES + lane] = meta;
           }
           if (lane == 0) mbar_expect_tx(bar + 8 * (B_FULL + s), n_valid * T_BLOCK);
           __syncwarp();
@@ -285,7 +289,7 @@ attn_tensor_kernel(PoolView pv, TensorArgs a, const __nv_bfloat16 *__restrict__ 
           tc_fence_after();
           for (int k = 0; k <= nt && ok; ++k) {
             if (k < nt) {
-              // ---- S[b] = Q . K^T for tile `it`
+              // ---- S[b] = Q . K^T for tile `it` (S[b] was last used by tile it - 2, whose P.V was issued before this)
               const uint32_t s = it % T_STAGES, b = it & 1;
               if (!wait_or_abort(bar + 8 * (B_FULL + s), (it / T_STAGES) & 1, abort_flag)) { ok = false; break; }
               tc_fence_after();
@@ -293,28 +297,30 @@ attn_tensor_kernel(PoolView pv, TensorArgs a, const __nv_bfloat16 *__restrict__ 
 #pragma unroll
               for (int ks = 0; ks < 8; ++ks) {
                 const uint32_t half = ks >> 2, kk = ks & 3;
-                mma_ss(tmem + COL_S + b * 64, smem_desc(q_addr + half * 16384 + kk * 32, 16, 1024),
+                mma_ss(tmem + COL_S + b * T_TILE, smem_desc(q_addr + half * 16384 + kk * 32, 16, 1024),
                        smem_desc(k_addr + half * 1024 + kk * 32, 16, 4096), IDESC_QK, ks > 0);
               }
               mma_commit(bar + 8 * (B_SFULL + b));
               if (k == nt - 1) mma_commit(bar + 8 * B_QFREE);   // the Q operand may be replaced once these finish
             }
             if (k > 0) {
-              // ---- O += P . V for tile `it - 1` (it has not been advanced for this k yet when k == nt)
-              const uint32_t j = (k < nt) ? it - 1 : it - 1;
+              // ---- O_g += P_g . V_g for both halves of tile `it - 1` (when k == nt, `it` already points past it)
+              const uint32_t j = it - 1;
               const uint32_t s = j % T_STAGES, b = j & 1;
-              if (k == 1 && uc > 0) {   // the unit's first P.V overwrites an O buffer: the previous unit's rows must be read out
+              if (k == 1 && uc > 0) {   // the unit's first P.V overwrites the accumulators: the previous unit's rows must be read out
                 if (!wait_or_abort(bar + 8 * B_OFREE, (uc - 1) & 1, abort_flag)) { ok = false; break; }
               }
-              if (!wait_or_abort(bar + 8 * (B_PFULL + b), (j >> 1) & 1, abort_flag)) { ok = false; break; }
-              tc_fence_after();
               const uint32_t v_addr = base + OFF_STAGE + s * T_STAGE_BYTES + 2048;
+              for (uint32_t g2 = 0; g2 < 2 && ok; ++g2) {
+                if (!wait_or_abort(bar + 8 * (B_PFULL + 2 * b + g2), (j >> 1) & 1, abort_flag)) { ok = false; break; }
+                tc_fence_after();
 #pragma unroll
-              for (int pg = 0; pg < PASTA_TILE_PAGES; ++pg)
-                mma_ts(tmem + COL_O + b * 128, tmem + COL_P + b * 32 + pg * 8,
-                       smem_desc(v_addr + pg * T_BLOCK, 1024, 4096), IDESC_PV, (k > 2) || (pg > 0));
+                for (int pg = 0; pg < T_HALF_PAGES; ++pg)
+                  mma_ts(tmem + COL_O + g2 * 128, tmem + COL_S + b * T_TILE + g2 * T_HALF + pg * 8,
+                         smem_desc(v_addr + (g2 * T_HALF_PAGES + pg) * T_BLOCK, 1024, 4096), IDESC_PV, (k > 1) || (pg > 0));
+              }
+              if (!ok) break;
               mma_commit(bar + 8 * (B_EMPTY + s));
-              mma_commit(bar + 8 * (B_PVDONE + b));
               if (k == nt) mma_commit(bar + 8 * B_OFULL);
             }
             if (k < nt) ++it;
@@ -360,10 +366,10 @@ attn_tensor_kernel(PoolView pv, TensorArgs a, const __nv_bfloat16 *__restrict__ 
     }
   } else {
     // ================================================================ softmax + epilogue (2 groups of 128 threads)
-    const int grp = (warp - 4) >> 2;                // tiles with (it & 1) == grp belong to this group
+    const int grp = (warp - 4) >> 2;                // this group's half of every tile: pages 4 grp .. 4 grp + 3
     const int row = (tid - 128) & 127;              // = TMEM lane
     const uint32_t lane_addr = static_cast<uint32_t>((warp & 3) * 32) << 16;
-    const uint32_t col_s = COL_S + grp * 64, col_o = COL_O + grp * 128;
+    const uint32_t col_o = COL_O + grp * 128;
     float2 *ml1 = reinterpret_cast<float2 *>(sm + OFF_ML1);
     uint32_t it = 0, uc = 0;
     bool ok = true;
@@ -383,16 +389,16 @@ attn_tensor_kernel(PoolView pv, TensorArgs a, const __nv_bfloat16 *__restrict__ 
         const int vis3 = x.n_streams > 3 ? visrow[3] : 0;
         float m_ref = -INFINITY, l = 0.f;
         for (int k = 0; k < nt; ++k, ++it) {
-          if (static_cast<int>(it & 1) != grp) continue;
-          const uint32_t s = it % T_STAGES, b = grp;
+          const uint32_t s = it % T_STAGES, b = it & 1;
+          const uint32_t col_s = COL_S + b * T_TILE + grp * T_HALF;
           // the tile's page metas are in shared memory once its copies have landed: fetch the row's thresholds early
           if (!wait_or_abort(bar + 8 * (B_FULL + s), (it / T_STAGES) & 1, abort_flag)) { ok = false; break; }
-          int thr[PASTA_TILE_PAGES];
+          int thr[T_HALF_PAGES];
           bool full = true;
           if (warp_active) {
 #pragma unroll
-            for (int pg = 0; pg < PASTA_TILE_PAGES; ++pg) {
-              const int meta = meta_s[s * 4 + pg];
+            for (int pg = 0; pg < T_HALF_PAGES; ++pg) {
+              const int meta = meta_s[s * PASTA_TILE_PAGES + grp * T_HALF_PAGES + pg];
               int t = 0;
               if (active && meta >= 0) {
                 const int sl = meta & 255;
@@ -406,27 +412,27 @@ attn_tensor_kernel(PoolView pv, TensorArgs a, const __nv_bfloat16 *__restrict__ 
           if (!wait_or_abort(bar + 8 * (B_SFULL + b), (it >> 1) & 1, abort_flag)) { ok = false; break; }
           tc_fence_after();
           if (warp_active) {
-            float sc[T_TILE];
+            float sc[T_HALF];
             tmem_ld32(tmem + lane_addr + col_s, sc);
             tmem_ld32(tmem + lane_addr + col_s + 32, sc + 32);
             if (!full) {
 #pragma unroll
-              for (int j = 0; j < T_TILE; ++j)
+              for (int j = 0; j < T_HALF; ++j)
                 if ((j & 15) >= thr[j >> 4]) sc[j] = -INFINITY;
             }
             float mx[4] = {sc[0], sc[1], sc[2], sc[3]};
 #pragma unroll
-            for (int j = 4; j < T_TILE; j += 4) {
+            for (int j = 4; j < T_HALF; j += 4) {
               mx[0] = fmaxf(mx[0], sc[j]); mx[1] = fmaxf(mx[1], sc[j + 1]);
               mx[2] = fmaxf(mx[2], sc[j + 2]); mx[3] = fmaxf(mx[3], sc[j + 3]);
             }
             const float mt = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * a.scale_log2;
             const bool need = mt > m_ref + 8.f;       // also true for the first visible tile (m_ref = -inf)
             const bool rescale = need && l > 0.f;
-            // this group's previous tile is it - 2: its P.V must be done before P[b] is overwritten or O[b] rescaled
-            if (it >= 2 && !wait_or_abort(bar + 8 * (B_PVDONE + b), ((it - 2) >> 1) & 1, abort_flag)) { ok = false; break; }
             if (__any_sync(0xffffffffu, rescale)) {
-              // O[b] and l are relative to m_ref: move them to the new reference
+              // O_g and l are relative to m_ref: move them to the new reference.  The accumulator is quiet once the
+              // P.V of the previous tile has finished, which is what releases that tile's stage.
+              if (!wait_or_abort(bar + 8 * (B_EMPTY + (it - 1) % T_STAGES), ((it - 1) / T_STAGES) & 1, abort_flag)) { ok = false; break; }
               tc_fence_after();
               const float f = rescale ? fast_exp2(m_ref - mt) : 1.f;
 #pragma unroll 1
@@ -443,9 +449,9 @@ attn_tensor_kernel(PoolView pv, TensorArgs a, const __nv_bfloat16 *__restrict__ 
             if (need) m_ref = mt;
             const float ref = (m_ref == -INFINITY) ? 0.f : m_ref;
             float ls[4] = {0.f, 0.f, 0.f, 0.f};
-            uint32_t pk[T_TILE / 2];
+            uint32_t pk[T_HALF / 2];
 #pragma unroll
-            for (int j = 0; j < T_TILE; j += 4) {
+            for (int j = 0; j < T_HALF; j += 4) {
               const float p0 = fast_exp2(fmaf(sc[j], a.scale_log2, -ref));
               const float p1 = fast_exp2(fmaf(sc[j + 1], a.scale_log2, -ref));
               const float p2 = fast_exp2(fmaf(sc[j + 2], a.scale_log2, -ref));
@@ -455,11 +461,11 @@ attn_tensor_kernel(PoolView pv, TensorArgs a, const __nv_bfloat16 *__restrict__ 
               pk[(j >> 1) + 1] = pack_bf16(p2, p3);
             }
             l += (ls[0] + ls[1]) + (ls[2] + ls[3]);
-            tmem_st32_u32(tmem + lane_addr + COL_P + b * 32, pk);
+            tmem_st32_u32(tmem + lane_addr + col_s, pk);      // P takes the place of the first 32 score columns
             tmem_st_wait();
           }
           tc_fence_before();
-          mbar_arrive(bar + 8 * (B_PFULL + b));
+          mbar_arrive(bar + 8 * (B_PFULL + 2 * b + grp));
         }
         if (!ok) break;
         // ---- epilogue: the unit's rows leave TMEM; group 0 folds group 1's accumulator into its own

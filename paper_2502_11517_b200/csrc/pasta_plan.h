@@ -20,7 +20,7 @@
 #include <cstdint>
 
 #define PASTA_PLAN_MAGIC 0x50415354
-#define PASTA_TILE_PAGES 4          // pages per tensor-core tile (64 tokens)
+#define PASTA_TILE_PAGES 8          // pages per tensor-core tile (128 tokens)
 #define PASTA_PAGE 16               // tokens per page
 #define PASTA_MAX_ROWS 128          // rows of the stacked-query matrix (threads * group)
 

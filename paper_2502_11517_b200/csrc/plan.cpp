@@ -157,8 +157,8 @@ pasta_status_t build_plan(const HostPool &pool, const std::vector<StepEntry> &en
     // Every tile has a position on a cost axis (tiles, plus `overhead` at the start of each (t-request, kv head)
     // run); CTA c owns positions [c, c + 1) * total / grid.  Positions are absolute, so rounding at one cut does
     // not move the others.  Cuts that would leave fewer than `min_piece` tiles on one side snap to the run's end.
-    const double overhead = 2.0;
-    const int32_t min_piece = 2;
+    const double overhead = 1.0;
+    const int32_t min_piece = 1;
     double total = 0;
     for (const TReq &t : treqs)
       total += lim.n_kv_heads * ((t.n_pages + PASTA_TILE_PAGES - 1) / PASTA_TILE_PAGES + overhead);

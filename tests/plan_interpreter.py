@@ -8,7 +8,7 @@ import numpy as np
  PH_OFF_APPEND, PH_OFF_QUERY, PH_OFF_TREQ, PH_OFF_TRANGE, PH_OFF_TUNIT, PH_OFF_TCTA, PH_OFF_WUNIT, PH_OFF_PAGES,
  PH_OFF_PMETA, PH_OFF_VIS, PH_OFF_TQ, PH_TOTAL_WORDS) = range(21)
 PQ, PT, PU, PW = 4, 6, 5, 4
-TILE_PAGES, PAGE = 4, 16
+TILE_PAGES, PAGE = 8, 16
 
 
 def run_plan(w, K, V, q, n_kv_heads):
