@@ -383,10 +383,11 @@ attn_tensor_kernel(PoolView pv, TensorArgs a, const __nv_bfloat16 *__restrict__ 
         const int32_t *visrow = plan + a.off_vis + x.vis_off + (active ? row / G : 0) * x.n_streams;
         // the row's visible lengths of the first four local streams stay in registers for the whole unit: a global
         // load per page would otherwise sit between two tiles of this group
-        const int vis0 = visrow[0];
-        const int vis1 = x.n_streams > 1 ? visrow[1] : 0;
-        const int vis2 = x.n_streams > 2 ? visrow[2] : 0;
-        const int vis3 = x.n_streams > 3 ? visrow[3] : 0;
+        int vis0 = visrow[0];
+        int vis1 = x.n_streams > 1 ? visrow[1] : 0;
+        int vis2 = x.n_streams > 2 ? visrow[2] : 0;
+        int vis3 = x.n_streams > 3 ? visrow[3] : 0;
+        asm volatile("" : "+r"(vis0), "+r"(vis1), "+r"(vis2), "+r"(vis3));   // loaded here, once, not again at each use
         float m_ref = -INFINITY, l = 0.f;
         for (int k = 0; k < nt; ++k, ++it) {
           const uint32_t s = it % T_STAGES, b = it & 1;
@@ -396,9 +397,11 @@ attn_tensor_kernel(PoolView pv, TensorArgs a, const __nv_bfloat16 *__restrict__ 
           int thr[T_HALF_PAGES];
           bool full = true;
           if (warp_active) {
+            const int4 m4 = *reinterpret_cast<const int4 *>(meta_s + s * PASTA_TILE_PAGES + grp * T_HALF_PAGES);
+            const int metas[T_HALF_PAGES] = {m4.x, m4.y, m4.z, m4.w};
 #pragma unroll
             for (int pg = 0; pg < T_HALF_PAGES; ++pg) {
-              const int meta = meta_s[s * PASTA_TILE_PAGES + grp * T_HALF_PAGES + pg];
+              const int meta = metas[pg];
               int t = 0;
               if (active && meta >= 0) {
                 const int sl = meta & 255;
