@@ -36,7 +36,7 @@ NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 # dram bytes (read + write) of one launch of the dominant kernel from an ncu capture of this workload,
 # or None when no capture matches the current kernel
-NCU_TRAFFIC_BYTES = {"long_shared_prefix": 1.092e9, "batched": None, "single_request": None}   # see profiles/
+NCU_TRAFFIC_BYTES = {("long_shared_prefix", "full"): 1.092e9, ("long_shared_prefix", "small"): 2.765e8}   # see profiles/
 
 
 def make_script(workload: str, size: str = "full"):
@@ -46,7 +46,10 @@ def make_script(workload: str, size: str = "full"):
     if workload == "batched":
         return cfg3_batched() if size == "full" else cfg3_batched(n_layers=4)
     if workload == "single_request":
-        return cfg2_single_request("a")
+        script = cfg2_single_request("a")
+        last = next(i for i, op in enumerate(script.ops) if op[0] == "step")
+        script.ops = script.ops[:last + 1]          # step A: four forks and the main thread
+        return script
     raise SystemExit(f"unknown workload {workload}")
 
 
@@ -313,7 +316,7 @@ def run_ours(args):
         "gpu_launches": launches,
         "roofline": {"bound": "hbm", "kernel": dom_name, "achieved": achieved, "peak": peak, "peak_kind": peak_kind,
                      "unit": "GB/s", "frac": achieved / peak, "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
-                     "traffic": NCU_TRAFFIC_BYTES.get(args.workload), "bytes_per_launch": dom_bytes_per_launch,
+                     "traffic": NCU_TRAFFIC_BYTES.get((args.workload, args.size)) if dom == 0 else None, "bytes_per_launch": dom_bytes_per_launch,
                      "ms_per_launch": dom_ms},
         "cpu_baseline": oracle_sample(args.workload, budget_s=20.0) if world == 1 and not args.no_cpu_baseline else None,
     }
@@ -347,11 +350,14 @@ def oracle_sample(workload: str, budget_s: float = 20.0, steps: int = 1):
     from oracle import OracleReplay
     from pasta_workloads import cfg2_single_request, cfg3_batched, cfg4_long_prefix
     if workload == "long_shared_prefix":
-        script = cfg4_long_prefix(n_requests=1); sample = "the 17 thread-tokens of 1 of 8 requests (32768-token prefix, 16 forks), 1 layer"
+        script = cfg4_long_prefix(n_requests=1); steps = max(steps, 4)
+        sample = "the 17 thread-tokens of 1 of 8 requests (32768-token prefix, 16 forks), 1 layer, 4 passes"
     elif workload == "batched":
-        script = cfg3_batched(n_requests=8, n_layers=1); sample = "the thread-tokens of the first 8 of 64 requests, 1 of 32 layers (time scaled by 32 layers)"
+        script = cfg3_batched(n_layers=1); steps = max(steps, 8)
+        sample = "all thread-tokens of the 64 requests, 1 of 32 layers, 8 passes (time scaled by 32 layers)"
     else:
-        script = cfg2_single_request("a"); script.ops = script.ops[:11]; sample = "step A: 5 thread-tokens of the request, 1 layer"
+        script = cfg2_single_request("a"); script.ops = script.ops[:11]; steps = max(steps, 50)
+        sample = "step A: 5 thread-tokens of the request, 1 layer, 50 passes"
     rep = OracleReplay(script)
     last = len(script.ops) - 1
     for i in range(last):
@@ -372,9 +378,11 @@ def oracle_sample(workload: str, budget_s: float = 20.0, steps: int = 1):
         for i, qq in enumerate(queries):
             decode_attention(rep.model, rep.stores[0], [qq], q[i:i + 1])
             done += 1
-            if time.perf_counter() - t_all > budget_s and steps == 1:
+            if time.perf_counter() - t_all > budget_s:
                 break
         times.append((time.perf_counter() - t0, done))
+        if time.perf_counter() - t_all > budget_s:
+            break
     dt = sum(t for t, _ in times); done = sum(d for _, d in times)
     layers = 32 if workload == "batched" else 1
     try:
