@@ -12,6 +12,9 @@ Workloads (synthetic, seeded; shapes of the five configurations):
   long_shared_prefix  8 requests x 32768-token prefix x 16 forks (chunks U[50,400]), 1 layer      [default]
   batched             64 requests, prefix U[256,2048], forks geometric, chunks U[10,300], 32 layers
   single_request      1 request, 768-token prefix, 4 forks, 1 layer (cache resident: a latency case)
+  trace               synthetic interpreter trace (cfg5): 256 requests x 32 layers, promises / forks / syncs as they
+                      come; every op of the trace is executed (step plan, append, attention, spawn, finish, sync merge);
+                      --steps decode steps are timed after --warmup untimed ones (--size small: 64 requests x 8 layers)
 With N > 1 (torchrun) every rank runs its own copy of the workload on its own GPU: requests are
 independent, there is no exchange between ranks ("weak" scaling).
 """
@@ -325,6 +328,142 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+def unique_tokens_per_step(script):
+    """Bookkeeping-only replay (a host-only pool): unique visible tokens of every step of a trace script."""
+    from paper_2502_11517_b200 import binding
+    geo = script.geometry
+    pool = binding.Pool(1, geo.n_q_heads, geo.n_kv_heads, geo.head_dim, script.n_pages, script.max_requests,
+                        script.max_threads_per_request, script.max_segments_per_thread, free_order=script.free_order,
+                        flags=binding.FLAG_HOST_ONLY)
+    lens, seen_by = {}, {}      # (req, stream) -> length; req -> set of streams somebody of the request can see
+    out = []
+    for op in script.ops:
+        kind = op[0]
+        if kind == "begin":
+            pool.request_begin(); lens[(op[1], 0)] = 0; seen_by[op[1]] = {0}
+        elif kind == "run":
+            pool.kv_append_run(op[1], op[2], op[3]); lens[(op[1], op[2])] = lens.get((op[1], op[2]), 0) + op[3]
+        elif kind == "spawn":
+            pool.thread_spawn(op[1]); lens[(op[1], op[2])] = 0
+        elif kind == "finish":
+            pool.thread_finish(op[1], op[2])
+        elif kind == "merge":
+            pool.sync_merge(op[1], None if op[2] is None else list(op[2])); seen_by[op[1]].update(op[2] or [])
+        elif kind == "step":
+            total = 0
+            reqs = {}
+            for r, t, n in op[1]:
+                lens[(r, t)] += n
+                reqs.setdefault(r, set()).add(t)
+            for r, ts in reqs.items():
+                total += sum(lens[(r, st)] for st in (seen_by[r] | ts))
+            out.append(total)
+    pool.close()
+    return out
+
+
+def run_trace(args):
+    import torch
+    from paper_2502_11517_b200 import binding
+    from paper_2502_11517_b200.build import build
+    from paper_2502_11517_b200.sharding import aggregate
+    from pasta_workloads import cfg5_trace
+    import torch.distributed as dist
+    rank = int(os.environ.get("RANK", "0")); world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    if rank == 0:
+        build()
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local)); dist.barrier()
+    device = torch.device("cuda", local); torch.cuda.set_device(device)
+    warm = max(args.warmup, 3)
+    n_req, n_layers = (256, 32) if args.size == "full" else (64, 8)
+    script = cfg5_trace(n_requests=n_req, n_steps=args.steps + warm, n_layers=n_layers)
+    geo = script.geometry
+    uniq = unique_tokens_per_step(script)
+    max_n = max(len(op[1]) for op in script.ops if op[0] == "step")
+    pool = binding.Pool(geo.n_layers, geo.n_q_heads, geo.n_kv_heads, geo.head_dim, script.n_pages, script.max_requests,
+                        script.max_threads_per_request, script.max_segments_per_thread, free_order=script.free_order,
+                        max_step_queries=max_n, max_layers_per_launch=min(8, geo.n_layers), device=local)
+    gen = torch.Generator(device=device); gen.manual_seed(script.seed + 977 * rank)
+
+    def randn(shape):
+        return torch.randn(shape, generator=gen, device=device, dtype=torch.float32).to(torch.bfloat16)
+
+    L = geo.n_layers
+    kv_pool = randn((L * max_n * geo.n_kv_heads * geo.head_dim,)); kv_pool2 = randn(kv_pool.shape)
+    q_pool = randn((L * max_n * geo.n_q_heads * geo.head_dim,))
+    out = torch.empty((L * max_n * geo.n_q_heads * geo.head_dim,), dtype=torch.float32, device=device)
+    stream = torch.cuda.current_stream(device)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    step_i = 0; tokens = 0; bytes_ = 0.0; merges = 0; host_s = 0.0
+    t_wall0 = t_wall1 = None; sampler = None; launches0 = 0
+    for op in script.ops:
+        kind = op[0]
+        if kind == "begin":
+            assert pool.request_begin() == op[1]
+        elif kind == "run":
+            done = 0
+            while done < op[3]:
+                cnt = min(op[3] - done, 2048)
+                shape = (L, cnt, geo.n_kv_heads, geo.head_dim)
+                pool.kv_append_run(op[1], op[2], cnt, randn(shape), randn(shape)); done += cnt
+        elif kind == "spawn":
+            assert pool.thread_spawn(op[1]) == op[2]
+        elif kind == "finish":
+            pool.thread_finish(op[1], op[2])
+        elif kind == "merge":
+            pool.sync_merge(op[1], None if op[2] is None else list(op[2])); merges += step_i >= warm
+        elif kind == "step":
+            if step_i == warm:
+                torch.cuda.synchronize(device)
+                if world > 1:
+                    dist.barrier()
+                launches0 = pool.launch_count()
+                sampler = ClockSampler(local) if rank == 0 else None
+                t_wall0 = time.time(); ev0.record(stream)
+            n = len(op[1])
+            h0 = time.perf_counter()
+            pool.step_begin([e[0] for e in op[1]], [e[1] for e in op[1]], [e[2] for e in op[1]])
+            host_s += (time.perf_counter() - h0) if step_i >= warm else 0.0
+            kn = kv_pool[:L * n * geo.n_kv_heads * geo.head_dim]; vn = kv_pool2[:kn.numel()]
+            pool.kv_append(kn, vn)
+            pool.decode_attn(q_pool[:L * n * geo.n_q_heads * geo.head_dim], out)
+            if step_i >= warm:
+                tokens += n; bytes_ += uniq[step_i] * geo.kv_bytes_per_token * L
+            step_i += 1
+    ev1.record(stream); torch.cuda.synchronize(device); t_wall1 = time.time()
+    if world > 1:
+        dist.barrier()
+    ms = ev0.elapsed_time(ev1)
+    clocks = sampler.stop(t_wall0, t_wall1) if sampler else None
+    launches = pool.launch_count() - launches0
+    assert pool.status() == 0, "a kernel reported an error"
+    all_tokens, worst_s = aggregate(float(tokens), ms * 1e-3)
+    if rank == 0:
+        peak, peak_kind = measured_peak()
+        gbs = bytes_ / (ms * 1e-3) / 1e9
+        print(json.dumps({
+            "metric": METRIC, "value": all_tokens / worst_s, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": warm,
+            "ms_per_step": worst_s * 1e3 / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": "trace", "size": args.size, "script": script.name, "requests": n_req, "layers": L,
+                       "thread_tokens_timed": tokens, "max_thread_tokens_per_step": max_n, "sync_merges_timed": int(merges),
+                       "pool_pages": script.n_pages, "pool_gb": script.n_pages * 65536 * L / 1e9,
+                       "unique_kv_bytes_timed": bytes_, "l2": "inputs larger than L2",
+                       "step_hbm_gbs": gbs, "step_frac_of_measured_peak": gbs / peak, "step_frac_of_nominal_8TBs": gbs / NOMINAL_HBM_GBS,
+                       "step_begin_call_ms": host_s * 1e3 / args.steps,
+                       "step_begin_note": "wall time inside pasta_step_begin; includes waiting for the device when the host runs ahead"},
+            "clocks": clocks, "e2e": None, "gpu_launches": launches,
+            "roofline": {"bound": "hbm", "kernel": "whole step (tensor + warp + merge + append)", "achieved": gbs, "peak": peak,
+                         "peak_kind": peak_kind, "unit": "GB/s", "frac": gbs / peak, "traffic": None},
+            "cpu_baseline": None}))
+    if world > 1:
+        dist.destroy_process_group()
+
+
 def time_sync_merge():
     from paper_2502_11517_b200 import binding
     best = None
@@ -433,6 +572,8 @@ def main():
         if args.steps == 200:
             args.steps, args.warmup = 3, 1
         run_reference(args)
+    elif args.workload == "trace":
+        run_trace(args)
     else:
         run_ours(args)
 
