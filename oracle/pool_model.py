@@ -26,6 +26,13 @@ What the paper leaves open, and the reading taken here:
     main-stream piece ending at p (splitting a piece if p is inside one), after chunks already
     placed at the same p with a smaller thread id and before those with a larger one;
   * only the main thread spawns; merging an unfinished fork is an error (the interpreter waits).
+
+Position ids (Section 4, "Training a PASTA-SFT model", and Section 6 "Positional Embedding"): the main thread
+cannot know how long an asynchronous block will be, so it skips ahead by the length PREDICTED in the promise:
+a fork's first token takes the position right after its <promise/>, the main thread's next token takes that
+position plus the predicted length.  Positions are never revised: if a chunk turns out longer than predicted,
+its ids run into the ids the main thread used after the promise (not monotone after sync); if shorter, a gap
+stays.  How the prediction is made (fixed 40, exact, multiples of ten, ground truth) is the caller's business.
 """
 from __future__ import annotations
 
@@ -50,6 +57,7 @@ class _Request:
         # a view is a list of [stream, start, length, anchor]; anchor = cut-off of a merged chunk, -1 for main pieces
         self.view: Dict[int, List[List[int]]] = {0: []}
         self.next_thread = 1
+        self.pos_next: Dict[int, int] = {0: 0}             # thread id -> position id of the thread's next token
 
 
 class PoolModel:
@@ -81,9 +89,12 @@ class PoolModel:
                 self.free.insert(0, page)
         del self.requests[req]
 
-    def thread_spawn(self, req: int) -> int:
-        """<promise/>: the new fork sees what the main thread sees right now, and nothing later."""
+    def thread_spawn(self, req: int, predicted_tokens: int = 0) -> int:
+        """<promise/>: the new fork sees what the main thread sees right now, and nothing later.  Its first token
+        takes the position after the promise; the main thread skips `predicted_tokens` positions."""
         r = self._req(req)
+        if predicted_tokens < 0:
+            raise PoolError(INVALID_ARG, "negative predicted length")
         t = r.next_thread
         if t >= self.max_threads:
             raise PoolError(CAPACITY, "too many threads")
@@ -93,6 +104,8 @@ class PoolModel:
         r.state[t] = ACTIVE
         r.cutoff[t] = r.stream_len[0]
         r.view[t] = [list(e) for e in r.view[0]]
+        r.pos_next[t] = r.pos_next[0]
+        r.pos_next[0] += predicted_tokens
         return t
 
     def thread_finish(self, req: int, thread: int) -> None:
@@ -154,6 +167,7 @@ class PoolModel:
             r.stream_pages[stream].append(self.free.pop(0))
         slot = (r.stream_pages[stream][k // self.page_size], k % self.page_size)
         r.stream_len[stream] = k + 1
+        r.pos_next[thread] += 1
         view = r.view[thread]
         if view and view[-1][0] == stream and view[-1][1] + view[-1][2] == k:
             view[-1][2] += 1
@@ -214,6 +228,10 @@ class PoolModel:
             out.extend((pages[k // self.page_size], k % self.page_size) for k in range(a, a + n))
         return out
 
+    def last_position(self, req: int, thread: int) -> int:
+        """Position id of the thread's newest token (the one a decode step's query belongs to)."""
+        return self._req(req).pos_next[thread] - 1
+
     def dump(self) -> dict:
         """Whole bookkeeping state in a canonical form."""
         reqs = {}
@@ -221,7 +239,7 @@ class PoolModel:
             r = self.requests[req]
             reqs[req] = {
                 "streams": {s: {"len": r.stream_len[s], "pages": list(r.stream_pages[s])} for s in sorted(r.stream_len)},
-                "threads": {t: {"state": r.state[t], "cutoff": r.cutoff[t],
+                "threads": {t: {"state": r.state[t], "cutoff": r.cutoff[t], "pos_next": r.pos_next[t],
                                 "view": [(s, a, n) for s, a, n, _ in r.view[t]]} for t in sorted(r.state)},
             }
         return {"requests": reqs, "free": list(self.free)}
