@@ -98,6 +98,18 @@ pasta_status_t pasta_request_end(pasta_pool_t *pool, int32_t req);
 /* <promise/>: a fork whose view is the main thread's view at this moment (call it after the promise
  * token was appended), followed by its own chunk.  Forks are numbered 1, 2, 3, … per request. */
 pasta_status_t pasta_thread_spawn(pasta_pool_t *pool, int32_t req, int32_t *out_thread);
+/*
+ * <promise/> with a length prediction (Section 4 "Training a PASTA-SFT model" and Section 6 "Positional
+ * Embedding": the main thread cannot know how long the asynchronous block will be, so it assigns position
+ * ids past the promise as if the block had the predicted length).  Like pasta_thread_spawn, and also:
+ * the fork's first token takes the position id right after the promise token, the main thread's next token
+ * takes that id plus predicted_tokens (>= 0; e.g. 10 x the promise's `tokens` attribute for the paper's
+ * Pred-10X scheme, 40 for Fixed-40).  Ids are never revised: a chunk longer than predicted runs into ids
+ * the main thread has used (not monotone after sync), a shorter one leaves a gap.
+ * pasta_thread_spawn is the same with predicted_tokens = 0.
+ */
+pasta_status_t pasta_thread_spawn_predicted(pasta_pool_t *pool, int32_t req, int32_t predicted_tokens,
+                                            int32_t *out_thread);
 /* </async>: the fork decodes no more; its chunk stays invisible to the main thread until merged. */
 pasta_status_t pasta_thread_finish(pasta_pool_t *pool, int32_t req, int32_t thread);
 
@@ -131,6 +143,21 @@ pasta_status_t pasta_step_begin(pasta_pool_t *pool, int32_t n, const int32_t *re
  * entry, (-1, -1) for entries with n_new == 0.  Host array of 2 * n entries. */
 pasta_status_t pasta_step_slots(pasta_pool_t *pool, int32_t *out_slots, int32_t capacity_entries);
 
+/* Position id of each entry's newest token (the one its query belongs to) for the last pasta_step_begin.
+ * Host array of n entries. */
+pasta_status_t pasta_step_positions(pasta_pool_t *pool, int32_t *out_pos, int32_t capacity_entries);
+
+/*
+ * pasta_kv_append with rotary position embedding fused in: every new K vector is rotated by its token's
+ * position id before it is stored (rotate-half form: element i pairs with element i + head_dim/2,
+ * angle = position * theta^(-2i/head_dim), angles evaluated in double precision, result rounded to bf16);
+ * V is copied unchanged.  theta > 1 (10000 for the usual base).
+ */
+pasta_status_t pasta_kv_append_rope(pasta_pool_t *pool, int32_t layer_begin, int32_t layer_count,
+                                    const void *k_new, const void *v_new, float theta, void *stream);
+/* Rotates the step's queries in place by the same rule: q device bf16 [layer_count, n, n_q_heads, head_dim]. */
+pasta_status_t pasta_rope_queries(pasta_pool_t *pool, int32_t layer_count, void *q, float theta, void *stream);
+
 /*
  * Copies the new tokens' K and V into their reserved slots for layers
  * [layer_begin, layer_begin + layer_count).  k_new, v_new: device bf16
@@ -163,6 +190,12 @@ pasta_status_t pasta_decode_attn(pasta_pool_t *pool, int32_t layer_begin, int32_
 pasta_status_t pasta_kv_append_run(pasta_pool_t *pool, int32_t req, int32_t thread, int32_t m,
                                    int32_t layer_begin, int32_t layer_count,
                                    const void *k, const void *v, void *stream);
+
+/* pasta_kv_append_run with the rotary embedding of pasta_kv_append_rope (consecutive position ids from the
+ * thread's next one). */
+pasta_status_t pasta_kv_append_run_rope(pasta_pool_t *pool, int32_t req, int32_t thread, int32_t m,
+                                        int32_t layer_begin, int32_t layer_count, const void *k, const void *v,
+                                        float theta, void *stream);
 
 /*
  * One whole step with HOST tensors: step_begin, copy k_new / v_new / q to the device, kv_append
@@ -214,7 +247,7 @@ pasta_status_t pasta_kv_read(pasta_pool_t *pool, int32_t layer, int32_t req, int
  * Serialises the bookkeeping state into host int32 words:
  *   n_requests, then per live request (ascending id):
  *     req, n_streams, per stream (ascending id): stream, len, n_pages, page ids…
- *     n_threads, per thread (ascending id): thread, state, cutoff, n_segments, (stream, start, len)…
+ *     n_threads, per thread (ascending id): thread, state, cutoff, next position id, n_segments, (stream, start, len)…
  *   n_free, free page ids in hand-out order.
  * *needed receives the number of words; nothing is written when capacity_words is too small
  * (the call then still returns PASTA_OK so that the size can be queried with host_buf == NULL).

@@ -25,6 +25,8 @@ EXPORTS = [
     "pasta_kv_append_run", "pasta_step_host_bytes", "pasta_step_host", "pasta_kv_read",
     "pasta_pool_dump", "pasta_plan_dump", "pasta_pool_status", "pasta_launch_count",
     "pasta_profile_enable", "pasta_profile_read", "pasta_decode_attn_noalloc",
+    "pasta_thread_spawn_predicted", "pasta_step_positions", "pasta_kv_append_rope", "pasta_rope_queries",
+    "pasta_kv_append_run_rope",
     "pasta_last_cuda_error",
 ]
 
@@ -155,6 +157,12 @@ class Pool:
         _check(lib().pasta_thread_spawn(self._h, req, C.byref(out)), "pasta_thread_spawn")
         return out.value
 
+    def thread_spawn_predicted(self, req: int, predicted_tokens: int) -> int:
+        out = C.c_int32()
+        _check(lib().pasta_thread_spawn_predicted(self._h, req, predicted_tokens, C.byref(out)),
+               "pasta_thread_spawn_predicted")
+        return out.value
+
     def thread_finish(self, req: int, thread: int) -> None:
         _check(lib().pasta_thread_finish(self._h, req, thread), "pasta_thread_finish")
 
@@ -177,6 +185,27 @@ class Pool:
         out = np.empty((self._last_n, 2), dtype=np.int32)
         _check(lib().pasta_step_slots(self._h, _ptr(out), self._last_n), "pasta_step_slots")
         return out
+
+    def step_positions(self) -> np.ndarray:
+        out = np.empty(self._last_n, dtype=np.int32)
+        _check(lib().pasta_step_positions(self._h, _ptr(out), self._last_n), "pasta_step_positions")
+        return out
+
+    def kv_append_rope(self, k_new, v_new, theta: float = 10000.0, layer_begin: int = 0,
+                       layer_count: Optional[int] = None, stream=None) -> None:
+        cnt = self.n_layers - layer_begin if layer_count is None else layer_count
+        _check(lib().pasta_kv_append_rope(self._h, layer_begin, cnt, _dev(k_new), _dev(v_new), C.c_float(theta),
+                                          _stream(stream)), "pasta_kv_append_rope")
+
+    def rope_queries(self, q, theta: float = 10000.0, layer_count: Optional[int] = None, stream=None) -> None:
+        cnt = self.n_layers if layer_count is None else layer_count
+        _check(lib().pasta_rope_queries(self._h, cnt, _dev(q), C.c_float(theta), _stream(stream)), "pasta_rope_queries")
+
+    def kv_append_run_rope(self, req: int, thread: int, m: int, k, v, theta: float = 10000.0, layer_begin: int = 0,
+                           layer_count: Optional[int] = None, stream=None) -> None:
+        cnt = self.n_layers - layer_begin if layer_count is None else layer_count
+        _check(lib().pasta_kv_append_run_rope(self._h, req, thread, m, layer_begin, cnt, _dev(k), _dev(v),
+                                              C.c_float(theta), _stream(stream)), "pasta_kv_append_run_rope")
 
     def kv_append(self, k_new, v_new, layer_begin: int = 0, layer_count: Optional[int] = None, stream=None) -> None:
         cnt = self.n_layers - layer_begin if layer_count is None else layer_count
@@ -254,8 +283,8 @@ class Pool:
                 streams[sid] = {"len": ln, "pages": take(npg)}
             threads = {}
             for _t in range(take()[0]):
-                tid, state, cutoff, nseg = take(4)
-                threads[tid] = {"state": state, "cutoff": cutoff,
+                tid, state, cutoff, pos_next, nseg = take(5)
+                threads[tid] = {"state": state, "cutoff": cutoff, "pos_next": pos_next,
                                 "view": [tuple(take(3)) for _k in range(nseg)]}
             reqs[req] = {"streams": streams, "threads": threads}
         free = take(take()[0])

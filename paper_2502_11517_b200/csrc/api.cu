@@ -265,7 +265,49 @@ pasta_status_t pasta_request_end(pasta_pool_t *p, int32_t req) {
 
 pasta_status_t pasta_thread_spawn(pasta_pool_t *p, int32_t req, int32_t *out_thread) {
   if (!p || !out_thread) return PASTA_ERR_INVALID_ARG;
-  return p->host.thread_spawn(req, out_thread);
+  return p->host.thread_spawn(req, 0, out_thread);
+}
+
+pasta_status_t pasta_thread_spawn_predicted(pasta_pool_t *p, int32_t req, int32_t predicted_tokens, int32_t *out_thread) {
+  if (!p || !out_thread) return PASTA_ERR_INVALID_ARG;
+  return p->host.thread_spawn(req, predicted_tokens, out_thread);
+}
+
+pasta_status_t pasta_step_positions(pasta_pool_t *p, int32_t *out_pos, int32_t capacity_entries) {
+  if (!p || !out_pos) return PASTA_ERR_INVALID_ARG;
+  if (!p->plan_valid) return PASTA_ERR_BAD_STATE;
+  const int32_t n = p->hdr.w[PH_N_QUERIES];
+  if (capacity_entries < n) return PASTA_ERR_CAPACITY;
+  std::memcpy(out_pos, p->plan.data() + p->hdr.w[PH_OFF_QPOS], size_t(n) * 4);
+  return PASTA_OK;
+}
+
+pasta_status_t pasta_kv_append_rope(pasta_pool_t *p, int32_t layer_begin, int32_t layer_count, const void *k_new,
+                                    const void *v_new, float theta, void *stream) {
+  if (!p) return PASTA_ERR_INVALID_ARG;
+  if (p->host_only || !p->plan_valid) return PASTA_ERR_BAD_STATE;
+  if (layer_begin < 0 || layer_count < 0 || layer_begin + layer_count > p->cfg.n_layers || !(theta > 1.f))
+    return PASTA_ERR_INVALID_ARG;
+  const int32_t n_app = p->hdr.w[PH_N_APPEND];
+  if (n_app == 0 || layer_count == 0) return PASTA_OK;
+  if (!k_new || !v_new) return PASTA_ERR_INVALID_ARG;
+  PASTA_CUDA(launch_kv_append_rope(p->pv, p->pv.plan + p->hdr.w[PH_OFF_APPEND], p->pv.plan + p->hdr.w[PH_OFF_APOS], 0, n_app,
+                                   layer_begin, layer_count, k_new, v_new, theta, static_cast<cudaStream_t>(stream)));
+  p->launches += 1;
+  return PASTA_OK;
+}
+
+pasta_status_t pasta_rope_queries(pasta_pool_t *p, int32_t layer_count, void *q, float theta, void *stream) {
+  if (!p) return PASTA_ERR_INVALID_ARG;
+  if (p->host_only || !p->plan_valid) return PASTA_ERR_BAD_STATE;
+  if (layer_count < 0 || layer_count > p->cfg.n_layers || !(theta > 1.f)) return PASTA_ERR_INVALID_ARG;
+  const int32_t n = p->hdr.w[PH_N_QUERIES];
+  if (n == 0 || layer_count == 0) return PASTA_OK;
+  if (!q) return PASTA_ERR_INVALID_ARG;
+  PASTA_CUDA(launch_rope_queries(p->pv, p->pv.plan + p->hdr.w[PH_OFF_QPOS], n, layer_count, q, theta,
+                                 static_cast<cudaStream_t>(stream)));
+  p->launches += 1;
+  return PASTA_OK;
 }
 
 pasta_status_t pasta_thread_finish(pasta_pool_t *p, int32_t req, int32_t thread) {
@@ -379,13 +421,15 @@ pasta_status_t pasta_decode_attn(pasta_pool_t *p, int32_t layer_begin, int32_t l
   return PASTA_OK;
 }
 
-pasta_status_t pasta_kv_append_run(pasta_pool_t *p, int32_t req, int32_t thread, int32_t m, int32_t layer_begin,
-                                   int32_t layer_count, const void *k, const void *v, void *stream) {
+static pasta_status_t append_run_impl(pasta_pool_t *p, int32_t req, int32_t thread, int32_t m, int32_t layer_begin,
+                                      int32_t layer_count, const void *k, const void *v, float theta, void *stream) {
   if (!p) return PASTA_ERR_INVALID_ARG;
   if (layer_begin < 0 || layer_count < 0 || layer_begin + layer_count > p->cfg.n_layers) return PASTA_ERR_INVALID_ARG;
   if (layer_count > 0 && p->host_only) return PASTA_ERR_BAD_STATE;
   if (layer_count > 0 && m > 0 && (!k || !v)) return PASTA_ERR_INVALID_ARG;
   std::vector<Slot> slots;
+  const Request *rq = p->host.request(req);
+  const int32_t pos0 = (rq && thread >= 0 && thread < static_cast<int32_t>(rq->threads.size())) ? rq->threads[thread].pos_next : 0;
   pasta_status_t s = p->host.reserve_run(req, thread, m, &slots);
   if (s != PASTA_OK) return s;
   p->plan_valid = false;
@@ -402,11 +446,25 @@ pasta_status_t pasta_kv_append_run(pasta_pool_t *p, int32_t req, int32_t thread,
     for (int32_t l = 0; l < layer_count; ++l) {     // the run's layers are [layer_count, m, …]: one launch per layer and chunk
       const uint16_t *kl = static_cast<const uint16_t *>(k) + (size_t(l) * m + begin) * tok;
       const uint16_t *vl = static_cast<const uint16_t *>(v) + (size_t(l) * m + begin) * tok;
-      PASTA_CUDA(launch_kv_append(p->pv, p->run_slots_dev, cnt, layer_begin + l, 1, kl, vl, st));
+      if (theta > 0.f)
+        PASTA_CUDA(launch_kv_append_rope(p->pv, p->run_slots_dev, nullptr, pos0 + begin, cnt, layer_begin + l, 1, kl, vl, theta, st));
+      else
+        PASTA_CUDA(launch_kv_append(p->pv, p->run_slots_dev, cnt, layer_begin + l, 1, kl, vl, st));
       p->launches += 1;
     }
   }
   return PASTA_OK;
+}
+
+pasta_status_t pasta_kv_append_run(pasta_pool_t *p, int32_t req, int32_t thread, int32_t m, int32_t layer_begin,
+                                   int32_t layer_count, const void *k, const void *v, void *stream) {
+  return append_run_impl(p, req, thread, m, layer_begin, layer_count, k, v, 0.f, stream);
+}
+
+pasta_status_t pasta_kv_append_run_rope(pasta_pool_t *p, int32_t req, int32_t thread, int32_t m, int32_t layer_begin,
+                                        int32_t layer_count, const void *k, const void *v, float theta, void *stream) {
+  if (!(theta > 1.f)) return PASTA_ERR_INVALID_ARG;
+  return append_run_impl(p, req, thread, m, layer_begin, layer_count, k, v, theta, stream);
 }
 
 pasta_status_t pasta_step_host_bytes(pasta_pool_t *p, int32_t n, size_t *out) {

@@ -18,6 +18,13 @@ cudaError_t launch_kv_append(const PoolView &pv, const int32_t *slots, int32_t n
 // inverse of K1 for one layer: gathers the listed slots into dense [n_tok, Hkv, D] arrays
 cudaError_t launch_kv_read(const PoolView &pv, const int32_t *slots, int32_t n_tok, int32_t layer,
                            void *k_out, void *v_out, cudaStream_t st);
+// K1 with rotary embedding of K by position id (pos: device array, or NULL for consecutive ids pos0, pos0 + 1, ...)
+cudaError_t launch_kv_append_rope(const PoolView &pv, const int32_t *slots, const int32_t *pos, int32_t pos0, int32_t n_tok,
+                                  int32_t layer_begin, int32_t layer_count, const void *k_new, const void *v_new,
+                                  double theta, cudaStream_t st);
+// rotates the step's queries in place by their tokens' position ids
+cudaError_t launch_rope_queries(const PoolView &pv, const int32_t *pos, int32_t n, int32_t layer_count, void *q, double theta,
+                                cudaStream_t st);
 // K3: warp-shuffle pass over streams seen by one query
 cudaError_t launch_attn_warp(const PoolView &pv, const PlanHeader &h, int32_t layer_begin, int32_t layer_count,
                              const void *q, float scale_log2, cudaStream_t st);

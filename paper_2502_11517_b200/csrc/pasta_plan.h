@@ -46,6 +46,8 @@ enum {
   PH_OFF_PMETA,       // parallel to pages (t-request lists only): (page index in its stream << 8) | local stream
   PH_OFF_VIS,         // per t-request: [n_threads][n_streams] visible length of local stream for thread
   PH_OFF_TQ,          // per t-request: [n_threads] query index of each row-thread
+  PH_OFF_APOS,        // position id of every appended token (parallel to the append table)
+  PH_OFF_QPOS,        // position id of every query's token
   PH_TOTAL_WORDS,
   PH_WORDS = 32
 };

@@ -252,9 +252,12 @@ pasta_status_t build_plan(const HostPool &pool, const std::vector<StepEntry> &en
     w.insert(w.end(), v.begin(), v.end());
     while (w.size() % 4) w.push_back(0);   // keep every table 16-byte aligned
   };
-  std::vector<int32_t> app;
-  for (int32_t i = 0; i < n; ++i)
-    if (entries[i].n_new) { app.push_back(slots[i].page); app.push_back(slots[i].offset); }
+  std::vector<int32_t> app, apos, qpos;
+  for (int32_t i = 0; i < n; ++i) {
+    const int32_t pos = pool.request(entries[i].req)->threads[entries[i].thread].pos_next - 1;   // the newest token
+    qpos.push_back(pos);
+    if (entries[i].n_new) { app.push_back(slots[i].page); app.push_back(slots[i].offset); apos.push_back(pos); }
+  }
   std::vector<int32_t> qtab(static_cast<size_t>(n) * PQ_WORDS);
   for (int32_t i = 0; i < n; ++i) {
     qtab[i * PQ_WORDS + PQ_TREQ] = q_treq[i];
@@ -291,6 +294,8 @@ pasta_status_t build_plan(const HostPool &pool, const std::vector<StepEntry> &en
   put(PH_OFF_PMETA, pmeta);
   put(PH_OFF_VIS, vis_tab);
   put(PH_OFF_TQ, tq_tab);
+  put(PH_OFF_APOS, apos);
+  put(PH_OFF_QPOS, qpos);
   w[PH_TOTAL_WORDS] = static_cast<int32_t>(w.size());
   if (static_cast<int64_t>(w.size()) > lim.max_words) return PASTA_ERR_CAPACITY;
   return PASTA_OK;

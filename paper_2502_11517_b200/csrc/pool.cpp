@@ -56,14 +56,16 @@ pasta_status_t HostPool::request_end(int32_t req) {
   return PASTA_OK;
 }
 
-pasta_status_t HostPool::thread_spawn(int32_t req, int32_t *out_thread) {
+pasta_status_t HostPool::thread_spawn(int32_t req, int32_t predicted_tokens, int32_t *out_thread) {
   Request *r = live(req);
-  if (!r) return PASTA_ERR_INVALID_ARG;
+  if (!r || predicted_tokens < 0) return PASTA_ERR_INVALID_ARG;
   int32_t t = static_cast<int32_t>(r->threads.size());
   if (t >= max_threads_) return PASTA_ERR_CAPACITY;
   Thread fork;
   fork.cutoff = r->streams[0].len;
   fork.view = r->threads[0].view;          // frozen snapshot of what the main thread sees now
+  fork.pos_next = r->threads[0].pos_next;  // the fork continues right after the promise ...
+  r->threads[0].pos_next += predicted_tokens;   // ... and the main thread skips the predicted block
   r->threads.push_back(std::move(fork));
   r->streams.push_back(Stream());
   *out_thread = t;
@@ -97,6 +99,7 @@ Slot HostPool::append_one(Request &r, int32_t thread) {
   }
   Slot slot{s.pages[k / page_size_], k % page_size_};
   s.len = k + 1;
+  r.threads[thread].pos_next += 1;
   std::vector<Seg> &view = r.threads[thread].view;
   if (!view.empty() && view.back().stream == thread && view.back().start + view.back().len == k)
     view.back().len += 1;
@@ -224,6 +227,7 @@ void HostPool::dump(std::vector<int32_t> *w) const {
       w->push_back(static_cast<int32_t>(t));
       w->push_back(th.state);
       w->push_back(th.cutoff);
+      w->push_back(th.pos_next);
       w->push_back(static_cast<int32_t>(th.view.size()));
       for (const Seg &s : th.view) {
         w->push_back(s.stream);

@@ -31,6 +31,7 @@ struct Stream {
 struct Thread {
   int32_t state = PASTA_THREAD_ACTIVE;
   int32_t cutoff = 0;
+  int32_t pos_next = 0;    // position id of the thread's next token
   std::vector<Seg> view;
 };
 
@@ -57,7 +58,7 @@ class HostPool {
 
   pasta_status_t request_begin(int32_t *out_req);
   pasta_status_t request_end(int32_t req);
-  pasta_status_t thread_spawn(int32_t req, int32_t *out_thread);
+  pasta_status_t thread_spawn(int32_t req, int32_t predicted_tokens, int32_t *out_thread);
   pasta_status_t thread_finish(int32_t req, int32_t thread);
   pasta_status_t sync_merge(int32_t req, int32_t n_threads, const int32_t *thread_ids);
 

@@ -5,7 +5,8 @@ pool (the oracle's model or the CUDA library):
 
     ("begin",  req)                      a request starts; `req` is the id the replayer must hand out
     ("run",    req, thread, m)           m tokens are appended to one thread's stream (prefill / catch-up)
-    ("spawn",  req, thread)              the main thread emitted <promise/>; `thread` is the new fork's id
+    ("spawn",  req, thread[, predicted]) the main thread emitted <promise/>; `thread` is the new fork's id; the optional
+                                         fourth field is the block length predicted in the promise (position ids)
     ("step",   ((req, thread, n_new), …)) one decode step: every listed thread appends n_new (0 or 1)
                                          tokens and then issues one attention query
     ("finish", req, thread)              a fork emitted </async>
@@ -352,7 +353,7 @@ def cfg5_trace(n_requests: int = 256, n_steps: int = 512, n_layers: int = 32,
 
 # --------------------------------------------------------------------------- random small scripts (property tests)
 def random_script(seed: int, geo: Optional[Geometry] = None, n_ops: int = 60, max_requests: int = 3,
-                  max_forks: int = 5, paper_flow: bool = False) -> Script:
+                  max_forks: int = 5, paper_flow: bool = False, predictions: bool = False) -> Script:
     """A random but valid operation sequence on a small pool.
 
     Exercises partial merges, merges of empty chunks, forks spawned after a merge, request reuse and
@@ -399,7 +400,8 @@ def random_script(seed: int, geo: Optional[Geometry] = None, n_ops: int = 60, ma
         if blocked:
             do_step([req])
         elif choice < 0.25 and r["next"] <= max_forks:
-            t = book.spawn(req); ops.append(("spawn", req, t))
+            t = book.spawn(req)
+            ops.append(("spawn", req, t, 10 * int(rng.integers(0, 6))) if predictions else ("spawn", req, t))
             if rng.random() < 0.5:
                 m = int(rng.integers(1, 3 * geo.page_size))
                 ops.append(("run", req, t, m)); book.add(req, t, m)

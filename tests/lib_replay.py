@@ -20,8 +20,8 @@ class LibReplay:
     """Applies operations one by one.  With a device pool, tensors of all layers are appended and
     `apply` returns (out, lse) as torch CUDA tensors [layers, n, Hq, d] / [layers, n, Hq] for steps."""
 
-    def __init__(self, script: Script, pool: binding.Pool, layers=None):
-        self.script, self.pool = script, pool
+    def __init__(self, script: Script, pool: binding.Pool, layers=None, rope_theta=None):
+        self.script, self.pool, self.rope_theta = script, pool, rope_theta
         self.layers = list(range(script.geometry.n_layers)) if layers is None else list(layers)
         self.last_slots = None
 
@@ -34,7 +34,8 @@ class LibReplay:
         elif kind == "end":
             p.request_end(op[1])
         elif kind == "spawn":
-            got = p.thread_spawn(op[1]); assert got == op[2], (got, op)
+            got = p.thread_spawn_predicted(op[1], op[3]) if len(op) > 3 else p.thread_spawn(op[1])
+            assert got == op[2], (got, op)
         elif kind == "finish":
             p.thread_finish(op[1], op[2])
         elif kind == "merge":
@@ -45,7 +46,10 @@ class LibReplay:
             else:
                 ks, vs = zip(*[run_tensors(self.script, i, l) for l in self.layers])
                 k = torch.stack(ks).cuda(); v = torch.stack(vs).cuda()
-                p.kv_append_run(op[1], op[2], op[3], k, v)
+                if self.rope_theta:
+                    p.kv_append_run_rope(op[1], op[2], op[3], k, v, self.rope_theta)
+                else:
+                    p.kv_append_run(op[1], op[2], op[3], k, v)
         elif kind == "step":
             reqs = [e[0] for e in op[1]]; thr = [e[1] for e in op[1]]; nn = [e[2] for e in op[1]]
             p.step_begin(reqs, thr, nn)
@@ -54,7 +58,11 @@ class LibReplay:
                 return None
             ks, vs, qs = zip(*[step_tensors(self.script, i, l) for l in self.layers])
             k = torch.stack(ks).cuda(); v = torch.stack(vs).cuda(); q = torch.stack(qs).cuda()
-            p.kv_append(k, v)
+            if self.rope_theta:
+                p.kv_append_rope(k, v, self.rope_theta)
+                p.rope_queries(q, self.rope_theta)
+            else:
+                p.kv_append(k, v)
             if not attend:
                 return None
             out = torch.empty(q.shape, dtype=torch.float32, device="cuda")

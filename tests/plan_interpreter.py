@@ -6,7 +6,7 @@ import numpy as np
 # header word indices (pasta_plan.h)
 (PH_MAGIC, PH_N_QUERIES, PH_N_APPEND, PH_N_TREQ, PH_N_TUNITS, PH_N_WUNITS, PH_T_ROWS, PH_ROWS, PH_T_GRID,
  PH_OFF_APPEND, PH_OFF_QUERY, PH_OFF_TREQ, PH_OFF_TRANGE, PH_OFF_TUNIT, PH_OFF_TCTA, PH_OFF_WUNIT, PH_OFF_PAGES,
- PH_OFF_PMETA, PH_OFF_VIS, PH_OFF_TQ, PH_TOTAL_WORDS) = range(21)
+ PH_OFF_PMETA, PH_OFF_VIS, PH_OFF_TQ, PH_OFF_APOS, PH_OFF_QPOS, PH_TOTAL_WORDS) = range(23)
 PQ, PT, PU, PW = 4, 6, 5, 4
 TILE_PAGES, PAGE = 8, 16
 

@@ -134,3 +134,26 @@ def test_bad_configurations_are_rejected():
         assert e.value.code == binding.INVALID_ARG
     with pytest.raises(binding.PastaError):
         binding.Pool(1, 4, 2, 64, 4, 1, 2, 4, free_order=[0, 1, 1, 3], flags=binding.FLAG_HOST_ONLY)
+
+
+@pytest.mark.parametrize("seed", range(20, 28))
+def test_position_ids_match_oracle(seed):
+    """Promises with length predictions: the library's position ids (per step entry, and the per-thread counters in
+    the dump) equal the oracle model's."""
+    script = random_script(seed, n_ops=90, geo=Geometry(1, 4, 2, 64, 16), predictions=True)
+    pool = make_pool(script, host_only=True)
+    lib = LibReplay(script, pool)
+    ora = OracleReplay(script, with_kv=False)
+    checked = 0
+    for i, op in enumerate(script.ops):
+        lib.apply(i)
+        if op[0] == "step":
+            ora.model.reserve(op[1]); ora.next_op += 1
+            want = [ora.model.last_position(e[0], e[1]) for e in op[1]]
+            assert pool.step_positions().tolist() == want
+            checked += 1
+        else:
+            ora.apply(i)
+        assert pool.dump() == ora.model.dump(), (i, op)
+    assert checked
+    pool.close()
