@@ -9,3 +9,4 @@ from .pool_model import (PoolModel, PoolError, OK, INVALID_ARG, OUT_OF_PAGES, BA
 from .attention import KVStore, attend, decode_attention  # noqa: F401
 from .replay import OracleReplay  # noqa: F401
 from .rope import rope, rope_bf16  # noqa: F401
+from .interpreter_model import paper_timeline  # noqa: F401

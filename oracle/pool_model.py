@@ -33,6 +33,12 @@ a fork's first token takes the position right after its <promise/>, the main thr
 position plus the predicted length.  Positions are never revised: if a chunk turns out longer than predicted,
 its ids run into the ids the main thread used after the promise (not monotone after sync); if shorter, a gap
 stays.  How the prediction is made (fixed 40, exact, multiples of ten, ground truth) is the caller's business.
+
+Spawning on a decoded promise (Section 3 "Efficiency", the walk through Fig. 2b: the <async> tag joins the pool at
+the timestamp of its <promise/>, and the fork decodes its first own token at the next one): a fork may be spawned
+while the promise is decoded but its KV is not in the pool yet (`pending=1`).  The fork's view then counts the
+main thread's NEXT token in; the result is the same as appending that token first and spawning afterwards, and
+the fork may take part in a step only if the main thread's token is in the pool by the end of that step's appends.
 """
 from __future__ import annotations
 
@@ -58,6 +64,8 @@ class _Request:
         self.view: Dict[int, List[List[int]]] = {0: []}
         self.next_thread = 1
         self.pos_next: Dict[int, int] = {0: 0}             # thread id -> position id of the thread's next token
+        self.pos_skip = 0                                  # positions the main thread skips after its next token
+        self.pos_last: Dict[int, int] = {0: -1}            # thread id -> position id of the thread's newest own token
 
 
 class PoolModel:
@@ -89,21 +97,42 @@ class PoolModel:
                 self.free.insert(0, page)
         del self.requests[req]
 
-    def thread_spawn(self, req: int, predicted_tokens: int = 0) -> int:
+    def thread_spawn(self, req: int, predicted_tokens: int = 0, pending: int = 0) -> int:
         """<promise/>: the new fork sees what the main thread sees right now, and nothing later.  Its first token
-        takes the position after the promise; the main thread skips `predicted_tokens` positions."""
+        takes the position after the promise; the main thread skips `predicted_tokens` positions.
+        pending=1: the promise is the main thread's next token, not appended yet; it counts as seen."""
         r = self._req(req)
-        if predicted_tokens < 0:
+        if predicted_tokens < 0 or pending not in (0, 1):
             raise PoolError(INVALID_ARG, "negative predicted length")
         t = r.next_thread
         if t >= self.max_threads:
             raise PoolError(CAPACITY, "too many threads")
+        if pending:
+            if not self._can_grow(r, 0):
+                raise PoolError(CAPACITY, "too many segments")
+            k = r.stream_len[0]
+            snapshot = [list(e) for e in r.view[0]]
+            if snapshot and snapshot[-1][0] == 0 and snapshot[-1][1] + snapshot[-1][2] == k:
+                snapshot[-1][2] += 1
+            else:
+                snapshot.append([0, k, 1, -1])
+            r.next_thread += 1
+            r.stream_len[t] = 0
+            r.stream_pages[t] = []
+            r.state[t] = ACTIVE
+            r.cutoff[t] = k + 1
+            r.view[t] = snapshot
+            r.pos_last[t] = -1
+            r.pos_next[t] = r.pos_next[0] + 1       # right after the promise, which takes pos_next[0]
+            r.pos_skip += predicted_tokens          # the main thread jumps once the promise is in
+            return t
         r.next_thread += 1
         r.stream_len[t] = 0
         r.stream_pages[t] = []
         r.state[t] = ACTIVE
         r.cutoff[t] = r.stream_len[0]
         r.view[t] = [list(e) for e in r.view[0]]
+        r.pos_last[t] = -1
         r.pos_next[t] = r.pos_next[0]
         r.pos_next[0] += predicted_tokens
         return t
@@ -135,6 +164,12 @@ class PoolModel:
                 raise PoolError(INVALID_ARG, "query with nothing visible")
             if n_new and not self._can_grow(r, thread):
                 raise PoolError(CAPACITY, "too many segments")
+        main_grows = {req for req, thread, n_new in entries if thread == 0 and n_new}
+        for req, thread, n_new in entries:
+            r = self.requests[req]
+            main_len = r.stream_len[0] + (1 if req in main_grows else 0)
+            if thread != 0 and r.cutoff[thread] > main_len:
+                raise PoolError(BAD_STATE, "the fork's promise is not in the pool")
         if need > len(self.free):
             raise PoolError(OUT_OF_PAGES, "pool exhausted")
         return [self._append_one(req, thread) if n_new else None for req, thread, n_new in entries]
@@ -145,6 +180,8 @@ class PoolModel:
             raise PoolError(INVALID_ARG, "bad run")
         if r.state[thread] != ACTIVE:
             raise PoolError(INVALID_ARG, "thread is not active")
+        if thread != 0 and r.cutoff[thread] > r.stream_len[0]:
+            raise PoolError(BAD_STATE, "the fork's promise is not in the pool")
         n = r.stream_len[thread]
         need = -(-(n + m) // self.page_size) - -(-n // self.page_size)
         if need > len(self.free):
@@ -167,7 +204,11 @@ class PoolModel:
             r.stream_pages[stream].append(self.free.pop(0))
         slot = (r.stream_pages[stream][k // self.page_size], k % self.page_size)
         r.stream_len[stream] = k + 1
+        r.pos_last[thread] = r.pos_next[thread]
         r.pos_next[thread] += 1
+        if thread == 0:
+            r.pos_next[0] += r.pos_skip
+            r.pos_skip = 0
         view = r.view[thread]
         if view and view[-1][0] == stream and view[-1][1] + view[-1][2] == k:
             view[-1][2] += 1
@@ -189,6 +230,9 @@ class PoolModel:
         for t in threads:
             if r.state[t] != FINISHED:
                 raise PoolError(BAD_STATE, "fork still decoding")
+        for t in threads:
+            if r.cutoff[t] > r.stream_len[0]:
+                raise PoolError(BAD_STATE, "the fork's promise is not in the pool")
         view = [list(e) for e in r.view[0]]
         for t in sorted(threads):
             n = r.stream_len[t]
@@ -230,7 +274,10 @@ class PoolModel:
 
     def last_position(self, req: int, thread: int) -> int:
         """Position id of the thread's newest token (the one a decode step's query belongs to)."""
-        return self._req(req).pos_next[thread] - 1
+        r = self._req(req)
+        if r.pos_last[thread] >= 0:
+            return r.pos_last[thread]
+        return r.pos_next[thread] - 1       # a fork without own tokens: the promise (or the token before it)
 
     def dump(self) -> dict:
         """Whole bookkeeping state in a canonical form."""

@@ -44,7 +44,7 @@ class OracleReplay:
         elif kind == "end":
             m.request_end(op[1])
         elif kind == "spawn":
-            got = m.thread_spawn(op[1], op[3] if len(op) > 3 else 0)
+            got = m.thread_spawn(op[1], op[3] if len(op) > 3 else 0, op[4] if len(op) > 4 else 0)
             assert got == op[2], (got, op)
         elif kind == "finish":
             m.thread_finish(op[1], op[2])

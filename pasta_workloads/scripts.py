@@ -5,8 +5,11 @@ pool (the oracle's model or the CUDA library):
 
     ("begin",  req)                      a request starts; `req` is the id the replayer must hand out
     ("run",    req, thread, m)           m tokens are appended to one thread's stream (prefill / catch-up)
-    ("spawn",  req, thread[, predicted]) the main thread emitted <promise/>; `thread` is the new fork's id; the optional
-                                         fourth field is the block length predicted in the promise (position ids)
+    ("spawn",  req, thread[, predicted[, pending]])
+                                         the main thread emitted <promise/>; `thread` is the new fork's id; the optional
+                                         fourth field is the block length predicted in the promise (position ids); a
+                                         fifth field of 1 says that the promise is the main thread's next token, decoded
+                                         but not appended yet
     ("step",   ((req, thread, n_new), …)) one decode step: every listed thread appends n_new (0 or 1)
                                          tokens and then issues one attention query
     ("finish", req, thread)              a fork emitted </async>

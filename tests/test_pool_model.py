@@ -144,3 +144,89 @@ def test_capacities():
     assert e.value.code == CAPACITY and m.dump() == before
     m.sync_merge(a, [t1])                        # [main 2][t1][main 2] fits
     assert len(m.view(a, 0)) == 3
+
+
+# ------------------------------------------------------------------ spawning on a decoded, not yet appended promise
+def _random_state(seed):
+    """A pool in some state reached by random valid operations, built twice."""
+    import copy
+    rng = np.random.default_rng(1000 + seed)
+    m = PoolModel(256, 4, max_segments_per_thread=64)
+    for _ in range(int(rng.integers(1, 4))):
+        req = m.request_begin()
+        m.append_run(req, 0, int(rng.integers(0, 11)))
+        for _round in range(int(rng.integers(0, 3))):
+            forks = [m.thread_spawn(req, int(rng.integers(0, 5)) * 10) for _k in range(int(rng.integers(1, 4)))]
+            m.append_run(req, 0, int(rng.integers(0, 6)))
+            for t in forks:
+                m.append_run(req, t, int(rng.integers(0, 7)))
+                m.thread_finish(req, t)
+            m.sync_merge(req, forks[:int(rng.integers(0, len(forks) + 1))])
+    return m, copy.deepcopy(m), rng
+
+
+@pytest.mark.parametrize("seed", range(12))
+def test_spawn_on_a_pending_promise_equals_append_then_spawn(seed):
+    a, b, rng = _random_state(seed)
+    for req in sorted(a.requests):
+        predicted = int(rng.integers(0, 6)) * 10
+        as_step = bool(rng.integers(0, 2))
+        # a: the promise enters the pool, then the fork is spawned and takes its first token
+        if as_step:
+            a.reserve([(req, 0, 1)])
+        else:
+            a.append_run(req, 0, 1)
+        ta = a.thread_spawn(req, predicted)
+        # b: the fork is spawned first; promise and the fork's first token enter in one step
+        tb = b.thread_spawn(req, predicted, pending=1)
+        assert ta == tb
+        with pytest.raises(PoolError) as e:
+            b.reserve([(req, tb, 1)])                 # the promise is not in the pool yet
+        assert e.value.code == BAD_STATE
+        with pytest.raises(PoolError) as e:
+            b.append_run(req, tb, 1)
+        assert e.value.code == BAD_STATE
+        if as_step:
+            sa = a.reserve([(req, ta, 1)])
+            sb = b.reserve([(req, 0, 1), (req, tb, 1)])
+            assert sb[1] == sa[0]
+        else:
+            b.append_run(req, 0, 1)
+        assert a.dump() == b.dump()
+        # and the two stay the same through the rest of the fork's life
+        for m in (a, b):
+            m.append_run(req, 0, 3)
+            m.append_run(req, ta, 5)
+            m.thread_finish(req, ta)
+            m.sync_merge(req, [ta])
+            m.append_run(req, 0, 1)
+        assert a.dump() == b.dump()
+        assert a.visible_slots(req, 0) == b.visible_slots(req, 0)
+
+
+def test_pending_spawn_position_ids_follow_the_closed_form():
+    # prompt of n tokens at positions 0..n-1; the promise takes n; the fork starts at n+1; with a predicted block
+    # of L tokens the main thread's token after the promise takes n+1+L (Section 6, "Positional Embedding")
+    n, L = 7, 30
+    m = PoolModel(64, 4)
+    req = m.request_begin()
+    m.append_run(req, 0, n)
+    t = m.thread_spawn(req, L, pending=1)
+    assert m.requests[req].pos_next[t] == n + 1
+    assert m.requests[req].pos_next[0] == n                 # the promise itself is not displaced
+    m.reserve([(req, 0, 1), (req, t, 1)])
+    assert m.last_position(req, 0) == n and m.last_position(req, t) == n + 1
+    m.reserve([(req, 0, 1), (req, t, 1)])
+    assert m.last_position(req, 0) == n + 1 + L and m.last_position(req, t) == n + 2
+
+
+def test_merging_a_fork_whose_promise_never_arrived_is_refused():
+    m = PoolModel(64, 4)
+    req = m.request_begin()
+    m.append_run(req, 0, 5)
+    t = m.thread_spawn(req, 0, pending=1)
+    m.thread_finish(req, t)
+    before = m.dump()
+    with pytest.raises(PoolError) as e:
+        m.sync_merge(req, [t])
+    assert e.value.code == BAD_STATE and m.dump() == before
