@@ -106,9 +106,17 @@ pasta_status_t pasta_thread_spawn(pasta_pool_t *pool, int32_t req, int32_t *out_
  * takes that id plus predicted_tokens (>= 0; e.g. 10 x the promise's `tokens` attribute for the paper's
  * Pred-10X scheme, 40 for Fixed-40).  Ids are never revised: a chunk longer than predicted runs into ids
  * the main thread has used (not monotone after sync), a shorter one leaves a gap.
- * pasta_thread_spawn is the same with predicted_tokens = 0.
+ *
+ * pending (0 or 1): 1 = the promise has been decoded but is not in the pool yet; it is the main thread's next
+ * token (Section 3 "Efficiency", the walk through Fig. 2b: the <async> tag joins the pool at the timestamp of its
+ * promise, so the promise and the fork's first token are fed to the model in one step).  The fork's view then
+ * counts that token in, the promise keeps the main thread's next position id and the jump by predicted_tokens
+ * follows it.  The outcome equals appending the promise first and spawning with pending = 0.  Until the promise
+ * is in the pool (by the appends of the same step at the latest) the fork can neither take part in a step, nor
+ * append a run, nor be merged: PASTA_ERR_BAD_STATE.  PASTA_ERR_CAPACITY if the main thread's segment list is full.
+ * pasta_thread_spawn is the same with predicted_tokens = 0 and pending = 0.
  */
-pasta_status_t pasta_thread_spawn_predicted(pasta_pool_t *pool, int32_t req, int32_t predicted_tokens,
+pasta_status_t pasta_thread_spawn_predicted(pasta_pool_t *pool, int32_t req, int32_t predicted_tokens, int32_t pending,
                                             int32_t *out_thread);
 /* </async>: the fork decodes no more; its chunk stays invisible to the main thread until merged. */
 pasta_status_t pasta_thread_finish(pasta_pool_t *pool, int32_t req, int32_t thread);

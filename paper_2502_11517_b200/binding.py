@@ -157,9 +157,9 @@ class Pool:
         _check(lib().pasta_thread_spawn(self._h, req, C.byref(out)), "pasta_thread_spawn")
         return out.value
 
-    def thread_spawn_predicted(self, req: int, predicted_tokens: int) -> int:
+    def thread_spawn_predicted(self, req: int, predicted_tokens: int, pending: int = 0) -> int:
         out = C.c_int32()
-        _check(lib().pasta_thread_spawn_predicted(self._h, req, predicted_tokens, C.byref(out)),
+        _check(lib().pasta_thread_spawn_predicted(self._h, req, predicted_tokens, pending, C.byref(out)),
                "pasta_thread_spawn_predicted")
         return out.value
 

@@ -265,12 +265,13 @@ pasta_status_t pasta_request_end(pasta_pool_t *p, int32_t req) {
 
 pasta_status_t pasta_thread_spawn(pasta_pool_t *p, int32_t req, int32_t *out_thread) {
   if (!p || !out_thread) return PASTA_ERR_INVALID_ARG;
-  return p->host.thread_spawn(req, 0, out_thread);
+  return p->host.thread_spawn(req, 0, 0, out_thread);
 }
 
-pasta_status_t pasta_thread_spawn_predicted(pasta_pool_t *p, int32_t req, int32_t predicted_tokens, int32_t *out_thread) {
+pasta_status_t pasta_thread_spawn_predicted(pasta_pool_t *p, int32_t req, int32_t predicted_tokens, int32_t pending,
+                                            int32_t *out_thread) {
   if (!p || !out_thread) return PASTA_ERR_INVALID_ARG;
-  return p->host.thread_spawn(req, predicted_tokens, out_thread);
+  return p->host.thread_spawn(req, predicted_tokens, pending, out_thread);
 }
 
 pasta_status_t pasta_step_positions(pasta_pool_t *p, int32_t *out_pos, int32_t capacity_entries) {
@@ -430,6 +431,8 @@ static pasta_status_t append_run_impl(pasta_pool_t *p, int32_t req, int32_t thre
   std::vector<Slot> slots;
   const Request *rq = p->host.request(req);
   const int32_t pos0 = (rq && thread >= 0 && thread < static_cast<int32_t>(rq->threads.size())) ? rq->threads[thread].pos_next : 0;
+  // consecutive position ids are assumed below: not so while the main thread owes a jump behind a pending promise
+  if (theta > 0.f && m > 1 && thread == 0 && rq && rq->threads[0].pos_skip != 0) return PASTA_ERR_BAD_STATE;
   pasta_status_t s = p->host.reserve_run(req, thread, m, &slots);
   if (s != PASTA_OK) return s;
   p->plan_valid = false;

@@ -254,7 +254,7 @@ pasta_status_t build_plan(const HostPool &pool, const std::vector<StepEntry> &en
   };
   std::vector<int32_t> app, apos, qpos;
   for (int32_t i = 0; i < n; ++i) {
-    const int32_t pos = pool.request(entries[i].req)->threads[entries[i].thread].pos_next - 1;   // the newest token
+    const int32_t pos = HostPool::query_position(pool.request(entries[i].req)->threads[entries[i].thread]);   // the newest token
     qpos.push_back(pos);
     if (entries[i].n_new) { app.push_back(slots[i].page); app.push_back(slots[i].offset); apos.push_back(pos); }
   }

@@ -56,16 +56,28 @@ pasta_status_t HostPool::request_end(int32_t req) {
   return PASTA_OK;
 }
 
-pasta_status_t HostPool::thread_spawn(int32_t req, int32_t predicted_tokens, int32_t *out_thread) {
+pasta_status_t HostPool::thread_spawn(int32_t req, int32_t predicted_tokens, int32_t pending, int32_t *out_thread) {
   Request *r = live(req);
-  if (!r || predicted_tokens < 0) return PASTA_ERR_INVALID_ARG;
+  if (!r || predicted_tokens < 0 || (pending != 0 && pending != 1)) return PASTA_ERR_INVALID_ARG;
   int32_t t = static_cast<int32_t>(r->threads.size());
   if (t >= max_threads_) return PASTA_ERR_CAPACITY;
+  if (pending && !can_extend(*r, 0)) return PASTA_ERR_CAPACITY;
   Thread fork;
-  fork.cutoff = r->streams[0].len;
-  fork.view = r->threads[0].view;          // frozen snapshot of what the main thread sees now
-  fork.pos_next = r->threads[0].pos_next;  // the fork continues right after the promise ...
-  r->threads[0].pos_next += predicted_tokens;   // ... and the main thread skips the predicted block
+  Thread &main_thread = r->threads[0];
+  const int32_t len0 = r->streams[0].len;
+  fork.cutoff = len0 + pending;
+  fork.view = main_thread.view;            // frozen snapshot of what the main thread sees now
+  if (pending) {                           // ... plus the promise it is about to append
+    if (!fork.view.empty() && fork.view.back().stream == 0 && fork.view.back().start + fork.view.back().len == len0)
+      fork.view.back().len += 1;
+    else
+      fork.view.push_back(Seg{0, len0, 1, -1});
+    fork.pos_next = main_thread.pos_next + 1;    // the promise takes pos_next, the fork continues behind it
+    main_thread.pos_skip += predicted_tokens;    // the main thread jumps once the promise is in
+  } else {
+    fork.pos_next = main_thread.pos_next;        // the fork continues right after the promise ...
+    main_thread.pos_next += predicted_tokens;    // ... and the main thread skips the predicted block
+  }
   r->threads.push_back(std::move(fork));
   r->streams.push_back(Stream());
   *out_thread = t;
@@ -99,7 +111,10 @@ Slot HostPool::append_one(Request &r, int32_t thread) {
   }
   Slot slot{s.pages[k / page_size_], k % page_size_};
   s.len = k + 1;
-  r.threads[thread].pos_next += 1;
+  Thread &th = r.threads[thread];
+  th.pos_last = th.pos_next;
+  th.pos_next += 1 + th.pos_skip;
+  th.pos_skip = 0;
   std::vector<Seg> &view = r.threads[thread].view;
   if (!view.empty() && view.back().stream == thread && view.back().start + view.back().len == k)
     view.back().len += 1;
@@ -134,6 +149,16 @@ pasta_status_t HostPool::reserve_step(const std::vector<StepEntry> &entries, std
     if (!e.n_new && t.view.empty()) return PASTA_ERR_INVALID_ARG;
     if (e.n_new && !can_extend(*r, e.thread)) return PASTA_ERR_CAPACITY;
   }
+  for (const StepEntry &e : entries) {     // a fork spawned on a pending promise needs that promise in the pool
+    if (e.thread == 0) continue;
+    const Request *r = live(e.req);
+    int32_t main_len = r->streams[0].len;
+    if (r->threads[e.thread].cutoff > main_len) {
+      for (const StepEntry &o : entries)
+        if (o.req == e.req && o.thread == 0 && o.n_new) { ++main_len; break; }
+      if (r->threads[e.thread].cutoff > main_len) return PASTA_ERR_BAD_STATE;
+    }
+  }
   if (need > free_.size()) return PASTA_ERR_OUT_OF_PAGES;
   // pass 2: commit
   slots->clear();
@@ -148,6 +173,7 @@ pasta_status_t HostPool::reserve_run(int32_t req, int32_t thread, int32_t m, std
   if (!r || thread < 0 || thread >= static_cast<int32_t>(r->threads.size()) || m < 0)
     return PASTA_ERR_INVALID_ARG;
   if (r->threads[thread].state != PASTA_THREAD_ACTIVE) return PASTA_ERR_INVALID_ARG;
+  if (thread != 0 && r->threads[thread].cutoff > r->streams[0].len) return PASTA_ERR_BAD_STATE;
   const int64_t n = r->streams[thread].len;
   const int64_t P = page_size_;
   const int64_t need = (n + m + P - 1) / P - (n + P - 1) / P;
@@ -177,6 +203,8 @@ pasta_status_t HostPool::sync_merge(int32_t req, int32_t n_threads, const int32_
     for (int32_t t : forks)
       if (r->threads[t].state != PASTA_THREAD_FINISHED) return PASTA_ERR_BAD_STATE;
   }
+  for (int32_t t : forks)
+    if (r->threads[t].cutoff > r->streams[0].len) return PASTA_ERR_BAD_STATE;   // its promise never arrived
   std::vector<Seg> view = r->threads[0].view;   // work on a copy: all or nothing
   for (int32_t t : forks) {                     // ascending id
     const int32_t len = r->streams[t].len;

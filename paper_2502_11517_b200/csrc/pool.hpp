@@ -32,6 +32,8 @@ struct Thread {
   int32_t state = PASTA_THREAD_ACTIVE;
   int32_t cutoff = 0;
   int32_t pos_next = 0;    // position id of the thread's next token
+  int32_t pos_last = -1;   // position id of the thread's newest own token (-1: none yet)
+  int32_t pos_skip = 0;    // main thread only: positions to skip once its next token is in
   std::vector<Seg> view;
 };
 
@@ -58,7 +60,11 @@ class HostPool {
 
   pasta_status_t request_begin(int32_t *out_req);
   pasta_status_t request_end(int32_t req);
-  pasta_status_t thread_spawn(int32_t req, int32_t predicted_tokens, int32_t *out_thread);
+  // pending = 1: the promise is the main thread's next token, decoded but not appended yet; the fork's view
+  // counts it in, and the fork may join a step only once that token is in the pool by the step's appends.
+  pasta_status_t thread_spawn(int32_t req, int32_t predicted_tokens, int32_t pending, int32_t *out_thread);
+  // position id of the token a query of this thread belongs to
+  static int32_t query_position(const Thread &t) { return t.pos_last >= 0 ? t.pos_last : t.pos_next - 1; }
   pasta_status_t thread_finish(int32_t req, int32_t thread);
   pasta_status_t sync_merge(int32_t req, int32_t n_threads, const int32_t *thread_ids);
 

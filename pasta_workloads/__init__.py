@@ -19,4 +19,5 @@ from .scripts import (  # noqa: F401
     random_script,
     step_tensors,
     run_tensors,
+    token_tensors,
 )

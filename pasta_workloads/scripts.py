@@ -80,6 +80,15 @@ def _randn_bf16(shape, g: torch.Generator, device: str) -> torch.Tensor:
     return torch.randn(shape, generator=g, device=device, dtype=torch.float32).to(torch.bfloat16)
 
 
+def token_tensors(seed: int, geo: "Geometry", thread: int, index: int, layer: int):
+    """(k, v, q) of the index-th token a thread feeds to the model, for one layer: k, v [Hkv, d], q [Hq, d] bf16.
+    For drivers that produce tokens one by one (no script): the tensors depend on who feeds the token and on
+    its rank in that thread, on nothing else."""
+    g = _gen(seed, thread * 1000003 + index, layer)
+    return (_randn_bf16((geo.n_kv_heads, geo.head_dim), g, "cpu"), _randn_bf16((geo.n_kv_heads, geo.head_dim), g, "cpu"),
+            _randn_bf16((geo.n_q_heads, geo.head_dim), g, "cpu"))
+
+
 def run_tensors(script: Script, op_index: int, layer: int, device: str = "cpu"):
     """K and V ([m, Hkv, d] bf16 each) carried by the "run" operation `op_index` for one layer."""
     op = script.ops[op_index]

@@ -34,7 +34,7 @@ class LibReplay:
         elif kind == "end":
             p.request_end(op[1])
         elif kind == "spawn":
-            got = p.thread_spawn_predicted(op[1], op[3]) if len(op) > 3 else p.thread_spawn(op[1])
+            got = p.thread_spawn_predicted(op[1], op[3], op[4] if len(op) > 4 else 0) if len(op) > 3 else p.thread_spawn(op[1])
             assert got == op[2], (got, op)
         elif kind == "finish":
             p.thread_finish(op[1], op[2])

@@ -1,0 +1,129 @@
+"""The library-side interpreter against the oracle's timeline: same tokens fed per step, same pool state after
+every step (pages, views, cut-offs, position ids), on the worked example of Fig. 2 and on random thread scripts.
+Step s+1 of the interpreter feeds what the paper's accounting enters at timestamp s."""
+import copy
+
+import numpy as np
+import pytest
+
+from oracle import PoolModel, paper_timeline
+from paper_2502_11517_b200 import binding
+from paper_2502_11517_b200.build import build
+from paper_2502_11517_b200.interpreter import Interpreter, Tags
+from test_interpreter_model import CLOSE, OPEN, PROMISE, SYNC, TAGS, fig2_scripts
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    build()
+
+
+class Scripted:
+    """A stand-in for the model: thread t's k-th decoded token is emissions[t][k]."""
+
+    def __init__(self, emissions):
+        self.emissions, self.count = emissions, {}
+
+    def __call__(self, entries):
+        out = []
+        for req, t, _tok in entries:
+            k = self.count.get((req, t), 0); self.count[(req, t)] = k + 1
+            out.append(self.emissions[t][k] if k < len(self.emissions[t]) else -1)
+        return out
+
+
+def oracle_run(prompt, emissions, n_pages, predicted):
+    model = PoolModel(n_pages, 16)
+    states, fed = {0: None}, {}
+
+    def snap(T, entered):
+        states[T] = copy.deepcopy(model.dump()); fed[T] = list(entered)
+
+    req, log, withheld = paper_timeline(model, prompt, emissions, predicted_length=predicted, on_timestamp=snap, **TAGS)
+    return states, fed, withheld
+
+
+def library_run(prompt, emissions, n_pages, predicted, n_steps):
+    pool = binding.Pool(1, 4, 2, 64, n_pages, 2, 16, 64, flags=binding.FLAG_HOST_ONLY)
+    it = Interpreter(pool, Tags(PROMISE, OPEN, CLOSE, SYNC), predicted_length=lambda req, k: predicted(k))
+    req = it.add_request(prompt)
+    fake = Scripted(emissions)
+    states, fed = {}, {}
+    for step in range(1, n_steps + 1):
+        entries = it.begin_step()
+        fed[step] = [(t, tok) for _r, t, tok in entries]
+        states[step] = pool.dump()
+        it.end_step(fake(entries))
+    pool.close()
+    return states, fed
+
+
+def random_threads(seed):
+    rng = np.random.default_rng(seed)
+    main, forks = [], {}
+    for _ in range(int(rng.integers(1, 4))):                  # promise groups, each closed by a <sync/>
+        main += [int(x) for x in rng.integers(100, 200, int(rng.integers(0, 4)))]
+        for _p in range(int(rng.integers(1, 4))):
+            main.append(PROMISE)
+            forks[len(forks) + 1] = [int(x) for x in rng.integers(200, 300, int(rng.integers(0, 9)))] + [CLOSE]
+            main += [int(x) for x in rng.integers(100, 200, int(rng.integers(0, 3)))]
+        main += [int(x) for x in rng.integers(100, 200, int(rng.integers(0, 12)))] + [SYNC]
+    main += [int(x) for x in rng.integers(100, 200, int(rng.integers(1, 4)))]
+    prompt = [int(x) for x in rng.integers(300, 400, int(rng.integers(1, 40)))]
+    return prompt, {0: main, **forks}
+
+
+def check(prompt, emissions, predicted):
+    o_states, o_fed, withheld = oracle_run(prompt, emissions, 64, predicted)
+    T_max = max(o_fed)
+    l_states, l_fed = library_run(prompt, emissions, 64, predicted, T_max + 1)
+    assert l_fed[1] == [(0, prompt[-1])]
+    for T in range(1, T_max + 1):
+        assert l_fed[T + 1] == o_fed[T], (T, l_fed[T + 1], o_fed[T])
+        want = o_states[T]
+        got = l_states[T + 1]
+        # thread states differ in one respect only: the library marks a fork finished after its </async> was fed,
+        # and merged right away once the waiting <sync/> may go on; the oracle's accounting does both when the
+        # tokens enter.  Compare everything else exactly.
+        for d in (want, got):
+            for r in d["requests"].values():
+                for th in r["threads"].values():
+                    th.pop("state")
+        assert got == want, T
+    return withheld
+
+
+def test_fig2_replay_through_the_library():
+    ids, prompt, emissions = fig2_scripts()
+    withheld = check(prompt, emissions, lambda k: 10)
+    assert withheld == [(3, 8)]
+
+
+@pytest.mark.parametrize("seed", range(20))
+def test_random_thread_scripts(seed):
+    prompt, emissions = random_threads(seed)
+    check(prompt, emissions, (lambda k: 0) if seed % 2 else (lambda k: 10 * (k % 4)))
+
+
+def test_sync_waits_and_merge_moves_nothing():
+    ids, prompt, emissions = fig2_scripts()
+    pool = binding.Pool(1, 4, 2, 64, 64, 2, 16, 64, flags=binding.FLAG_HOST_ONLY)
+    it = Interpreter(pool, Tags(PROMISE, OPEN, CLOSE, SYNC))
+    req = it.add_request(prompt)
+    fake = Scripted(emissions)
+    waited = []
+    pages_before = None
+    for step in range(1, 12):
+        entries = it.begin_step()
+        if it.waiting_at_sync(req):
+            assert all(t != 0 for _r, t, _tok in entries)      # the main thread is not fed while it waits
+            pages_before = {s: v["pages"] for s, v in pool.dump()["requests"][req]["streams"].items()}
+        it.end_step(fake(entries))
+        waited.append(it.waiting_at_sync(req))
+    assert waited == [False, False, True, True, True, True, True, False, False, False, False]
+    streams = pool.dump()["requests"][req]["streams"]
+    for s, pages in pages_before.items():
+        assert streams[s]["pages"][:len(pages)] == pages        # chunks stay where they were written
+    view = pool.dump()["requests"][req]["threads"][0]["view"]
+    assert [seg[0] for seg in view] == [0, 1, 0, 2, 0]          # each chunk right behind its promise
+    pool.close()

@@ -157,3 +157,47 @@ def test_position_ids_match_oracle(seed):
         assert pool.dump() == ora.model.dump(), (i, op)
     assert checked
     pool.close()
+
+
+@pytest.mark.parametrize("seed", range(8))
+def test_pending_spawn_matches_oracle(seed):
+    """Spawning on a decoded, not yet appended promise: same state as the oracle after every call, same refusals."""
+    rng = np.random.default_rng(77 + seed)
+    pool = binding.Pool(1, 4, 2, 64, 128, 2, 8, 6, flags=binding.FLAG_HOST_ONLY)
+    model = PoolModel(128, 16, max_requests=2, max_threads_per_request=8, max_segments_per_thread=6)
+
+    def both(name_lib, name_ora, *args):
+        a, b = _codes(lambda: getattr(pool, name_lib)(*args), lambda: getattr(model, name_ora)(*args))
+        assert a == b, (name_lib, args, a, b)
+        assert pool.dump() == model.dump(), (name_lib, args)
+        return a
+
+    req = pool.request_begin(); assert model.request_begin() == req
+    both("kv_append_run", "append_run", req, 0, int(rng.integers(0, 40)))
+    live = []
+    for _ in range(30):
+        what = int(rng.integers(0, 6))
+        if what == 0:
+            code = both("thread_spawn_predicted", "thread_spawn", req, int(rng.integers(0, 4)) * 10, int(rng.integers(0, 2)))
+            if code == 0:
+                live.append(max(model.requests[req].state))
+        elif what == 1:
+            entries = [(req, 0, 1)] if rng.integers(0, 2) else []
+            entries += [(req, t, int(rng.integers(0, 2))) for t in live if rng.integers(0, 2)]
+            if not entries:
+                continue
+            a, b = _codes(lambda: pool.step_begin(*zip(*entries)), lambda: model.reserve(entries))
+            assert a == b, (entries, a, b)
+            assert pool.dump() == model.dump()
+            if a == 0:
+                want = [model.last_position(r, t) for r, t, _n in entries]
+                assert pool.step_positions().tolist() == want
+        elif what == 2 and live:
+            both("kv_append_run", "append_run", req, live[int(rng.integers(0, len(live)))], int(rng.integers(0, 20)))
+        elif what == 3 and live:
+            t = live.pop(int(rng.integers(0, len(live))))
+            both("thread_finish", "thread_finish", req, t)
+            both("sync_merge", "sync_merge", req, [t])
+        elif what == 4:
+            both("kv_append_run", "append_run", req, 0, int(rng.integers(0, 3)))
+    pool.close()
