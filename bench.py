@@ -39,7 +39,7 @@ NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 # dram bytes (read + write) of one launch of the dominant kernel from an ncu capture of this workload,
 # or None when no capture matches the current kernel
-NCU_TRAFFIC_BYTES = {("long_shared_prefix", "full"): 1.092e9, ("long_shared_prefix", "small"): 2.765e8}   # see profiles/
+NCU_TRAFFIC_BYTES = {}   # (workload, size) -> DRAM bytes per launch of the dominant kernel, from profiles/
 
 
 def make_script(workload: str, size: str = "full"):
@@ -171,7 +171,7 @@ def build_state(script, device, seed_offset=0, grow_tokens=640):
 
 def unique_tokens(pool, entries):
     """Per request, the union of what the step's threads see (a shared prefix counts once); and the part of
-    it that is seen by two or more threads (what the tensor-core kernel reads)."""
+    it that the tensor-core kernel reads: everything, for requests whose stacked query rows fit one MMA tile."""
     dump = pool.dump()
     by_req = {}
     for req, t, _ in entries:
@@ -185,9 +185,11 @@ def unique_tokens(pool, entries):
                 vis[s] = max(vis.get(s, 0), a + n)
             for s, v in vis.items():
                 seen.setdefault(s, []).append(v)
+        on_tensor = (pool.head_dim == 128 and len(threads) * (pool.n_q_heads // pool.n_kv_heads) <= 128
+                     and len(seen) <= 255)
         for s, vs in seen.items():
             total += max(vs)
-            if len(vs) >= 2:
+            if on_tensor:
                 shared += max(vs)
     return total, shared
 

@@ -182,9 +182,11 @@ pasta_status_t pasta_kv_append(pasta_pool_t *pool, int32_t layer_begin, int32_t 
  * included).  q: device bf16 [layer_count, n, n_q_heads, head_dim]; out: device fp32 of the same
  * shape; lse: optional device fp32 [layer_count, n, n_q_heads] (natural-log sum of exponentials of
  * the scaled scores), may be NULL; scale 0 means 1/sqrt(head_dim).
- * Streams seen by two or more threads of the step are staged into shared memory once per kv head
- * and scored against all those threads' queries on tensor cores; streams seen by one thread take
- * a warp-shuffle kernel; a merge kernel combines the partial results (fp32 throughout).
+ * With head_dim 128, the streams a request's threads read are staged into shared memory once per kv
+ * head and scored against all those threads' queries on tensor cores (rows that may not see a page are
+ * masked), as long as threads x (n_q_heads / n_kv_heads) <= 128 and the request has at most 255 streams;
+ * other requests and head sizes take a warp-shuffle kernel; a merge kernel combines the partial results
+ * (fp32 throughout).
  */
 pasta_status_t pasta_decode_attn(pasta_pool_t *pool, int32_t layer_begin, int32_t layer_count,
                                  const void *q, void *out, float *lse, float scale, void *stream);

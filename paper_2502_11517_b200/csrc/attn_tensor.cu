@@ -1,7 +1,8 @@
-// K2: tensor-core pass over streams shared by several queries of a request (head_dim 128).
+// K2: tensor-core pass over every stream the queries of a request read (head_dim 128): the prefix they share is
+// staged once for all of them; a fork's own chunk rides along with the other rows masked.
 //
 // One persistent CTA per SM walks its contiguous range of t-units.  A t-unit is a range of 128-token tiles
-// (8 pages) of one request's shared page list, for one kv head.  Rows of the score matrix are the request's
+// (8 pages) of one request's page list, for one kv head.  Rows of the score matrix are the request's
 // queries times the `group` query heads of that kv head (<= 128 rows, zero padded):
 //
 //   S[128 x 128] = Q[128 x 128] . K_tile^T            tcgen05.mma (N = 128), A and B from shared memory, D in TMEM
@@ -217,14 +218,14 @@ attn_tensor_kernel(PoolView pv, TensorArgs a, const __nv_bfloat16 *__restrict__ 
     for (int s = 0; s < T_STAGES; ++s) { mbar_init(bar + 8 * (B_FULL + s), 1); mbar_init(bar + 8 * (B_EMPTY + s), 1); }
     for (int b = 0; b < 2; ++b) {
       mbar_init(bar + 8 * (B_SFULL + b), 1);
-      mbar_init(bar + 8 * (B_PFULL + 2 * b), 128);
-      mbar_init(bar + 8 * (B_PFULL + 2 * b + 1), 128);
+      mbar_init(bar + 8 * (B_PFULL + 2 * b), 4);        // one arrival per warp: 32 arrivals of a warp on one
+      mbar_init(bar + 8 * (B_PFULL + 2 * b + 1), 4);    // barrier word are served one after the other
     }
-    mbar_init(bar + 8 * B_QFULL, 64);
+    mbar_init(bar + 8 * B_QFULL, 2);
     mbar_init(bar + 8 * B_QFREE, 1);
     mbar_init(bar + 8 * B_OFULL, 1);
-    mbar_init(bar + 8 * B_OFREE, 128);
-    mbar_init(bar + 8 * B_MLFULL, 128);
+    mbar_init(bar + 8 * B_OFREE, 4);
+    mbar_init(bar + 8 * B_MLFULL, 4);
     misc[1] = 0;
     mbar_init_fence();
   }
@@ -361,7 +362,8 @@ attn_tensor_kernel(PoolView pv, TensorArgs a, const __nv_bfloat16 *__restrict__ 
             *reinterpret_cast<uint4 *>(dst + (c >> 3) * 16384 + (((c & 7) ^ r8) << 4)) = val[c];
         }
         fence_proxy_async();
-        mbar_arrive(bar + 8 * B_QFULL);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar + 8 * B_QFULL);
       }
     }
   } else {
@@ -468,7 +470,8 @@ attn_tensor_kernel(PoolView pv, TensorArgs a, const __nv_bfloat16 *__restrict__ 
             tmem_st_wait();
           }
           tc_fence_before();
-          mbar_arrive(bar + 8 * (B_PFULL + 2 * b + grp));
+          __syncwarp();
+          if (lane == 0) mbar_arrive(bar + 8 * (B_PFULL + 2 * b + grp));
         }
         if (!ok) break;
         // ---- epilogue: the unit's rows leave TMEM; group 0 folds group 1's accumulator into its own
@@ -476,7 +479,8 @@ attn_tensor_kernel(PoolView pv, TensorArgs a, const __nv_bfloat16 *__restrict__ 
         tc_fence_after();
         if (grp == 1) {
           if (active) ml1[row] = make_float2(m_ref, l);
-          mbar_arrive(bar + 8 * B_MLFULL);
+          __syncwarp();
+          if (lane == 0) mbar_arrive(bar + 8 * B_MLFULL);
           continue;
         }
         if (!wait_or_abort(bar + 8 * B_MLFULL, uc & 1, abort_flag)) { ok = false; break; }
@@ -510,7 +514,8 @@ attn_tensor_kernel(PoolView pv, TensorArgs a, const __nv_bfloat16 *__restrict__ 
           }
         }
         tc_fence_before();
-        mbar_arrive(bar + 8 * B_OFREE);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar + 8 * B_OFREE);
       }
     }
   }

@@ -25,10 +25,10 @@ cudaError_t launch_kv_append_rope(const PoolView &pv, const int32_t *slots, cons
 // rotates the step's queries in place by their tokens' position ids
 cudaError_t launch_rope_queries(const PoolView &pv, const int32_t *pos, int32_t n, int32_t layer_count, void *q, double theta,
                                 cudaStream_t st);
-// K3: warp-shuffle pass over streams seen by one query
+// K3: warp-shuffle pass for requests the tensor-core kernel does not take (other head sizes, too many rows or streams)
 cudaError_t launch_attn_warp(const PoolView &pv, const PlanHeader &h, int32_t layer_begin, int32_t layer_count,
                              const void *q, float scale_log2, cudaStream_t st);
-// K2: tensor-core pass over streams shared by several queries (head_dim 128 only)
+// K2: tensor-core pass over all streams of a request whose stacked queries fit 128 rows (head_dim 128 only)
 cudaError_t launch_attn_tensor(const PoolView &pv, const PlanHeader &h, int32_t layer_begin, int32_t layer_count,
                                const void *q, float scale_log2, cudaStream_t st);
 bool tensor_path_available();       // false while the tensor-core kernel is compiled out

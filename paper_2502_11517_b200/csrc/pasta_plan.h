@@ -6,13 +6,14 @@
 //   query      one (request, thread) entry of the step, index n in entry order
 //   stream     one page list: a request's main-thread tokens (id 0) or one fork's chunk (id = fork id).
 //              Every thread sees a PREFIX [0, vis) of every stream (vis may be 0).
-//   t-request  a request with at least one stream seen by >= 2 queries of the step ("shared").
-//              Its shared streams' pages are concatenated into one page list that is cut into
+//   t-request  a request served by the tensor-core kernel: head_dim 128, its queries times `group` fit
+//              PASTA_MAX_ROWS rows, at most 255 streams.  The pages of every stream its queries read (the prefix
+//              they share and each fork's own chunk alike) are concatenated into one page list that is cut into
 //              tiles of PASTA_TILE_PAGES pages; rows of the score matrix are the request's queries
 //              times the `group` query heads of one kv head: row = t_idx * group + h_local.
 //   t-unit     (t-request, kv head, tile range): one CTA-sized piece of the tensor-core kernel; it
 //              writes one partial result (m, l, O[d]) per row.
-//   w-unit     (query, kv head, token range of one stream seen by that query alone): one warp of
+//   w-unit     (query, kv head, token range of one stream) of a request that is no t-request: one warp of
 //              the warp-shuffle kernel; it writes `group` partial rows.
 //   partial rows are numbered per layer: t-unit rows first (row_base + row), then
 //              t_rows + w_unit * group + h_local.

@@ -16,7 +16,7 @@ struct StreamUse {
   int32_t page_off = -1;          // where its pages were put in the page table (w-units)
 };
 
-struct WPiece {                   // one stream seen by one query alone
+struct WPiece {                   // one stream read by one query on the warp path
   int32_t query, page_off, vis;
 };
 
@@ -95,11 +95,14 @@ pasta_status_t build_plan(const HostPool &pool, const std::vector<StepEntry> &en
     }
     for (int32_t ti = 0; ti < T; ++ti) q_vis[ti].resize(uses.size(), 0);
 
-    bool tensor = lim.tensor_path && T >= 2 && T * G <= PASTA_MAX_ROWS;
+    // A request whose stacked rows fit one MMA tile sends EVERY stream it reads through the tensor-core kernel, the
+    // private chunks too: rows that may not see a page are masked there, the MMA costs the same for any number of
+    // valid rows, and the pass stays bandwidth-bound; the warp kernel is left with what does not fit.
+    bool tensor = lim.tensor_path && T >= 1 && T * G <= PASTA_MAX_ROWS;
     int32_t n_shared = 0;
     if (tensor) {
       for (StreamUse &u : uses)
-        if (u.n_seen >= 2) u.local = n_shared++;
+        if (u.n_seen >= 1) u.local = n_shared++;
       if (n_shared == 0 || n_shared > 255) {
         tensor = false;
         for (StreamUse &u : uses) u.local = -1;

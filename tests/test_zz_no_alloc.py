@@ -52,8 +52,8 @@ def test_noalloc_refuses_steps_beyond_its_fixed_size():
     from pasta_workloads import cfg4_long_prefix, step_tensors
     from lib_replay import LibReplay, make_pool
     build()
-    script = cfg4_long_prefix(6, 3000, 16)                     # needs more partial rows than the array holds
-    pool = make_pool(script)
+    script = cfg4_long_prefix(6, 3000, 31)                     # 128 stacked rows per unit: more partial rows than the array holds
+    pool = make_pool(script, max_step_queries=256)
     rep = LibReplay(script, pool)
     last = len(script.ops) - 1
     for i in range(last + 1):
