@@ -398,20 +398,40 @@ attn_tensor_kernel(PoolView pv, TensorArgs a, const __nv_bfloat16 *__restrict__ 
           if (!wait_or_abort(bar + 8 * (B_FULL + s), (it / T_STAGES) & 1, abort_flag)) { ok = false; break; }
           int thr[T_HALF_PAGES];
           bool full = true;
-          if (warp_active) {
-            const int4 m4 = *reinterpret_cast<const int4 *>(meta_s + s * PASTA_TILE_PAGES + grp * T_HALF_PAGES);
-            const int metas[T_HALF_PAGES] = {m4.x, m4.y, m4.z, m4.w};
+          const int4 m4 = *reinterpret_cast<const int4 *>(meta_s + s * PASTA_TILE_PAGES + grp * T_HALF_PAGES);
+          // pages that every thread of the request sees in full need no thresholds (the same answer for the whole CTA)
+          const bool no_mask = (m4.x | m4.y | m4.z | m4.w) >= 0 && ((m4.x & m4.y & m4.z & m4.w) & PASTA_PMETA_ALL_VISIBLE);
+          if (warp_active && !no_mask) {
+            const int base_meta = m4.x & ~PASTA_PMETA_ALL_VISIBLE;
+            const bool run = m4.x >= 0 && m4.w >= 0 && (m4.y & ~PASTA_PMETA_ALL_VISIBLE) == base_meta + (1 << 8) &&
+                             (m4.z & ~PASTA_PMETA_ALL_VISIBLE) == base_meta + (2 << 8) &&
+                             (m4.w & ~PASTA_PMETA_ALL_VISIBLE) == base_meta + (3 << 8);
+            if (run) {
+              // four consecutive pages of one stream (the usual case): one look-up of the row's visible length
+              const int sl = base_meta & 255;
+              int vis;
+              if (sl < 4) vis = sl == 0 ? vis0 : sl == 1 ? vis1 : sl == 2 ? vis2 : vis3;
+              else vis = visrow[sl];
+              const int rem = active ? vis - PASTA_PMETA_PAGE(base_meta) * PASTA_PAGE : 0;
 #pragma unroll
-            for (int pg = 0; pg < T_HALF_PAGES; ++pg) {
-              const int meta = metas[pg];
-              int t = 0;
-              if (active && meta >= 0) {
-                const int sl = meta & 255;
-                const int vis = sl == 0 ? vis0 : sl == 1 ? vis1 : sl == 2 ? vis2 : sl == 3 ? vis3 : visrow[sl];
-                t = min(max(vis - (meta >> 8) * PASTA_PAGE, 0), PASTA_PAGE);
+              for (int pg = 0; pg < T_HALF_PAGES; ++pg) thr[pg] = min(max(rem - pg * PASTA_PAGE, 0), PASTA_PAGE);
+              full = rem >= T_HALF_PAGES * PASTA_PAGE;
+            } else {
+              const int metas[T_HALF_PAGES] = {m4.x, m4.y, m4.z, m4.w};
+#pragma unroll
+              for (int pg = 0; pg < T_HALF_PAGES; ++pg) {
+                const int meta = metas[pg];
+                int t = 0;
+                if (active && meta >= 0) {
+                  const int sl = meta & 255;
+                  int vis;
+                  if (sl < 4) vis = sl == 0 ? vis0 : sl == 1 ? vis1 : sl == 2 ? vis2 : vis3;
+                  else vis = visrow[sl];
+                  t = min(max(vis - PASTA_PMETA_PAGE(meta) * PASTA_PAGE, 0), PASTA_PAGE);
+                }
+                thr[pg] = t;
+                full = full && (t == PASTA_PAGE);
               }
-              thr[pg] = t;
-              full = full && (t == PASTA_PAGE);
             }
           }
           if (!wait_or_abort(bar + 8 * (B_SFULL + b), (it >> 1) & 1, abort_flag)) { ok = false; break; }

@@ -24,6 +24,10 @@
 #define PASTA_TILE_PAGES 8          // pages per tensor-core tile (128 tokens)
 #define PASTA_PAGE 16               // tokens per page
 #define PASTA_MAX_ROWS 128          // rows of the stacked-query matrix (threads * group)
+// a page's meta word: bits 0-7 local stream, bits 8-29 page index within the stream, bit 30 set when every thread
+// of the t-request sees the whole page (no row needs a mask there); -1 marks an unused slot of a tile
+#define PASTA_PMETA_ALL_VISIBLE (1 << 30)
+#define PASTA_PMETA_PAGE(meta) (((meta) >> 8) & 0x3FFFFF)
 
 // header words
 enum {

@@ -115,13 +115,16 @@ pasta_status_t build_plan(const HostPool &pool, const std::vector<StepEntry> &en
       t.n_streams = n_shared;
       t.vis_off = static_cast<int32_t>(vis_tab.size());
       t.tq_off = static_cast<int32_t>(tq_tab.size());
-      for (const StreamUse &u : uses) {
+      for (size_t ui = 0; ui < uses.size(); ++ui) {
+        const StreamUse &u = uses[ui];
         if (u.local < 0) continue;
         const std::vector<int32_t> &sp = r->streams[u.stream].pages;
         const int32_t np = (u.max_vis + P - 1) / P;
+        int32_t min_vis = u.max_vis;             // what EVERY thread of the request sees of this stream
+        for (int32_t ti = 0; ti < T; ++ti) min_vis = std::min(min_vis, q_vis[ti][ui]);
         for (int32_t k = 0; k < np; ++k) {
           pages.push_back(sp[k]);
-          pmeta.push_back((k << 8) | u.local);
+          pmeta.push_back((k << 8) | u.local | ((k + 1) * P <= min_vis ? PASTA_PMETA_ALL_VISIBLE : 0));
         }
       }
       t.n_pages = static_cast<int32_t>(pages.size()) - t.page_off;

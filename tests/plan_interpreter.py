@@ -9,6 +9,7 @@ import numpy as np
  PH_OFF_PMETA, PH_OFF_VIS, PH_OFF_TQ, PH_OFF_APOS, PH_OFF_QPOS, PH_TOTAL_WORDS) = range(23)
 PQ, PT, PU, PW = 4, 6, 5, 4
 TILE_PAGES, PAGE = 8, 16
+STATS = {'flagged': 0, 'pages': 0}    # pages the plans marked as visible in full to every thread, of all pages walked
 
 
 def run_plan(w, K, V, q, n_kv_heads):
@@ -41,8 +42,11 @@ def run_plan(w, K, V, q, n_kv_heads):
                 s_all, v_all = [], []
                 for pi in range(tb * TILE_PAGES, min(te * TILE_PAGES, n_pages)):
                     page, meta = pages[page_off + pi], pmeta[page_off + pi]
-                    thr = vis[ti, meta & 255] - (meta >> 8) * PAGE
+                    thr = vis[ti, meta & 255] - ((meta >> 8) & 0x3FFFFF) * PAGE
                     cnt = int(np.clip(thr, 0, PAGE))
+                    if meta & (1 << 30):        # the plan claims that no row needs a mask on this page
+                        assert cnt == PAGE, (u, ti, pi)
+                    STATS['flagged'], STATS['pages'] = STATS['flagged'] + bool(meta & (1 << 30)), STATS['pages'] + 1
                     s_all.append(K[page, :cnt, g] @ q[tq[ti], h] * scale)
                     v_all.append(V[page, :cnt, g])
                 s = np.concatenate(s_all); v = np.concatenate(v_all)

@@ -91,3 +91,10 @@ def test_small_partial_budget_still_plans():
     script = cfg3_batched(4, 1, prefix_range=(300, 600))
     n = len(script.ops[-1][1])
     check_script(script, max_partial_rows=n * 32 * 2 + 160 * 128)
+
+
+def test_zz_all_visible_page_flag_is_exercised():
+    """The plans interpreted above marked some pages as visible in full to every thread (checked page by page in
+    plan_interpreter.run_plan) and left others unmarked."""
+    from plan_interpreter import STATS
+    assert 0 < STATS["flagged"] < STATS["pages"], STATS
