@@ -169,6 +169,55 @@ def build_state(script, device, seed_offset=0, grow_tokens=640):
     return pool, entries, randn
 
 
+def build_state_naive_rows(script, device, seed_offset=0, grow_tokens=640):
+    """The same set-up in the comparison layout of the paper's Appendix B: every thread a dense row of its own, the
+    main thread's row duplicated into each fork's row at spawn (paper_2502_11517_b200/naive_rows.py).  Returns the
+    pool, the final step's entries (one fork-less request per thread) and the bytes duplicated."""
+    import torch
+    from paper_2502_11517_b200 import binding
+    from paper_2502_11517_b200.naive_rows import NaiveRows
+    geo = script.geometry
+    entries = list(script.ops[-1][1])
+    n_rows = sum(op[0] in ("begin", "spawn") for op in script.ops)
+    main_len, own_len = {}, {}
+    for op in script.ops[:-1]:
+        if op[0] == "run":
+            (main_len if op[2] == 0 else own_len)[(op[1], op[2])] = (main_len if op[2] == 0 else own_len).get((op[1], op[2]), 0) + op[3]
+    longest = max(main_len.values()) + max(own_len.values(), default=0) + grow_tokens + 32
+    n_pages = n_rows * (longest // 16 + 2)
+    pool = binding.Pool(geo.n_layers, geo.n_q_heads, geo.n_kv_heads, geo.head_dim, n_pages, n_rows, 1, 4,
+                        max_step_queries=len(entries), max_layers_per_launch=geo.n_layers, device=device.index or 0)
+    gen = torch.Generator(device=device)
+    gen.manual_seed(script.seed + 977 * seed_offset)
+
+    def randn(shape):
+        return torch.randn(shape, generator=gen, device=device, dtype=torch.float32).to(torch.bfloat16)
+
+    rows = NaiveRows(pool)
+    for op in script.ops[:-1]:
+        kind = op[0]
+        if kind == "begin":
+            rows.begin(op[1])
+        elif kind == "spawn":
+            rows.spawn(op[1], op[2])
+        elif kind == "finish":
+            pass
+        elif kind == "merge":
+            rows.merge(op[1], [] if op[2] is None else list(op[2]))
+        elif kind == "run":
+            done = 0
+            while done < op[3]:
+                cnt = min(op[3] - done, 4096)
+                shape = (geo.n_layers, cnt, geo.n_kv_heads, geo.head_dim)
+                rows.run(op[1], op[2], cnt, randn(shape), randn(shape))
+                done += cnt
+        else:
+            raise ValueError(kind)
+    torch.cuda.synchronize(device)
+    row_entries = [(rows.row[(req, t)], 0, n) for req, t, n in entries]
+    return pool, row_entries, randn, rows.bytes_copied_at_spawn
+
+
 def unique_tokens(pool, entries):
     """Per request, the union of what the step's threads see (a shared prefix counts once); and the part of
     it that the tensor-core kernel reads: everything, for requests whose stacked query rows fit one MMA tile."""
@@ -213,8 +262,12 @@ def run_ours(args):
     script = make_script(args.workload, args.size)
     geo = script.geometry
     e2e_steps = max(3, min(args.steps, 50))
-    pool, entries, randn = build_state(script, device, seed_offset=rank,
-                                       grow_tokens=args.steps + max(args.warmup, 3) + e2e_steps + 3)
+    grow = args.steps + max(args.warmup, 3) + e2e_steps + 3
+    spawn_copy_bytes = None
+    if args.layout == "naive_rows":
+        pool, entries, randn, spawn_copy_bytes = build_state_naive_rows(script, device, seed_offset=rank, grow_tokens=grow)
+    else:
+        pool, entries, randn = build_state(script, device, seed_offset=rank, grow_tokens=grow)
     n = len(entries)
     reqs = [e[0] for e in entries]; thr = [e[1] for e in entries]
     ones = [1] * n
@@ -304,7 +357,7 @@ def run_ours(args):
         "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {
-            "workload": args.workload, "size": args.size, "script": script.name, "requests": len(set(reqs)), "thread_tokens_per_step": n,
+            "workload": args.workload, "size": args.size, "layout": args.layout, "script": script.name, "requests": len(set(reqs)), "thread_tokens_per_step": n,
             "layers": L, "n_q_heads": geo.n_q_heads, "n_kv_heads": geo.n_kv_heads, "head_dim": geo.head_dim,
             "page_size": geo.page_size, "unique_kv_tokens_per_layer": avg_tokens,
             "unique_kv_bytes_per_step": step_bytes, "l2": "inputs larger than L2" if step_bytes / L > 126e6 * 1.5 else
@@ -314,6 +367,7 @@ def run_ours(args):
             "kernel_ms_per_step": {"tensor": kernel_ms[0] / timed_steps, "warp": kernel_ms[1] / timed_steps,
                                    "merge": kernel_ms[2] / timed_steps, "steps_timed": timed_steps},
             "sync_merge_host_us": merge_us,
+            **({"bytes_duplicated_at_spawn": spawn_copy_bytes} if spawn_copy_bytes is not None else {}),
         },
         "clocks": clocks,
         "e2e": {"value": e2e_tokens / e2e_s, "unit": UNIT, "h2d_bytes_per_step": h2d,
@@ -321,7 +375,7 @@ def run_ours(args):
         "gpu_launches": launches,
         "roofline": {"bound": "hbm", "kernel": dom_name, "achieved": achieved, "peak": peak, "peak_kind": peak_kind,
                      "unit": "GB/s", "frac": achieved / peak, "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
-                     "traffic": NCU_TRAFFIC_BYTES.get((args.workload, args.size)) if dom == 0 else None, "bytes_per_launch": dom_bytes_per_launch,
+                     "traffic": NCU_TRAFFIC_BYTES.get((args.workload, args.size)) if dom == 0 and args.layout == "pool" else None, "bytes_per_launch": dom_bytes_per_launch,
                      "ms_per_launch": dom_ms},
         "cpu_baseline": oracle_sample(args.workload, budget_s=20.0) if world == 1 and not args.no_cpu_baseline else None,
     }
@@ -567,6 +621,9 @@ def main():
     ap.add_argument("--workload", default="long_shared_prefix")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--layout", default="pool", choices=["pool", "naive_rows"],
+                    help="pool: the library's shared paged pool (default).  naive_rows: the comparison layout of the "
+                         "paper's Appendix B (one dense row per thread, prefix duplicated), on the same kernels")
     ap.add_argument("--size", default="full", choices=["full", "small"],
                     help="small: a reduced copy of the workload for profiler captures (prefix 8192 / 4 layers)")
     args = ap.parse_args()
