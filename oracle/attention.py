@@ -81,14 +81,15 @@ def decode_attention(model: PoolModel, store: KVStore, queries: Sequence[Tuple[i
                      scale: Optional[float] = None, return_weights: bool = False):
     """Attention of one decode step for one layer.
 
-    queries: (request, thread) per row of q ([n, Hq, d]).  Returns out [n, Hq, d] fp64 and
+    queries: (request, thread) or (request, thread, hide) per row of q ([n, Hq, d]); hide = newest tokens of the
+    thread the query does not see (PoolModel.queries_of).  Returns out [n, Hq, d] fp64 and
     lse [n, Hq] fp64 (and the list of weight arrays when asked)."""
     q = _to_f32(q).astype(np.float64)
     out = np.empty(q.shape, dtype=np.float64)
     lse = np.empty(q.shape[:2], dtype=np.float64)
     weights: List[np.ndarray] = []
-    for i, (req, thread) in enumerate(queries):
-        k, v = store.gather(model.visible_slots(req, thread))
+    for i, qr in enumerate(queries):
+        k, v = store.gather(model.visible_slots(*qr))
         out[i], lse[i], w = attend(q[i], k, v, scale)
         if return_weights:
             weights.append(w)

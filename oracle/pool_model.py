@@ -25,7 +25,11 @@ What the paper leaves open, and the reading taken here:
     of one stream coalesced; a merged chunk with cut-off p goes immediately after the
     main-stream piece ending at p (splitting a piece if p is inside one), after chunks already
     placed at the same p with a smaller thread id and before those with a larger one;
-  * only the main thread spawns; merging an unfinished fork is an error (the interpreter waits).
+  * only the main thread spawns; merging an unfinished fork is an error (the interpreter waits);
+  * a thread may feed several tokens in one step (a chunk of the prompt; Section 3 "Efficiency" has the promise and
+    the <async> tag enter at one timestamp): every new token then issues its own query, which sees the thread's
+    view up to and including that token and none of the later ones, exactly as if the tokens had been fed in
+    successive steps.
 
 Position ids (Section 4, "Training a PASTA-SFT model", and Section 6 "Positional Embedding"): the main thread
 cannot know how long an asynchronous block will be, so it skips ahead by the length PREDICTED in the promise:
@@ -147,32 +151,50 @@ class PoolModel:
 
     # ------------------------------------------------------------------ appending
     def reserve(self, entries: Sequence[Tuple[int, int, int]]) -> List[Optional[Tuple[int, int]]]:
-        """One step: entries (req, thread, n_new) in order; returns the (page, offset) slot of every
-        appended token (None for attention-only entries).  All-or-nothing."""
+        """One step: entries (req, thread, n_new) in order; returns one element per QUERY: the (page, offset) slot
+        of each appended token, or None for the single query of an attention-only entry.  All-or-nothing."""
         seen = set()
         need = 0
         for req, thread, n_new in entries:
             r = self._req(req)
-            if thread not in r.state or (req, thread) in seen or n_new not in (0, 1):
+            if thread not in r.state or (req, thread) in seen or n_new < 0:
                 raise PoolError(INVALID_ARG, "bad step entry")
             if r.state[thread] != ACTIVE:
                 raise PoolError(INVALID_ARG, "thread is not active")
             seen.add((req, thread))
-            if n_new and r.stream_len[thread] % self.page_size == 0:
-                need += 1
+            n = r.stream_len[thread]
+            need += -(-(n + n_new) // self.page_size) - -(-n // self.page_size)
             if not n_new and not r.view[thread]:
                 raise PoolError(INVALID_ARG, "query with nothing visible")
             if n_new and not self._can_grow(r, thread):
                 raise PoolError(CAPACITY, "too many segments")
-        main_grows = {req for req, thread, n_new in entries if thread == 0 and n_new}
+        main_grows = {req: n_new for req, thread, n_new in entries if thread == 0 and n_new}
         for req, thread, n_new in entries:
             r = self.requests[req]
-            main_len = r.stream_len[0] + (1 if req in main_grows else 0)
+            main_len = r.stream_len[0] + main_grows.get(req, 0)
             if thread != 0 and r.cutoff[thread] > main_len:
                 raise PoolError(BAD_STATE, "the fork's promise is not in the pool")
         if need > len(self.free):
             raise PoolError(OUT_OF_PAGES, "pool exhausted")
-        return [self._append_one(req, thread) if n_new else None for req, thread, n_new in entries]
+        out: List[Optional[Tuple[int, int]]] = []
+        self.step_positions: List[int] = []          # position id of each query's token
+        for req, thread, n_new in entries:
+            if n_new == 0:
+                out.append(None)
+                self.step_positions.append(self.last_position(req, thread))
+            for _ in range(n_new):
+                out.append(self._append_one(req, thread))
+                self.step_positions.append(self.last_position(req, thread))
+        return out
+
+    @staticmethod
+    def queries_of(entries: Sequence[Tuple[int, int, int]]) -> List[Tuple[int, int, int]]:
+        """(req, thread, hide) per query of a step: `hide` = how many of the thread's newest tokens the query does
+        not see (the tokens of the same step that come after its own)."""
+        out = []
+        for req, thread, n_new in entries:
+            out.extend((req, thread, max(1, n_new) - 1 - j) for j in range(max(1, n_new)))
+        return out
 
     def append_run(self, req: int, thread: int, m: int) -> List[Tuple[int, int]]:
         r = self._req(req)
@@ -263,13 +285,16 @@ class PoolModel:
         r = self._req(req)
         return [(s, a, n) for s, a, n, _ in r.view[thread]]
 
-    def visible_slots(self, req: int, thread: int) -> List[Tuple[int, int]]:
-        """(page, offset) of every visible token, in logical order."""
+    def visible_slots(self, req: int, thread: int, hide: int = 0) -> List[Tuple[int, int]]:
+        """(page, offset) of every visible token, in logical order; `hide` newest tokens of the thread's own stream
+        left out (a query for an earlier one of several tokens fed in one step)."""
         r = self._req(req)
+        own_end = r.stream_len[thread] - hide
         out = []
         for s, a, n, _ in r.view[thread]:
             pages = r.stream_pages[s]
-            out.extend((pages[k // self.page_size], k % self.page_size) for k in range(a, a + n))
+            end = min(a + n, own_end) if s == thread else a + n
+            out.extend((pages[k // self.page_size], k % self.page_size) for k in range(a, end))
         return out
 
     def last_position(self, req: int, thread: int) -> int:

@@ -57,7 +57,7 @@ class OracleReplay:
                 store.write(slots, k, v)
         elif kind == "step":
             slots = [s for s in m.reserve(op[1]) if s is not None]
-            queries = [(e[0], e[1]) for e in op[1]]
+            queries = m.queries_of(op[1])
             result = {}
             for l, store in self.stores.items():
                 k, v, q = tensors[l] if tensors else step_tensors(self.script, op_index, l)

@@ -10,8 +10,9 @@ pool (the oracle's model or the CUDA library):
                                          fourth field is the block length predicted in the promise (position ids); a
                                          fifth field of 1 says that the promise is the main thread's next token, decoded
                                          but not appended yet
-    ("step",   ((req, thread, n_new), …)) one decode step: every listed thread appends n_new (0 or 1)
-                                         tokens and then issues one attention query
+    ("step",   ((req, thread, n_new), …)) one decode step: every listed thread appends n_new >= 0 tokens and issues
+                                         one attention query per new token (each blind to the later ones), or
+                                         one query over what it sees already when n_new == 0
     ("finish", req, thread)              a fork emitted </async>
     ("merge",  req, threads | None)      <sync/>: merge the named finished forks (None = all finished ones)
     ("end",    req)                      the request is over, its pages return to the pool
@@ -102,13 +103,14 @@ def run_tensors(script: Script, op_index: int, layer: int, device: str = "cpu"):
 def step_tensors(script: Script, op_index: int, layer: int, device: str = "cpu"):
     """(k_new, v_new, q) of the "step" operation `op_index` for one layer.
 
-    k_new, v_new: [number of entries with n_new == 1, Hkv, d]; q: [number of entries, Hq, d].
+    k_new, v_new: [number of appended tokens, Hkv, d]; q: [number of queries, Hq, d], where an entry
+    with n_new tokens contributes max(1, n_new) queries (one per new token, or one over the existing view).
     """
     op = script.ops[op_index]
     assert op[0] == "step"
     geo = script.geometry
     g = _gen(script.seed, op_index, layer, device)
-    n = len(op[1])
+    n = sum(max(1, e[2]) for e in op[1])
     n_app = sum(e[2] for e in op[1])
     k = _randn_bf16((n_app, geo.n_kv_heads, geo.head_dim), g, device)
     v = _randn_bf16((n_app, geo.n_kv_heads, geo.head_dim), g, device)
@@ -365,13 +367,15 @@ def cfg5_trace(n_requests: int = 256, n_steps: int = 512, n_layers: int = 32,
 
 # --------------------------------------------------------------------------- random small scripts (property tests)
 def random_script(seed: int, geo: Optional[Geometry] = None, n_ops: int = 60, max_requests: int = 3,
-                  max_forks: int = 5, paper_flow: bool = False, predictions: bool = False) -> Script:
+                  max_forks: int = 5, paper_flow: bool = False, predictions: bool = False,
+                  multi_token: bool = False) -> Script:
     """A random but valid operation sequence on a small pool.
 
     Exercises partial merges, merges of empty chunks, forks spawned after a merge, request reuse and
     steps mixing appending and attention-only entries.  With paper_flow=True the main thread always
     appends a token right after a merge before anything else happens to that request (the paper's
     <sync/> token), which is the situation the token-graph formulation of visibility describes.
+    With multi_token=True about a third of the appending entries feed 2 to 5 tokens in their step.
     """
     geo = geo or Geometry(1, 4, 2, 8, 4)
     rng = np.random.default_rng(seed)
@@ -389,12 +393,14 @@ def random_script(seed: int, geo: Optional[Geometry] = None, n_ops: int = 60, ma
                 n_new = 1 if (rng.random() < 0.8 or r["len"][t] == 0) else 0
                 if t == 0 and req in need_sync_token:
                     n_new = 1
+                if multi_token and n_new == 1 and rng.random() < 0.35:
+                    n_new = int(rng.integers(2, 6))
                 entries.append((req, t, n_new))
         order = rng.permutation(len(entries))
         entries = [entries[i] for i in order]
         for e in entries:
             book.add(e[0], e[1], e[2])
-            if e[1] == 0 and e[2] == 1:
+            if e[1] == 0 and e[2] >= 1:
                 need_sync_token.discard(e[0])
         ops.append(("step", tuple(entries)))
 

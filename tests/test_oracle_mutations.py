@@ -24,9 +24,11 @@ MUTATIONS = [
     ("pool_model.py", "r.cutoff[t] = r.stream_len[0]", "r.cutoff[t] = max(r.stream_len[0] - 1, 0)"),   # cut-off off by one
     ("pool_model.py", "if k % self.page_size == 0:", "if (k + 1) % self.page_size == 0 or not r.stream_pages[stream]:"),  # paging
     ("pool_model.py", "(anchor == p and s > t)", "(anchor == p and s < t)"),          # tie order of merged chunks
-    ("pool_model.py", "for k in range(a, a + n))", "for k in range(a, a + n - 1))"),  # last token of a piece dropped
+    ("pool_model.py", "for k in range(a, end))", "for k in range(a, end - 1))"),      # last token of a piece dropped
     ("pool_model.py", "self.free.insert(0, page)", "self.free.append(page)"),         # where freed pages go
     ("pool_model.py", "if s == 0 and a < p < a + ln:", "if s == 0 and a < p <= a + ln:"),   # split at a piece's end
+    ("pool_model.py", "own_end = r.stream_len[thread] - hide", "own_end = r.stream_len[thread]"),   # later tokens of the step seen
+    ("pool_model.py", "max(1, n_new) - 1 - j)", "j)"),                                 # hide counts from the wrong end
 ]
 
 
@@ -102,6 +104,20 @@ def _pins(O):
     r = m.request_begin(); m.append_run(r, 0, 4); f1 = m.thread_spawn(r); m.append_run(r, f1, 1); m.thread_finish(r, f1)
     m.sync_merge(r, [f1])
     assert m.view(r, 0) == [(0, 0, 4), (f1, 0, 1)]
+    # several tokens of a thread in one step = the same tokens one step at a time
+    rng = np.random.default_rng(11)
+    ms = [O.PoolModel(64, 4), O.PoolModel(64, 4)]
+    st = [O.KVStore(64, 4, 1, 4), O.KVStore(64, 4, 1, 4)]
+    k0, v0 = rng.standard_normal((5, 1, 4)), rng.standard_normal((5, 1, 4))
+    for mm, ss in zip(ms, st):
+        r = mm.request_begin(); ss.write(mm.append_run(r, 0, 5), k0, v0)
+    k, v, q = rng.standard_normal((3, 1, 4)), rng.standard_normal((3, 1, 4)), rng.standard_normal((3, 2, 4))
+    st[0].write(ms[0].reserve([(0, 0, 3)]), k, v)
+    out, _ = O.decode_attention(ms[0], st[0], O.PoolModel.queries_of([(0, 0, 3)]), q)
+    for j in range(3):
+        st[1].write(ms[1].reserve([(0, 0, 1)]), k[j:j + 1], v[j:j + 1])
+        o1, _ = O.decode_attention(ms[1], st[1], [(0, 0)], q[j:j + 1])
+        np.testing.assert_allclose(out[j], o1[0], rtol=0, atol=1e-12)
 
 
 def test_unmodified_copy_passes_every_pin():

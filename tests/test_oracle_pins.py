@@ -304,3 +304,43 @@ def test_config2_shapes():
         total = sum(n for _, _, n in view)
         assert total == 769 + sum(script.notes["chunks"])
         assert [s for s, _, _ in view if s != 0] == [1, 2, 3, 4]
+
+
+# ------------------------------------------------------------------ several tokens of one thread in one step
+@pytest.mark.parametrize("seed", range(6))
+def test_multi_token_step_equals_successive_single_token_steps(seed):
+    """A step in which threads feed several tokens must give every new token the attention output it would get
+    if the tokens were fed one step at a time (causal among the new tokens)."""
+    from oracle import KVStore, PoolModel, decode_attention
+    rng = np.random.default_rng(500 + seed)
+    Hq, Hkv, d, P = 4, 2, 8, 4
+    models = [PoolModel(64, P), PoolModel(64, P)]
+    stores = [KVStore(64, P, Hkv, d), KVStore(64, P, Hkv, d)]
+
+    def feed(which, entries, k, v, q):
+        slots = [s for s in models[which].reserve(entries) if s is not None]
+        stores[which].write(slots, k, v)
+        return decode_attention(models[which], stores[which], PoolModel.queries_of(entries), q)
+
+    for which in (0, 1):                                 # same history on both: a prompt, two forks with some tokens
+        m = models[which]
+        g = np.random.default_rng(900 + seed)
+        r = m.request_begin()
+        n0 = int(g.integers(1, 9))
+        stores[which].write(m.append_run(r, 0, n0), g.standard_normal((n0, Hkv, d)), g.standard_normal((n0, Hkv, d)))
+        for _ in range(2):
+            t = m.thread_spawn(r)
+            n1 = int(g.integers(0, 6))
+            stores[which].write(m.append_run(r, t, n1), g.standard_normal((n1, Hkv, d)), g.standard_normal((n1, Hkv, d)))
+    entries = [(0, 1, int(rng.integers(2, 6))), (0, 0, int(rng.integers(1, 6))), (0, 2, int(rng.integers(0, 4)))]
+    n_app = sum(e[2] for e in entries); n_q = sum(max(1, e[2]) for e in entries)
+    k = rng.standard_normal((n_app, Hkv, d)); v = rng.standard_normal((n_app, Hkv, d)); q = rng.standard_normal((n_q, Hq, d))
+    out, lse = feed(0, entries, k, v, q)
+    ai = qi = 0
+    for req, t, n in entries:
+        for j in range(max(1, n)):
+            nn = 1 if n else 0
+            o1, l1 = feed(1, [(req, t, nn)], k[ai:ai + nn], v[ai:ai + nn], q[qi:qi + 1])
+            assert np.abs(o1[0] - out[qi]).max() < 1e-12 and np.abs(l1[0] - lse[qi]).max() < 1e-12, (req, t, j)
+            ai += nn; qi += 1
+    assert models[0].dump() == models[1].dump()

@@ -104,7 +104,7 @@ def test_errors_leave_the_pool_unchanged():
     with pytest.raises(PoolError) as e:
         m.sync_merge(r, [t])                     # still decoding: the interpreter has to wait
     assert e.value.code == BAD_STATE and m.dump() == before
-    for bad in ([(r, 0, 1), (r, 0, 1)], [(r, 9, 1)], [(7, 0, 1)], [(r, 0, 2)]):
+    for bad in ([(r, 0, 1), (r, 0, 1)], [(r, 9, 1)], [(7, 0, 1)], [(r, 0, -1)]):
         with pytest.raises(PoolError) as e:
             m.reserve(bad)
         assert e.value.code == INVALID_ARG and m.dump() == before
@@ -230,3 +230,39 @@ def test_merging_a_fork_whose_promise_never_arrived_is_refused():
     with pytest.raises(PoolError) as e:
         m.sync_merge(req, [t])
     assert e.value.code == BAD_STATE and m.dump() == before
+
+
+# ------------------------------------------------------------------ several tokens of one thread in one step
+@pytest.mark.parametrize("seed", range(8))
+def test_multi_token_entry_equals_single_token_steps(seed):
+    a, b, rng = _random_state(seed)
+    for req in sorted(a.requests):
+        threads = [0] + [t for t, st in a.requests[req].state.items() if t != 0 and st == 0]
+        entries = [(req, t, int(rng.integers(0, 6))) for t in threads if a.requests[req].view[t] or t == 0]
+        entries = [(r, t, max(n, 1) if not a.requests[r].view[t] else n) for r, t, n in entries]
+        got = a.reserve(entries)
+        want, want_pos = [], []
+        for r, t, n in entries:                       # the same tokens, one step each, in the same order
+            if n == 0:
+                want += b.reserve([(r, t, 0)]); want_pos += b.step_positions
+            for _ in range(n):
+                want += b.reserve([(r, t, 1)]); want_pos += b.step_positions
+        assert got == want and a.step_positions == want_pos
+        assert a.dump() == b.dump()
+        # query j of an entry sees what the thread saw right after its j-th token went in: everything but the later ones
+        for (r, t, hide) in PoolModel.queries_of(entries):
+            full = a.visible_slots(r, t)
+            assert a.visible_slots(r, t, hide) == [s for s in full if s not in set(full[len(full) - hide:])] if hide else full
+
+
+def test_multi_token_page_count_and_refusal():
+    m = PoolModel(3, 4)
+    r = m.request_begin()
+    m.append_run(r, 0, 3)
+    before = m.dump()
+    with pytest.raises(PoolError) as e:
+        m.reserve([(r, 0, 10)])                        # tokens 3..12 need pages 1, 2 and 3: only two are left
+    assert e.value.code == OUT_OF_PAGES and m.dump() == before
+    slots = m.reserve([(r, 0, 9)])                     # tokens 3..11: pages 1 and 2
+    assert len(slots) == 9 and len(m.free) == 0
+    assert PoolModel.queries_of([(r, 0, 3), (r, 1, 0), (r, 2, 1)]) == [(r, 0, 2), (r, 0, 1), (r, 0, 0), (r, 1, 0), (r, 2, 0)]
