@@ -136,9 +136,17 @@ pasta_status_t pasta_sync_merge(pasta_pool_t *pool, int32_t req, int32_t n_threa
 /*
  * Reserves the pool slot of every token appended in this step and plans the attention of the
  * step.  Entry i is thread thread_ids[i] of request req_ids[i] (host arrays, n entries, each
- * thread at most once, ACTIVE threads only) and appends n_new[i] tokens (0 or 1; NULL = all 1).
+ * thread at most once, ACTIVE threads only) and appends n_new[i] >= 0 tokens (NULL = all 1).
  * Pages are taken in list order, one whenever a stream's token index is a multiple of 16.
  * An entry that would see nothing (no visible token and n_new == 0) is INVALID_ARG.
+ * QUERIES.  An entry with n_new <= 1 issues one attention query (for its new token, or over what the thread
+ * sees already).  An entry with n_new = m > 1 (several tokens of one thread fed in one step: a prompt chunk, a
+ * promise together with what follows it) issues m queries, one per new token in order, each seeing the
+ * thread's view up to and including its own token and none of the later ones — causal attention among the new
+ * tokens, the same results as m steps of one token.  The step's queries are numbered in entry order; every
+ * per-query array of the calls below (q, out, lse, slots, positions) has one row per query, and k_new / v_new
+ * one row per appended token in the same order.  The number of queries is bounded by max_step_queries
+ * (CAPACITY, nothing reserved).
  * If the bookkeeping succeeds but the step cannot be planned within the pool's capacities, the call
  * returns CAPACITY with the tokens already reserved (the one exception to "unchanged on failure").
  * The plan is uploaded on `stream`; it is used by the pasta_kv_append and pasta_decode_attn calls
@@ -147,13 +155,13 @@ pasta_status_t pasta_sync_merge(pasta_pool_t *pool, int32_t req, int32_t n_threa
 pasta_status_t pasta_step_begin(pasta_pool_t *pool, int32_t n, const int32_t *req_ids,
                                 const int32_t *thread_ids, const int32_t *n_new, void *stream);
 
-/* (page, offset) reserved by the last pasta_step_begin for each of its entries, two int32 per
- * entry, (-1, -1) for entries with n_new == 0.  Host array of 2 * n entries. */
-pasta_status_t pasta_step_slots(pasta_pool_t *pool, int32_t *out_slots, int32_t capacity_entries);
+/* (page, offset) reserved by the last pasta_step_begin for the token of each of its queries, two int32 per
+ * query, (-1, -1) for the query of an entry with n_new == 0.  Host array; capacity in queries (CAPACITY if
+ * smaller than the step's number of queries). */
+pasta_status_t pasta_step_slots(pasta_pool_t *pool, int32_t *out_slots, int32_t capacity_queries);
 
-/* Position id of each entry's newest token (the one its query belongs to) for the last pasta_step_begin.
- * Host array of n entries. */
-pasta_status_t pasta_step_positions(pasta_pool_t *pool, int32_t *out_pos, int32_t capacity_entries);
+/* Position id of each query's token for the last pasta_step_begin.  Host array; capacity in queries. */
+pasta_status_t pasta_step_positions(pasta_pool_t *pool, int32_t *out_pos, int32_t capacity_queries);
 
 /*
  * pasta_kv_append with rotary position embedding fused in: every new K vector is rotated by its token's
@@ -213,6 +221,7 @@ pasta_status_t pasta_kv_append_run_rope(pasta_pool_t *pool, int32_t req, int32_t
  * host bf16 [n_layers, n_app, n_kv_heads, head_dim]; q: host bf16 [n_layers, n, n_q_heads, head_dim];
  * out: host fp32 like q.  staging: device scratch of at least pasta_step_host_bytes(pool, n)
  * bytes, caller-owned.  Pinned host memory makes the copies asynchronous; pageable works too.
+ * Entries append at most one token each here (n_new[i] > 1: INVALID_ARG, nothing reserved).
  */
 pasta_status_t pasta_step_host_bytes(pasta_pool_t *pool, int32_t n, size_t *out);
 pasta_status_t pasta_step_host(pasta_pool_t *pool, int32_t n, const int32_t *req_ids,

@@ -179,7 +179,8 @@ class Pool:
         nn = None if n_new is None else _i32(n_new)
         st = C.c_void_p(0) if self.host_only else _stream(stream)
         _check(lib().pasta_step_begin(self._h, len(r), _ptr(r), _ptr(t), _ptr(nn), st), "pasta_step_begin")
-        self._last_n = len(r)
+        # queries of the step: one per entry, or one per new token of an entry that appends several
+        self._last_n = len(r) if nn is None else int(np.maximum(nn, 1).sum())
 
     def step_slots(self) -> np.ndarray:
         out = np.empty((self._last_n, 2), dtype=np.int32)

@@ -77,8 +77,8 @@ struct pasta_pool {
   cudaEvent_t pinned_free[kStaging] = {nullptr, nullptr, nullptr, nullptr};
   int next_pinned = 0;
   int32_t *status_host = nullptr;     // pinned, one word
-  std::vector<StepEntry> entries;
-  std::vector<Slot> slots;
+  std::vector<StepQuery> queries;   // of the step planned last, in entry order
+  std::vector<Slot> slots;          // parallel to queries
   std::vector<int32_t> plan;
   PlanHeader hdr{};
   bool plan_valid = false;
@@ -324,16 +324,22 @@ pasta_status_t pasta_sync_merge(pasta_pool_t *p, int32_t req, int32_t n_threads,
 pasta_status_t pasta_step_begin(pasta_pool_t *p, int32_t n, const int32_t *req_ids, const int32_t *thread_ids,
                                 const int32_t *n_new, void *stream) {
   if (!p || n < 0 || (n > 0 && (!req_ids || !thread_ids))) return PASTA_ERR_INVALID_ARG;
-  if (n > p->d.max_queries) return PASTA_ERR_CAPACITY;
   std::vector<StepEntry> entries(n);
-  for (int32_t i = 0; i < n; ++i) entries[i] = StepEntry{req_ids[i], thread_ids[i], n_new ? n_new[i] : 1};
+  int64_t n_queries = 0;
+  for (int32_t i = 0; i < n; ++i) {
+    entries[i] = StepEntry{req_ids[i], thread_ids[i], n_new ? n_new[i] : 1};
+    if (entries[i].n_new < 0) return PASTA_ERR_INVALID_ARG;
+    n_queries += std::max(1, entries[i].n_new);
+  }
+  if (n_queries > p->d.max_queries) return PASTA_ERR_CAPACITY;
   std::vector<Slot> slots;
-  pasta_status_t s = p->host.reserve_step(entries, &slots);
+  std::vector<StepQuery> queries;
+  pasta_status_t s = p->host.reserve_step(entries, &queries, &slots);
   if (s != PASTA_OK) return s;
   p->plan_valid = false;
-  p->entries.swap(entries);
+  p->queries.swap(queries);
   p->slots.swap(slots);
-  s = build_plan(p->host, p->entries, p->slots, limits_of(p), &p->plan);
+  s = build_plan(p->host, p->queries, p->slots, limits_of(p), &p->plan);
   if (s != PASTA_OK) return s;   // the tokens stay reserved; only the attention of this step cannot be planned
   std::memcpy(p->hdr.w, p->plan.data(), sizeof(p->hdr.w));
   if (!p->host_only) {
@@ -490,6 +496,9 @@ pasta_status_t pasta_step_host(pasta_pool_t *p, int32_t n, const int32_t *req_id
   if (s != PASTA_OK) return s;
   if (staging_bytes < need || (reinterpret_cast<uintptr_t>(staging) & 255)) return PASTA_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (n_new)
+    for (int32_t i = 0; i < n; ++i)
+      if (n_new[i] > 1) return PASTA_ERR_INVALID_ARG;   // the staging layout is one query per entry
   s = pasta_step_begin(p, n, req_ids, thread_ids, n_new, stream);
   if (s != PASTA_OK) return s;
   const size_t L = p->cfg.n_layers, d = p->cfg.head_dim;

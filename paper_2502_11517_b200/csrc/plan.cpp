@@ -30,7 +30,7 @@ struct TUnit {
 
 }  // namespace
 
-pasta_status_t build_plan(const HostPool &pool, const std::vector<StepEntry> &entries,
+pasta_status_t build_plan(const HostPool &pool, const std::vector<StepQuery> &entries,
                           const std::vector<Slot> &slots, const PlanLimits &lim,
                           std::vector<int32_t> *out) {
   const int32_t n = static_cast<int32_t>(entries.size());
@@ -76,6 +76,9 @@ pasta_status_t build_plan(const HostPool &pool, const std::vector<StepEntry> &en
       const Thread &th = r->threads[entries[qs[ti]].thread];
       vis_of.assign(n_streams_all, 0);
       for (const Seg &s : th.view) vis_of[s.stream] = std::max(vis_of[s.stream], s.start + s.len);
+      // a query for an earlier one of several tokens appended in this step does not see the later ones: they are
+      // the end of the thread's own stream (stream id = thread id)
+      vis_of[entries[qs[ti]].thread] -= entries[qs[ti]].hide;
       for (const Seg &s : th.view) {
         if (use_index[s.stream] < 0) {
           use_index[s.stream] = static_cast<int32_t>(uses.size());
@@ -250,7 +253,7 @@ pasta_status_t build_plan(const HostPool &pool, const std::vector<StepEntry> &en
 
   // ---- assemble
   int32_t n_app = 0;
-  for (const StepEntry &e : entries) n_app += e.n_new;
+  for (const Slot &s : slots) n_app += s.page >= 0;
   std::vector<int32_t> &w = *out;
   w.assign(PH_WORDS, 0);
   auto put = [&](int off_field, const std::vector<int32_t> &v) {
@@ -260,9 +263,9 @@ pasta_status_t build_plan(const HostPool &pool, const std::vector<StepEntry> &en
   };
   std::vector<int32_t> app, apos, qpos;
   for (int32_t i = 0; i < n; ++i) {
-    const int32_t pos = HostPool::query_position(pool.request(entries[i].req)->threads[entries[i].thread]);   // the newest token
+    const int32_t pos = slots[i].pos;
     qpos.push_back(pos);
-    if (entries[i].n_new) { app.push_back(slots[i].page); app.push_back(slots[i].offset); apos.push_back(pos); }
+    if (slots[i].page >= 0) { app.push_back(slots[i].page); app.push_back(slots[i].offset); apos.push_back(pos); }
   }
   std::vector<int32_t> qtab(static_cast<size_t>(n) * PQ_WORDS);
   for (int32_t i = 0; i < n; ++i) {

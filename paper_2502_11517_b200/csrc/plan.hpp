@@ -9,15 +9,15 @@ namespace pasta {
 
 struct PlanLimits {
   int32_t n_q_heads, n_kv_heads, head_dim;
-  int32_t max_queries;   // step entries
+  int32_t max_queries;   // queries of a step
   int32_t max_rows;      // partial rows per layer
   int64_t max_words;     // size of the device copy of the plan
   int32_t grid;          // CTAs the tensor-core kernel may use (one per SM)
   bool tensor_path;      // false: every stream goes to the warp-shuffle kernel
 };
 
-// Plans the attention of one step.  `slots` are the slots reserved for the entries.
-pasta_status_t build_plan(const HostPool &pool, const std::vector<StepEntry> &entries,
+// Plans the attention of one step: one query per element of `queries`, `slots` parallel to it.
+pasta_status_t build_plan(const HostPool &pool, const std::vector<StepQuery> &queries,
                           const std::vector<Slot> &slots, const PlanLimits &lim,
                           std::vector<int32_t> *words);
 

@@ -109,7 +109,7 @@ Slot HostPool::append_one(Request &r, int32_t thread) {
     s.pages.push_back(free_.front());
     free_.pop_front();
   }
-  Slot slot{s.pages[k / page_size_], k % page_size_};
+  Slot slot{s.pages[k / page_size_], k % page_size_, 0};
   s.len = k + 1;
   Thread &th = r.threads[thread];
   th.pos_last = th.pos_next;
@@ -123,7 +123,8 @@ Slot HostPool::append_one(Request &r, int32_t thread) {
   return slot;
 }
 
-pasta_status_t HostPool::reserve_step(const std::vector<StepEntry> &entries, std::vector<Slot> *slots) {
+pasta_status_t HostPool::reserve_step(const std::vector<StepEntry> &entries, std::vector<StepQuery> *queries,
+                                      std::vector<Slot> *slots) {
   // pass 1: validate everything, count pages
   size_t need = 0;
   std::vector<std::pair<int32_t, int32_t>> seen;
@@ -132,7 +133,7 @@ pasta_status_t HostPool::reserve_step(const std::vector<StepEntry> &entries, std
     Request *r = live(e.req);
     if (!r) return PASTA_ERR_INVALID_ARG;
     if (e.thread < 0 || e.thread >= static_cast<int32_t>(r->threads.size())) return PASTA_ERR_INVALID_ARG;
-    if (e.n_new != 0 && e.n_new != 1) return PASTA_ERR_INVALID_ARG;
+    if (e.n_new < 0) return PASTA_ERR_INVALID_ARG;
     seen.emplace_back(e.req, e.thread);
   }
   {
@@ -145,7 +146,10 @@ pasta_status_t HostPool::reserve_step(const std::vector<StepEntry> &entries, std
     Request *r = live(e.req);
     const Thread &t = r->threads[e.thread];
     if (t.state != PASTA_THREAD_ACTIVE) return PASTA_ERR_INVALID_ARG;
-    if (e.n_new && r->streams[e.thread].len % page_size_ == 0) ++need;
+    if (e.n_new) {   // pages opened by tokens len .. len + n_new - 1
+      const int64_t len = r->streams[e.thread].len, P = page_size_;
+      need += static_cast<size_t>((len + e.n_new + P - 1) / P - (len + P - 1) / P);
+    }
     if (!e.n_new && t.view.empty()) return PASTA_ERR_INVALID_ARG;
     if (e.n_new && !can_extend(*r, e.thread)) return PASTA_ERR_CAPACITY;
   }
@@ -155,16 +159,27 @@ pasta_status_t HostPool::reserve_step(const std::vector<StepEntry> &entries, std
     int32_t main_len = r->streams[0].len;
     if (r->threads[e.thread].cutoff > main_len) {
       for (const StepEntry &o : entries)
-        if (o.req == e.req && o.thread == 0 && o.n_new) { ++main_len; break; }
+        if (o.req == e.req && o.thread == 0 && o.n_new) { main_len += o.n_new; break; }
       if (r->threads[e.thread].cutoff > main_len) return PASTA_ERR_BAD_STATE;
     }
   }
   if (need > free_.size()) return PASTA_ERR_OUT_OF_PAGES;
   // pass 2: commit
   slots->clear();
-  slots->reserve(entries.size());
-  for (const StepEntry &e : entries)
-    slots->push_back(e.n_new ? append_one(requests_[e.req], e.thread) : Slot{-1, -1});
+  queries->clear();
+  for (const StepEntry &e : entries) {
+    Request &r = requests_[e.req];
+    if (e.n_new == 0) {
+      slots->push_back(Slot{-1, -1, query_position(r.threads[e.thread])});
+      queries->push_back(StepQuery{e.req, e.thread, 0});
+    }
+    for (int32_t j = 0; j < e.n_new; ++j) {
+      Slot s = append_one(r, e.thread);
+      s.pos = r.threads[e.thread].pos_last;
+      slots->push_back(s);
+      queries->push_back(StepQuery{e.req, e.thread, e.n_new - 1 - j});
+    }
+  }
   return PASTA_OK;
 }
 

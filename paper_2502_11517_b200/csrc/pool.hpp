@@ -47,8 +47,16 @@ struct StepEntry {
   int32_t req, thread, n_new;
 };
 
+// One attention query of a step.  An entry that appends m >= 1 tokens issues m queries, one per new token, each
+// blind to the tokens appended after its own (`hide` = how many of the thread's newest tokens it may not see);
+// an entry that appends nothing issues one query over what the thread sees already.
+struct StepQuery {
+  int32_t req, thread, hide;
+};
+
 struct Slot {
-  int32_t page, offset;
+  int32_t page, offset;   // {-1, -1} for a query without a new token
+  int32_t pos;            // position id of the query's token
 };
 
 class HostPool {
@@ -68,8 +76,10 @@ class HostPool {
   pasta_status_t thread_finish(int32_t req, int32_t thread);
   pasta_status_t sync_merge(int32_t req, int32_t n_threads, const int32_t *thread_ids);
 
-  // Validates the whole step first, then reserves; slots[i] = {-1,-1} when n_new == 0.
-  pasta_status_t reserve_step(const std::vector<StepEntry> &entries, std::vector<Slot> *slots);
+  // Validates the whole step first, then reserves.  Outputs one element per QUERY, in entry order (an entry with
+  // n_new tokens contributes max(1, n_new) of them).
+  pasta_status_t reserve_step(const std::vector<StepEntry> &entries, std::vector<StepQuery> *queries,
+                              std::vector<Slot> *slots);
   pasta_status_t reserve_run(int32_t req, int32_t thread, int32_t m, std::vector<Slot> *slots);
 
   const Request *request(int32_t req) const;

@@ -68,8 +68,8 @@ def _oracle_slots(ora, op):
         if not n_new:
             out.append(None); continue
         r = ora.model.requests[req]
-        k = r.stream_len[t] - 1
-        out.append((r.stream_pages[t][k // 16], k % 16))
+        for k in range(r.stream_len[t] - n_new, r.stream_len[t]):     # one slot per new token
+            out.append((r.stream_pages[t][k // 16], k % 16))
     return out
 
 
@@ -140,6 +140,23 @@ def test_config5_trace_reduced(lib):
 def test_random_scripts(lib, seed):
     geo = Geometry(1, 8, 2, 128, 16) if seed % 2 else Geometry(1, 4, 2, 64, 16)
     run_script(lib, random_script(40 + seed, n_ops=70, geo=geo))
+
+
+@pytest.mark.parametrize("seed", range(4))
+def test_random_scripts_with_several_tokens_per_entry(lib, seed):
+    geo = Geometry(1, 8, 2, 128, 16) if seed % 2 else Geometry(1, 4, 2, 64, 16)
+    run_script(lib, random_script(60 + seed, n_ops=70, geo=geo, multi_token=True))
+
+
+def test_prompt_fed_in_chunks(lib):
+    """Chunked prefill: a 300-token prompt fed 30 tokens per step (120 stacked rows on the tensor-core path), then two
+    forks and the main thread feeding 3, 1 and 5 tokens in one step."""
+    from pasta_workloads import Script
+    geo = Geometry(2, 32, 8, 128, 16)
+    ops = [("begin", 0), ("run", 0, 0, 1)] + [("step", ((0, 0, 30),)) for _ in range(10)]
+    ops += [("spawn", 0, 1), ("spawn", 0, 2), ("run", 0, 1, 20), ("step", ((0, 1, 3), (0, 2, 1), (0, 0, 5)))]
+    script = Script("chunked_prefill", geo, 64, np.arange(64, dtype=np.int32), 2, 4, 8, 7, ops)
+    run_script(lib, script)
 
 
 def test_page_placement_does_not_change_the_result(lib):

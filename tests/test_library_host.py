@@ -59,6 +59,11 @@ def test_bookkeeping_matches_oracle_on_configs(maker):
     _same_state(maker())
 
 
+@pytest.mark.parametrize("seed", range(6))
+def test_bookkeeping_matches_oracle_with_several_tokens_per_entry(seed):
+    _same_state(random_script(100 + seed, n_ops=90, geo=Geometry(1, 4, 2, 64, 16), multi_token=True))
+
+
 def test_bookkeeping_matches_oracle_on_a_trace():
     _same_state(cfg5_trace(12, 160, 1, prompt_range=(16, 200), p_promise=0.08, mean_chunk=20.0), every_op=False)
     _same_state(cfg5_trace(6, 120, 1, prompt_range=(16, 100), p_promise=0.1, mean_chunk=15.0, overlap=True))
@@ -90,7 +95,7 @@ def test_error_codes_match_and_leave_state_unchanged():
         (lambda: pool.step_begin([0, 0], [0, 0]), lambda: m.reserve([(0, 0, 1), (0, 0, 1)])),
         (lambda: pool.step_begin([0], [7]), lambda: m.reserve([(0, 7, 1)])),
         (lambda: pool.step_begin([1], [0]), lambda: m.reserve([(1, 0, 1)])),
-        (lambda: pool.step_begin([0], [0], [2]), lambda: m.reserve([(0, 0, 2)])),
+        (lambda: pool.step_begin([0], [0], [-1]), lambda: m.reserve([(0, 0, -1)])),
         (lambda: pool.thread_finish(0, 0), lambda: m.thread_finish(0, 0)),
         (lambda: pool.thread_finish(0, 5), lambda: m.thread_finish(0, 5)),
         (lambda: pool.request_end(1), lambda: m.request_end(1)),
@@ -182,16 +187,15 @@ def test_pending_spawn_matches_oracle(seed):
             if code == 0:
                 live.append(max(model.requests[req].state))
         elif what == 1:
-            entries = [(req, 0, 1)] if rng.integers(0, 2) else []
-            entries += [(req, t, int(rng.integers(0, 2))) for t in live if rng.integers(0, 2)]
+            entries = [(req, 0, int(rng.integers(1, 4)))] if rng.integers(0, 2) else []
+            entries += [(req, t, int(rng.integers(0, 4))) for t in live if rng.integers(0, 2)]
             if not entries:
                 continue
             a, b = _codes(lambda: pool.step_begin(*zip(*entries)), lambda: model.reserve(entries))
             assert a == b, (entries, a, b)
             assert pool.dump() == model.dump()
             if a == 0:
-                want = [model.last_position(r, t) for r, t, _n in entries]
-                assert pool.step_positions().tolist() == want
+                assert pool.step_positions().tolist() == model.step_positions
         elif what == 2 and live:
             both("kv_append_run", "append_run", req, live[int(rng.integers(0, len(live)))], int(rng.integers(0, 20)))
         elif what == 3 and live:

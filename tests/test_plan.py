@@ -41,8 +41,8 @@ def check_script(script, flags=0, steps=None, **kw):
             lib.apply(i)
             k, v, q = step_tensors(script, i, 0)
             j = 0
-            for e, s in zip(op[1], lib.last_slots):
-                if e[2]:
+            for s in lib.last_slots:                  # one slot per query; (-1, -1) where nothing was appended
+                if s[0] >= 0:
                     K[s[0], s[1]] = _f64(k[j]); V[s[0], s[1]] = _f64(v[j]); j += 1
             if steps is not None and i not in steps:
                 ora.apply(i, attend=False)
@@ -70,6 +70,12 @@ def test_plan_on_random_scripts_d64(seed):
 @pytest.mark.parametrize("flags", [0, binding.FLAG_NO_TENSOR_PATH])
 def test_plan_on_random_scripts_d128(seed, flags):
     check_script(random_script(seed, n_ops=70, geo=Geometry(1, 8, 2, 128, 16)), flags=flags)
+
+
+@pytest.mark.parametrize("seed", range(20, 28))
+def test_plan_with_several_tokens_per_entry(seed):
+    geo = Geometry(1, 8, 2, 128, 16) if seed % 2 else Geometry(1, 4, 2, 64, 16)
+    check_script(random_script(seed, n_ops=70, geo=geo, multi_token=True))
 
 
 @pytest.mark.parametrize("maker", [cfg1_tiny, lambda: cfg1_tiny("cutoffs"), lambda: cfg1_tiny("append"),
