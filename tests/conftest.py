@@ -12,4 +12,4 @@ if TESTS not in sys.path:
 
 
 def pytest_configure(config):
-    config.addinivalue_line("markers", "gpu: needs a CUDA device (run on the GPU box)")
+    config.addinivalue_line("markers", "gpu: needs a CUDA device")

@@ -1,0 +1,82 @@
+"""GPU parity on the edges of the method and of the kernels' limits: empty steps, one-token contexts, ragged page
+and tile boundaries, exactly as many stacked rows as the tensor-core tile holds and one thread more, every supported
+group size, more streams than the tensor-core path takes, forks with empty chunks."""
+import numpy as np
+import pytest
+
+from pasta_workloads import Geometry, Script
+from test_gpu_parity import lib, run_script  # noqa: F401  (fixture + helper)
+
+pytestmark = pytest.mark.gpu
+
+
+def manual(ops, geo, n_pages=256, max_threads=40, max_segments=8, max_requests=2):
+    return Script("manual", geo, n_pages, np.random.default_rng(3).permutation(n_pages).astype(np.int32),
+                  max_requests, max_threads, max_segments, 31, list(ops))
+
+
+def test_empty_step(lib):
+    import torch
+    pool = lib.Pool(1, 8, 2, 128, 8, 1, 2, 2)
+    pool.step_begin([], [], [])
+    q = torch.empty((1, 0, 8, 128), dtype=torch.bfloat16, device="cuda")
+    out = torch.empty((1, 0, 8, 128), dtype=torch.float32, device="cuda")
+    pool.kv_append(q[:, :, :2], q[:, :, :2])
+    pool.decode_attn(q, out)
+    torch.cuda.synchronize()
+    assert pool.status() == 0
+    pool.close()
+
+
+@pytest.mark.parametrize("prefix", [1, 15, 16, 17, 127, 128, 129, 255, 257])
+def test_ragged_prefix_lengths(lib, prefix):
+    geo = Geometry(1, 32, 8, 128, 16)
+    ops = [("begin", 0), ("run", 0, 0, prefix), ("spawn", 0, 1), ("spawn", 0, 2), ("run", 0, 2, 17),
+           ("step", ((0, 0, 1), (0, 1, 0), (0, 2, 1))),       # fork 1 has an empty chunk and only reads the prefix
+           ("step", ((0, 1, 1), (0, 2, 0)))]
+    run_script(lib, manual(ops, geo))
+
+
+@pytest.mark.parametrize("n_forks,tensor_units", [(31, True), (32, False)])
+def test_as_many_rows_as_the_tile_holds_and_one_thread_more(lib, n_forks, tensor_units):
+    geo = Geometry(1, 32, 8, 128, 16)                          # group 4: 32 threads fill the 128 rows
+    ops = [("begin", 0), ("run", 0, 0, 300)]
+    for t in range(1, n_forks + 1):
+        ops += [("spawn", 0, t), ("run", 0, t, 3 + t % 5)]
+    ops.append(("step", tuple((0, t, 1) for t in range(n_forks + 1))))
+    script = manual(ops, geo, n_pages=256, max_threads=40)
+    from lib_replay import LibReplay, make_pool
+    pool = make_pool(script, host_only=True, max_step_queries=64)
+    rep = LibReplay(script, pool)
+    for i in range(len(script.ops)):
+        rep.apply(i)
+    w = pool.plan_words()
+    assert (w[4] > 0) == tensor_units and (w[5] > 0) == (not tensor_units)     # t-units / w-units of the plan
+    pool.close()
+    run_script(lib, script, max_step_queries=64)
+
+
+@pytest.mark.parametrize("hq,hkv,d", [(8, 8, 128), (8, 4, 128), (16, 2, 128), (8, 8, 64), (16, 2, 64)])
+def test_group_sizes(lib, hq, hkv, d):
+    geo = Geometry(2, hq, hkv, d, 16)
+    ops = [("begin", 0), ("run", 0, 0, 200), ("spawn", 0, 1), ("run", 0, 0, 40), ("spawn", 0, 2), ("run", 0, 1, 33),
+           ("step", ((0, 0, 1), (0, 1, 1), (0, 2, 1))), ("finish", 0, 1), ("finish", 0, 2), ("merge", 0, None),
+           ("step", ((0, 0, 1),))]
+    run_script(lib, manual(ops, geo))
+
+
+def test_more_streams_than_the_tensor_path_takes(lib):
+    geo = Geometry(1, 8, 2, 128, 16)
+    n = 260
+    ops = [("begin", 0), ("run", 0, 0, 50)]
+    for t in range(1, n + 1):
+        ops += [("spawn", 0, t), ("run", 0, t, 1 + t % 3), ("finish", 0, t)]
+    ops += [("merge", 0, None), ("step", ((0, 0, 1),))]        # the main thread now reads 261 streams
+    run_script(lib, manual(ops, geo, n_pages=400, max_threads=n + 2, max_segments=2 * n + 4))
+
+
+def test_fork_spawned_before_any_token(lib):
+    geo = Geometry(1, 8, 2, 128, 16)
+    ops = [("begin", 0), ("spawn", 0, 1), ("run", 0, 1, 5), ("run", 0, 0, 9),
+           ("step", ((0, 1, 1), (0, 0, 1))), ("finish", 0, 1), ("merge", 0, (1,)), ("step", ((0, 0, 1),))]
+    run_script(lib, manual(ops, geo))
