@@ -442,7 +442,7 @@ def run_trace(args):
     max_n = max(len(op[1]) for op in script.ops if op[0] == "step")
     pool = binding.Pool(geo.n_layers, geo.n_q_heads, geo.n_kv_heads, geo.head_dim, script.n_pages, script.max_requests,
                         script.max_threads_per_request, script.max_segments_per_thread, free_order=script.free_order,
-                        max_step_queries=max_n, max_layers_per_launch=min(8, geo.n_layers), device=local)
+                        max_step_queries=max_n, max_layers_per_launch=geo.n_layers, device=local)
     gen = torch.Generator(device=device); gen.manual_seed(script.seed + 977 * rank)
 
     def randn(shape):
@@ -478,6 +478,7 @@ def run_trace(args):
                 if world > 1:
                     dist.barrier()
                 launches0 = pool.launch_count()
+                pool.profile_enable(True)
                 sampler = ClockSampler(local) if rank == 0 else None
                 t_wall0 = time.time(); ev0.record(stream)
             n = len(op[1])
@@ -496,6 +497,8 @@ def run_trace(args):
     ms = ev0.elapsed_time(ev1)
     clocks = sampler.stop(t_wall0, t_wall1) if sampler else None
     launches = pool.launch_count() - launches0
+    kernel_ms, kernel_launches = pool.profile_read()
+    timed_calls = max(1, max(kernel_launches))
     assert pool.status() == 0, "a kernel reported an error"
     all_tokens, worst_s = aggregate(float(tokens), ms * 1e-3)
     if rank == 0:
@@ -510,6 +513,8 @@ def run_trace(args):
                        "pool_pages": script.n_pages, "pool_gb": script.n_pages * 65536 * L / 1e9,
                        "unique_kv_bytes_timed": bytes_, "l2": "inputs larger than L2",
                        "step_hbm_gbs": gbs, "step_frac_of_measured_peak": gbs / peak, "step_frac_of_nominal_8TBs": gbs / NOMINAL_HBM_GBS,
+                       "kernel_ms_per_step": {"tensor": kernel_ms[0] / timed_calls, "warp": kernel_ms[1] / timed_calls,
+                                              "merge": kernel_ms[2] / timed_calls, "steps_timed": timed_calls},
                        "step_begin_call_ms": host_s * 1e3 / args.steps,
                        "step_begin_note": "wall time inside pasta_step_begin; includes waiting for the device when the host runs ahead"},
             "clocks": clocks, "e2e": None, "gpu_launches": launches,

@@ -1,4 +1,5 @@
 // K1 (KV append), its inverse (read-back), K3 (warp-shuffle attention pass) and K4 (log-sum-exp merge).
+#include <algorithm>
 #include "device_common.cuh"
 #include "kernels.hpp"
 
@@ -393,19 +394,24 @@ cudaError_t launch_attn_warp(const PoolView &pv, const PlanHeader &h, int32_t la
 }
 
 // =============================================================================================
-// K4: log-sum-exp merge.  One warp per (layer, query, head): m* = max m_i,
+// K4: log-sum-exp merge.  One warp per (query, head, group of layers), looping over its layers: m* = max m_i,
 // out = sum_i 2^(m_i - m*) O_i / sum_i 2^(m_i - m*) l_i,  lse = ln2 * (m* + log2 of that sum).
+// Which partial rows belong to a (query, head) is the same for every layer, so the look-ups in the plan are made
+// once per warp, and the (m, l) pairs of the next layer are fetched while this layer's outputs are summed.
 // =============================================================================================
 __global__ void __launch_bounds__(256)
 merge_kernel(PoolView pv, int32_t n_queries, int32_t layer_count, int32_t off_query, int32_t off_trange,
-             int32_t off_tunit, int32_t t_rows, float *__restrict__ out, float *__restrict__ lse) {
+             int32_t off_tunit, int32_t t_rows, int32_t layers_per_warp, float *__restrict__ out,
+             float *__restrict__ lse) {
   const int D = pv.head_dim, Hq = pv.n_q_heads, G = Hq / pv.n_kv_heads;
   const int64_t gw = (static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x) >> 5;
   const int lane = threadIdx.x & 31;
-  if (gw >= static_cast<int64_t>(layer_count) * n_queries * Hq) return;
+  const int64_t per_group = static_cast<int64_t>(n_queries) * Hq;
+  const int ll_begin = static_cast<int>(gw / per_group) * layers_per_warp;
+  if (ll_begin >= layer_count) return;
+  const int ll_end = min(layer_count, ll_begin + layers_per_warp);
   const int h = static_cast<int>(gw % Hq);
-  const int n = static_cast<int>((gw / Hq) % n_queries);
-  const int ll = static_cast<int>(gw / (static_cast<int64_t>(Hq) * n_queries));
+  const int n = static_cast<int>((gw % per_group) / Hq);
   const int g = h / G, hl = h % G;
   const int32_t *Q = pv.plan + off_query + n * PQ_WORDS;
   const int treq = Q[PQ_TREQ], tidx = Q[PQ_TIDX], w0 = Q[PQ_WUNIT0], nw = Q[PQ_NW];
@@ -415,66 +421,81 @@ merge_kernel(PoolView pv, int32_t n_queries, int32_t layer_count, int32_t off_qu
     nt = pv.plan[off_trange + (treq * pv.n_kv_heads + g) * 2 + 1] - tb;
   }
   const int total = nt + nw;
-  const int64_t lbase = static_cast<int64_t>(ll) * pv.rows_per_layer;
-  auto row_of = [&](int i) -> int64_t {
-    if (i < nt) return lbase + pv.plan[off_tunit + (tb + i) * PU_WORDS + PU_ROW_BASE] + tidx * G + hl;
-    return lbase + t_rows + static_cast<int64_t>(w0 + g * nw + (i - nt)) * G + hl;
+  auto row_of = [&](int i) -> int64_t {     // within one layer
+    if (i < nt) return pv.plan[off_tunit + (tb + i) * PU_WORDS + PU_ROW_BASE] + tidx * G + hl;
+    return t_rows + static_cast<int64_t>(w0 + g * nw + (i - nt)) * G + hl;
   };
   const int E = D >> 5;                    // 4 or 2 elements per lane
-  float acc[4] = {0.f, 0.f, 0.f, 0.f};
-  float L = 0.f, mstar = -INFINITY;
   // lane i looks up partial row i (and i + 32, ...) once; the weighted sum then takes rows and weights from the
   // lanes' registers, so that only the loads of the partial outputs are left in the loop
-  for (int base_i = 0; base_i < total; base_i += 32) {
-    const int i = base_i + lane;
-    int64_t my_row = 0;
-    float2 my_ml = make_float2(-INFINITY, 0.f);
-    if (i < total) { my_row = row_of(i); my_ml = pv.part_ml[my_row]; }
-    float m_here = my_ml.y > 0.f ? my_ml.x : -INFINITY;
+  const int64_t first_row = lane < total ? row_of(lane) : 0;
+  float2 next_ml = make_float2(-INFINITY, 0.f);
+  if (lane < total) next_ml = pv.part_ml[static_cast<int64_t>(ll_begin) * pv.rows_per_layer + first_row];
+  for (int ll = ll_begin; ll < ll_end; ++ll) {
+    const int64_t lbase = static_cast<int64_t>(ll) * pv.rows_per_layer;
+    const float2 first_ml = next_ml;
+    if (ll + 1 < ll_end && lane < total) next_ml = pv.part_ml[lbase + pv.rows_per_layer + first_row];
+    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+    float L = 0.f, mstar = -INFINITY;
+    for (int base_i = 0; base_i < total; base_i += 32) {
+      const int i = base_i + lane;
+      int64_t my_row = lbase + first_row;
+      float2 my_ml = first_ml;
+      if (base_i > 0) {
+        my_ml = make_float2(-INFINITY, 0.f);
+        if (i < total) { my_row = lbase + row_of(i); my_ml = pv.part_ml[my_row]; }
+      }
+      float m_here = my_ml.y > 0.f ? my_ml.x : -INFINITY;
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) m_here = fmaxf(m_here, __shfl_xor_sync(0xffffffffu, m_here, o));
-    if (m_here > mstar) {                  // warp-uniform: move what has been summed so far to the new maximum
-      const float f = fast_exp2(mstar - m_here);    // 0 when nothing has been summed yet
-      L *= f;
+      for (int o = 16; o > 0; o >>= 1) m_here = fmaxf(m_here, __shfl_xor_sync(0xffffffffu, m_here, o));
+      if (m_here > mstar) {                  // warp-uniform: move what has been summed so far to the new maximum
+        const float f = fast_exp2(mstar - m_here);    // 0 when nothing has been summed yet
+        L *= f;
 #pragma unroll
-      for (int e = 0; e < 4; ++e) acc[e] *= f;
-      mstar = m_here;
-    }
-    const float my_w = my_ml.y > 0.f ? fast_exp2(my_ml.x - mstar) : 0.f;
-    const int cnt = min(32, total - base_i);
-    for (int k = 0; k < cnt; ++k) {
-      const float w = __shfl_sync(0xffffffffu, my_w, k);
-      const float lk = __shfl_sync(0xffffffffu, my_ml.y, k);
-      const int64_t row = __shfl_sync(0xffffffffu, my_row, k);
-      if (w == 0.f) continue;              // nothing visible in that piece (warp-uniform)
-      L = fmaf(w, lk, L);
-      const float *src = pv.part_o + row * D + lane * E;
-      if (E == 4) {
-        const float4 v = *reinterpret_cast<const float4 *>(src);
-        acc[0] = fmaf(w, v.x, acc[0]); acc[1] = fmaf(w, v.y, acc[1]);
-        acc[2] = fmaf(w, v.z, acc[2]); acc[3] = fmaf(w, v.w, acc[3]);
-      } else {
-        const float2 v = *reinterpret_cast<const float2 *>(src);
-        acc[0] = fmaf(w, v.x, acc[0]); acc[1] = fmaf(w, v.y, acc[1]);
+        for (int e = 0; e < 4; ++e) acc[e] *= f;
+        mstar = m_here;
+      }
+      const float my_w = my_ml.y > 0.f ? fast_exp2(my_ml.x - mstar) : 0.f;
+      const int cnt = min(32, total - base_i);
+      for (int k = 0; k < cnt; ++k) {
+        const float w = __shfl_sync(0xffffffffu, my_w, k);
+        const float lk = __shfl_sync(0xffffffffu, my_ml.y, k);
+        const int64_t row = __shfl_sync(0xffffffffu, my_row, k);
+        if (w == 0.f) continue;              // nothing visible in that piece (warp-uniform)
+        L = fmaf(w, lk, L);
+        const float *src = pv.part_o + row * D + lane * E;
+        if (E == 4) {
+          const float4 v = *reinterpret_cast<const float4 *>(src);
+          acc[0] = fmaf(w, v.x, acc[0]); acc[1] = fmaf(w, v.y, acc[1]);
+          acc[2] = fmaf(w, v.z, acc[2]); acc[3] = fmaf(w, v.w, acc[3]);
+        } else {
+          const float2 v = *reinterpret_cast<const float2 *>(src);
+          acc[0] = fmaf(w, v.x, acc[0]); acc[1] = fmaf(w, v.y, acc[1]);
+        }
       }
     }
+    const float inv = L > 0.f ? 1.f / L : 0.f;
+    float *dst = out + ((static_cast<int64_t>(ll) * n_queries + n) * Hq + h) * D + lane * E;
+    if (E == 4) *reinterpret_cast<float4 *>(dst) = make_float4(acc[0] * inv, acc[1] * inv, acc[2] * inv, acc[3] * inv);
+    else *reinterpret_cast<float2 *>(dst) = make_float2(acc[0] * inv, acc[1] * inv);
+    if (lse && lane == 0)
+      lse[(static_cast<int64_t>(ll) * n_queries + n) * Hq + h] = (mstar + log2f(L)) * 0.6931471805599453f;
   }
-  const float inv = L > 0.f ? 1.f / L : 0.f;
-  float *dst = out + ((static_cast<int64_t>(ll) * n_queries + n) * Hq + h) * D + lane * E;
-  if (E == 4) *reinterpret_cast<float4 *>(dst) = make_float4(acc[0] * inv, acc[1] * inv, acc[2] * inv, acc[3] * inv);
-  else *reinterpret_cast<float2 *>(dst) = make_float2(acc[0] * inv, acc[1] * inv);
-  if (lse && lane == 0)
-    lse[(static_cast<int64_t>(ll) * n_queries + n) * Hq + h] = (mstar + log2f(L)) * 0.6931471805599453f;
 }
 
 cudaError_t launch_merge(const PoolView &pv, const PlanHeader &h, int32_t layer_count, float *out, float *lse,
                          cudaStream_t st) {
-  const int64_t warps = static_cast<int64_t>(layer_count) * h.w[PH_N_QUERIES] * pv.n_q_heads;
-  if (warps == 0) return cudaSuccess;
+  const int64_t per_group = static_cast<int64_t>(h.w[PH_N_QUERIES]) * pv.n_q_heads;
+  if (per_group == 0 || layer_count == 0) return cudaSuccess;
+  // enough warps to fill the machine a few times over; beyond that, more layers per warp (its plan look-ups are shared)
+  const int64_t want_warps = 4 * 148 * 64;
+  const int64_t groups = std::min<int64_t>(layer_count, std::max<int64_t>(1, (want_warps + per_group - 1) / per_group));
+  const int32_t layers_per_warp = static_cast<int32_t>((layer_count + groups - 1) / groups);
+  const int64_t warps = per_group * ((layer_count + layers_per_warp - 1) / layers_per_warp);
   const int64_t blocks = (warps * 32 + 255) / 256;
   merge_kernel<<<static_cast<unsigned>(blocks), 256, 0, st>>>(pv, h.w[PH_N_QUERIES], layer_count, h.w[PH_OFF_QUERY],
                                                               h.w[PH_OFF_TRANGE], h.w[PH_OFF_TUNIT], h.w[PH_T_ROWS],
-                                                              out, lse);
+                                                              layers_per_warp, out, lse);
   return cudaGetLastError();
 }
 
