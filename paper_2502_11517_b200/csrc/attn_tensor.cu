@@ -156,6 +156,20 @@ __device__ __forceinline__ void tmem_st32_u32(uint32_t taddr, const uint32_t *r)
 }
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
+// two fp32 lanes at once: {x0, x1} = {a0, a1} * {b, b} + {c, c}
+__device__ __forceinline__ void fma2(float &x0, float &x1, float a0, float a1, float b, float c) {
+  asm("{\n\t.reg .b64 ra, rb, rc, rd;\n\t"
+      "mov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %4};\n\tmov.b64 rc, {%5, %5};\n\t"
+      "fma.rn.f32x2 rd, ra, rb, rc;\n\tmov.b64 {%0, %1}, rd;\n\t}"
+      : "=f"(x0), "=f"(x1) : "f"(a0), "f"(a1), "f"(b), "f"(c));
+}
+// {s0, s1} += {p0, p1}
+__device__ __forceinline__ void add2(float &s0, float &s1, float p0, float p1) {
+  asm("{\n\t.reg .b64 ra, rb, rd;\n\t"
+      "mov.b64 ra, {%0, %1};\n\tmov.b64 rb, {%2, %3};\n\t"
+      "add.rn.f32x2 rd, ra, rb;\n\tmov.b64 {%0, %1}, rd;\n\t}"
+      : "+f"(s0), "+f"(s1) : "f"(p0), "f"(p1));
+}
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   uint32_t r;
   asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
@@ -477,11 +491,12 @@ attn_tensor_kernel(PoolView pv, TensorArgs a, const __nv_bfloat16 *__restrict__ 
             uint32_t pk[T_HALF / 2];
 #pragma unroll
             for (int j = 0; j < T_HALF; j += 4) {
-              const float p0 = fast_exp2(fmaf(sc[j], a.scale_log2, -ref));
-              const float p1 = fast_exp2(fmaf(sc[j + 1], a.scale_log2, -ref));
-              const float p2 = fast_exp2(fmaf(sc[j + 2], a.scale_log2, -ref));
-              const float p3 = fast_exp2(fmaf(sc[j + 3], a.scale_log2, -ref));
-              ls[0] += p0; ls[1] += p1; ls[2] += p2; ls[3] += p3;
+              float x0, x1, x2, x3;
+              fma2(x0, x1, sc[j], sc[j + 1], a.scale_log2, -ref);
+              fma2(x2, x3, sc[j + 2], sc[j + 3], a.scale_log2, -ref);
+              const float p0 = fast_exp2(x0), p1 = fast_exp2(x1), p2 = fast_exp2(x2), p3 = fast_exp2(x3);
+              add2(ls[0], ls[1], p0, p1);
+              add2(ls[2], ls[3], p2, p3);
               pk[j >> 1] = pack_bf16(p0, p1);
               pk[(j >> 1) + 1] = pack_bf16(p2, p3);
             }
