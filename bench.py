@@ -544,32 +544,43 @@ def time_sync_merge():
 
 
 # ------------------------------------------------------------------------------------------------ oracle arm
-def oracle_sample(workload: str, budget_s: float = 20.0, steps: int = 1):
-    """Times the fp64 CPU oracle, as it stands, on a bounded sample of the workload: the queries of the
-    workload's first request(s), in layer 0.  Returns the cpu_baseline object."""
+_ORACLE_STATE = {}
+
+
+def _oracle_state(workload: str):
+    """The oracle replayed up to the workload's last step (bookkeeping and append done once), kept for reuse."""
+    if workload in _ORACLE_STATE:
+        return _ORACLE_STATE[workload]
     from oracle import OracleReplay
-    from pasta_workloads import cfg2_single_request, cfg3_batched, cfg4_long_prefix
+    from pasta_workloads import cfg2_single_request, cfg3_batched, cfg4_long_prefix, step_tensors
     if workload == "long_shared_prefix":
-        script = cfg4_long_prefix(n_requests=1); steps = max(steps, 4)
+        script = cfg4_long_prefix(n_requests=1); passes = 4
         sample = "the 17 thread-tokens of 1 of 8 requests (32768-token prefix, 16 forks), 1 layer, 4 passes"
     elif workload == "batched":
-        script = cfg3_batched(n_layers=1); steps = max(steps, 8)
+        script = cfg3_batched(n_layers=1); passes = 8
         sample = "all thread-tokens of the 64 requests, 1 of 32 layers, 8 passes (time scaled by 32 layers)"
     else:
-        script = cfg2_single_request("a"); script.ops = script.ops[:11]; steps = max(steps, 50)
+        script = cfg2_single_request("a"); script.ops = script.ops[:11]; passes = 50
         sample = "step A: 5 thread-tokens of the request, 1 layer, 50 passes"
     rep = OracleReplay(script)
     last = len(script.ops) - 1
     for i in range(last):
         rep.apply(i, attend=False)
-    # the step's bookkeeping and append happen once; the attention is what is timed
-    from oracle import decode_attention
-    from pasta_workloads import step_tensors
     op = script.ops[last]
     k, v, q = step_tensors(script, last, 0)
     slots = [s for s in rep.model.reserve(op[1]) if s is not None]
     rep.stores[0].write(slots, k, v)
     queries = [(e[0], e[1]) for e in op[1]]
+    _ORACLE_STATE[workload] = (rep, queries, q, sample, passes)
+    return _ORACLE_STATE[workload]
+
+
+def oracle_sample(workload: str, budget_s: float = 20.0, steps: int = 1):
+    """Times the fp64 CPU oracle, as it stands, on a bounded sample of the workload: the queries of the
+    workload's first request(s), in layer 0 (the attention is what is timed).  Returns the cpu_baseline object."""
+    from oracle import decode_attention
+    rep, queries, q, sample, passes = _oracle_state(workload)
+    steps = max(steps, passes)
     times = []
     t_all = time.perf_counter()
     for _ in range(steps):
@@ -599,7 +610,8 @@ def run_reference(args):
     if rank != 0:
         return
     t0 = time.perf_counter()
-    per_step = max(2.0, min(20.0, 120.0 / max(1, args.steps + args.warmup)))
+    _oracle_state(args.workload)                       # set-up once, outside the steps
+    per_step = max(0.25, min(20.0, 150.0 / max(1, args.steps + args.warmup)))
     for _ in range(args.warmup):
         oracle_sample(args.workload, budget_s=per_step)
     res = [oracle_sample(args.workload, budget_s=per_step) for _ in range(args.steps)]
