@@ -36,6 +36,7 @@ sys.path.insert(0, ROOT)
 METRIC = "decode-attn thread-tokens/s"
 UNIT = "thread-tokens/s"
 NOMINAL_HBM_GBS = 8000.0
+SEED_EXTRAS = 2502115
 FALLBACK_HBM_GBS = 6650.0
 # dram bytes (read + write) of one launch of the dominant kernel from an ncu capture of this workload,
 # or None when no capture matches the current kernel
@@ -525,6 +526,120 @@ def run_trace(args):
         dist.destroy_process_group()
 
 
+def run_extras(args):
+    """Measurements of the steps around the decode path: rotary embedding fused into the append, the host
+    interpreter's cost per step, a prompt fed in chunks of several tokens per step.  One JSON line; `value` is the
+    chunked-prefill rate in thread-tokens/s (one query per prompt token)."""
+    import torch
+    from paper_2502_11517_b200 import binding
+    from paper_2502_11517_b200.build import build
+    from paper_2502_11517_b200.interpreter import Interpreter, Tags
+    build()
+    device = torch.device("cuda", 0); torch.cuda.set_device(device)
+    gen = torch.Generator(device=device); gen.manual_seed(SEED_EXTRAS)
+
+    def randn(shape):
+        return torch.randn(shape, generator=gen, device=device, dtype=torch.float32).to(torch.bfloat16)
+
+    def timed(fn, reps):
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+        torch.cuda.synchronize(); ev[0].record(); [fn() for _ in range(reps)]; ev[1].record(); torch.cuda.synchronize()
+        return ev[0].elapsed_time(ev[1]) / reps
+
+    # ---- 1. append with and without the rotary embedding: 512 threads x 8 layers, one token each
+    L, Hq, Hkv, d, n = 8, 32, 8, 128, 512
+    pool = binding.Pool(L, Hq, Hkv, d, 4096, n, 1, 2, max_step_queries=n)
+    reqs = [pool.request_begin() for _ in range(n)]
+    for r in reqs:
+        pool.kv_append_run(r, 0, 16, randn((L, 16, Hkv, d)), randn((L, 16, Hkv, d)))
+    k, v = randn((L, n, Hkv, d)), randn((L, n, Hkv, d))
+    append_us = {}
+    for name, call in (("plain", lambda: pool.kv_append(k, v)), ("rope", lambda: pool.kv_append_rope(k, v, 10000.0))):
+        def one():
+            pool.step_begin(reqs, [0] * n, [1] * n)
+            call()
+        for _ in range(3):
+            one()
+        both = timed(one, 20)
+        plan_only = timed(lambda: pool.step_begin(reqs, [0] * n, [0] * n), 20)
+        append_us[name] = (both - plan_only) * 1e3
+    append_bytes = 2 * L * n * Hkv * d * 2 * 2              # K and V, read and written
+    pool.close()
+
+    # ---- 2. the host interpreter alone (host-only pool): 64 responses of three forks each
+    tags = Tags(1, 2, 3, 4)
+    hp = binding.Pool(1, Hq, Hkv, d, 8192, 64, 8, 16, flags=binding.FLAG_HOST_ONLY, max_step_queries=512)
+    it = Interpreter(hp, tags, predicted_length=lambda r, kk: 40)
+    main = [1, 1, 1] + [50] * 40 + [4] + [51] * 8
+    forks = {1: [60] * 30 + [3], 2: [61] * 45 + [3], 3: [62] * 20 + [3]}
+    for _ in range(64):
+        it.add_request(list(range(100, 400)))
+    count = {}
+    t0 = time.perf_counter(); steps = 0; fed = 0
+    while steps < 60:
+        entries = it.begin_step()
+        nxt = []
+        for req, t, _tok in entries:
+            kk = count.get((req, t), 0); count[(req, t)] = kk + 1
+            src = main if t == 0 else forks[t]
+            nxt.append(src[kk] if kk < len(src) else 52)
+        it.end_step(nxt)
+        steps += 1; fed += len(entries)
+    interp_s = time.perf_counter() - t0
+    hp.close()
+
+    # ---- 3. a prompt of 8192 tokens fed 32 tokens per step (128 stacked rows on the tensor-core path), 1 layer
+    prompt, chunk = 8192, 32
+    pool = binding.Pool(1, Hq, Hkv, d, 1024, 1, 1, 2, max_step_queries=chunk)
+    r = pool.request_begin()
+    kc, vc, qc = randn((1, chunk, Hkv, d)), randn((1, chunk, Hkv, d)), randn((1, chunk, Hq, d))
+    out = torch.empty((1, chunk, Hq, d), dtype=torch.float32, device=device)
+
+    def feed(m):
+        pool.step_begin([r], [0], [m])
+        pool.kv_append(kc[:, :m], vc[:, :m])
+        pool.decode_attn(qc[:, :m], out[:, :m])
+
+    for _ in range(4):
+        feed(chunk)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    n_chunks = prompt // chunk - 4
+    torch.cuda.synchronize(); ev0.record()
+    for _ in range(n_chunks):
+        feed(chunk)
+    ev1.record(); torch.cuda.synchronize()
+    chunk_ms = ev0.elapsed_time(ev1)
+    pool.close()
+    pool = binding.Pool(1, Hq, Hkv, d, 1024, 1, 1, 2, max_step_queries=chunk)
+    r = pool.request_begin()
+    for _ in range(8):
+        feed(1)
+    torch.cuda.synchronize(); ev0.record()
+    for _ in range(512):
+        feed(1)
+    ev1.record(); torch.cuda.synchronize()
+    single_ms = ev0.elapsed_time(ev1)
+    assert pool.status() == 0
+    pool.close()
+    chunk_rate = n_chunks * chunk / (chunk_ms * 1e-3)
+    print(json.dumps({
+        "metric": METRIC, "value": chunk_rate, "unit": UNIT, "n_gpus": 1, "steps": n_chunks, "warmup": 4,
+        "ms_per_step": chunk_ms / n_chunks, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+        "data": "synthetic",
+        "config": {"workload": "extras",
+                   "chunked_prefill": {"prompt_tokens": prompt, "tokens_per_step": chunk, "layers": 1,
+                                       "thread_tokens_per_s": chunk_rate, "ms_per_step": chunk_ms / n_chunks,
+                                       "one_token_per_step_thread_tokens_per_s": 512 / (single_ms * 1e-3),
+                                       "one_token_per_step_ms": single_ms / 512},
+                   "rope_append": {"threads": n, "layers": L, "plain_us": append_us["plain"], "rope_us": append_us["rope"],
+                                   "bytes_moved": append_bytes,
+                                   "rope_gbs": append_bytes / (append_us["rope"] * 1e-6) / 1e9},
+                   "interpreter_host_only": {"responses": 64, "steps": steps, "thread_tokens_fed": fed,
+                                             "us_per_step": interp_s / steps * 1e6,
+                                             "thread_tokens_per_s": fed / interp_s}},
+        "clocks": None, "e2e": None, "gpu_launches": None, "roofline": None, "cpu_baseline": None}))
+
+
 def time_sync_merge():
     from paper_2502_11517_b200 import binding
     best = None
@@ -650,6 +765,8 @@ def main():
         run_reference(args)
     elif args.workload == "trace":
         run_trace(args)
+    elif args.workload == "extras":
+        run_extras(args)
     else:
         run_ours(args)
 
