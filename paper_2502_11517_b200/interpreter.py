@@ -12,7 +12,10 @@ What it does (paper, Section 3 "Interpreter" and "Efficiency"; Fig. 2a):
     moves), the held <sync/> enters the pool and the main thread resumes, now conditioned on all chunks.
 
 Tokens enter the pool when they are fed to the model: a step feeds every runnable thread's pending token, the
-caller runs the model (pasta_kv_append + pasta_decode_attn inside it) and hands back one next token per thread.
+caller runs the model (pasta_kv_append + pasta_decode_attn inside it) and hands back one next token per fed token.
+A prompt can be fed through the same steps, several tokens at a time (`add_request(..., chunk=m)`): the request's
+entry then carries up to m tokens, each with its own query, and only what the model says after the prompt's last
+token is used.
 The interpreter is token-id agnostic: the four tag ids and a function that reads the predicted length out of a
 promise are given by the caller.
 """
@@ -35,6 +38,8 @@ class _Thread:
     pending: Optional[int]           # token to feed at the next step (None: nothing to feed)
     done: bool = False               # a fork that emitted </async>
     tokens: List[int] = field(default_factory=list)   # tokens fed so far (for inspection)
+    backlog: List[int] = field(default_factory=list)  # prompt tokens still to feed before `pending` (chunked prefill)
+    chunk: int = 1                   # how many backlog tokens one step may feed
 
 
 @dataclass
@@ -58,11 +63,17 @@ class Interpreter:
         self._entries: List[Tuple[int, int]] = []
 
     # ------------------------------------------------------------------ requests
-    def add_request(self, prompt: Sequence[int], k=None, v=None, stream=None) -> int:
-        """The prompt's tokens except the last are appended now, with their KV (k, v: device tensors
+    def add_request(self, prompt: Sequence[int], k=None, v=None, stream=None, chunk: int = 0) -> int:
+        """chunk == 0: the prompt's tokens except the last are appended now, with their KV (k, v: device tensors
         [layers, len(prompt) - 1, Hkv, d], or None on a host-only pool); the last prompt token is the first
-        pending input."""
+        pending input.  chunk > 0: nothing is appended now; the prompt is fed through the following steps, up to
+        `chunk` tokens per step, like any other token (the model computes their KV and attention)."""
         req = self.pool.request_begin()
+        if chunk > 0:
+            main = _Thread(pending=prompt[-1], backlog=list(prompt[:-1]), chunk=chunk)
+            self.requests[req] = _Request(threads={0: main})
+            self._promises[req] = 0
+            return req
         if len(prompt) > 1:
             self.pool.kv_append_run(req, 0, len(prompt) - 1, k, v, stream=stream)
         main = _Thread(pending=prompt[-1], tokens=list(prompt[:-1]))
@@ -76,9 +87,11 @@ class Interpreter:
 
     # ------------------------------------------------------------------ one decode step
     def begin_step(self, stream=None) -> List[Tuple[int, int, int]]:
-        """Feeds every runnable thread's pending token: reserves its slot and plans the step.
-        Returns the step's entries (request, thread, token) in order; the caller runs the model on them."""
+        """Feeds every runnable thread's pending token (or its next chunk of prompt tokens): reserves the slots and
+        plans the step.  Returns one (request, thread, token) per fed token, in the order of the step's queries;
+        the caller runs the model on them."""
         entries = []
+        step_reqs, step_threads, step_new = [], [], []
         for req, r in self.requests.items():
             if r.finished:
                 continue
@@ -86,22 +99,34 @@ class Interpreter:
             # promise the main thread feeds now (its prefix needs that promise appended first)
             runnable = [t for t, th in r.threads.items() if th.pending is not None and not th.done]
             order = sorted(runnable, key=lambda t: (1 if t == 0 else 2 if not r.threads[t].tokens else 0, t))
-            entries.extend((req, t, r.threads[t].pending) for t in order)
+            for t in order:
+                th = r.threads[t]
+                if th.backlog:                  # a chunk of the prompt; the pending token joins it when it fits
+                    feed = th.backlog[:th.chunk]
+                    del th.backlog[:len(feed)]
+                    if not th.backlog and len(feed) < th.chunk:
+                        feed.append(th.pending); th.pending = None
+                else:
+                    feed = [th.pending]; th.pending = None
+                entries.extend((req, t, tok) for tok in feed)
+                th.tokens.extend(feed)
+                step_reqs.append(req); step_threads.append(t); step_new.append(len(feed))
         self._entries = [(e[0], e[1]) for e in entries]
         if entries:
-            self.pool.step_begin([e[0] for e in entries], [e[1] for e in entries], [1] * len(entries), stream=stream)
-            for req, t, tok in entries:
-                th = self.requests[req].threads[t]
-                th.tokens.append(tok)
-                th.pending = None
+            self.pool.step_begin(step_reqs, step_threads, step_new, stream=stream)
         return entries
 
     def end_step(self, next_tokens: Sequence[int], end_of_text: Optional[int] = None) -> None:
         """next_tokens[i] is what the model produced for entry i of begin_step."""
         assert len(next_tokens) == len(self._entries)
-        for (req, t), tok in zip(self._entries, next_tokens):
+        last_of = {}
+        for i, key in enumerate(self._entries):
+            last_of[key] = i                      # only what follows a thread's newest token counts
+        for i, ((req, t), tok) in enumerate(zip(self._entries, next_tokens)):
             r = self.requests[req]
             th = r.threads[t]
+            if last_of[(req, t)] != i or th.backlog or th.pending is not None:
+                continue                          # inside a prompt chunk: the model's continuation is not used
             fed = th.tokens[-1]
             if t == 0:
                 if end_of_text is not None and tok == end_of_text:

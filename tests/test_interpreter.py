@@ -127,3 +127,39 @@ def test_sync_waits_and_merge_moves_nothing():
     view = pool.dump()["requests"][req]["threads"][0]["view"]
     assert [seg[0] for seg in view] == [0, 1, 0, 2, 0]          # each chunk right behind its promise
     pool.close()
+
+
+def test_prompt_fed_in_chunks_ends_in_the_same_state():
+    """Feeding the prompt through the steps, 7 tokens at a time, only delays the response: 20 + 1 prompt tokens take
+    three steps instead of one, after which every step feeds the same tokens and leaves the same pool state."""
+    ids, prompt, emissions = fig2_scripts()
+
+    def run(chunk, n_steps):
+        pool = binding.Pool(1, 4, 2, 64, 64, 2, 16, 64, flags=binding.FLAG_HOST_ONLY)
+        it = Interpreter(pool, Tags(PROMISE, OPEN, CLOSE, SYNC), predicted_length=lambda req, k: 10)
+        it.add_request(prompt, chunk=chunk)
+        fake = Scripted(emissions)
+        fed, states = [], []
+        for _ in range(n_steps):
+            entries = it.begin_step()
+            fed.append([(t, tok) for _r, t, tok in entries])
+            states.append(pool.dump())
+            # the scripted stand-in answers per fed token; inside a prompt chunk its answers must be ignored, so it
+            # is asked only for the thread's newest token and the other slots get a token that would derail the run
+            newest = {}
+            for i, (r, t, _tok) in enumerate(entries):
+                newest[(r, t)] = i
+            in_prompt = bool(it.requests[0].threads[0].backlog or it.requests[0].threads[0].pending is not None)
+            answers = [PROMISE] * len(entries)
+            real = [e for i, e in enumerate(entries) if newest[(e[0], e[1])] == i and not (e[1] == 0 and in_prompt)]
+            for e, tok in zip(real, fake(real)):
+                answers[newest[(e[0], e[1])]] = tok
+            it.end_step(answers)
+        pool.close()
+        return fed, states
+
+    fed1, st1 = run(0, 11)
+    fed7, st7 = run(7, 13)
+    assert [len(f) for f in fed7[:3]] == [7, 7, 7] and [tok for _t, tok in sum(fed7[:3], [])] == prompt
+    assert fed7[3:] == fed1[1:]
+    assert st7[2:] == st1[:]          # the same states, two steps later (the state after the whole prompt included)
