@@ -270,18 +270,20 @@ def run_ours(args):
     else:
         pool, entries, randn = build_state(script, device, seed_offset=rank, grow_tokens=grow)
     n = len(entries)
-    reqs = [e[0] for e in entries]; thr = [e[1] for e in entries]
-    ones = [1] * n
+    reqs = np.asarray([e[0] for e in entries], dtype=np.int32); thr = np.asarray([e[1] for e in entries], dtype=np.int32)
+    ones = np.ones(n, dtype=np.int32)
     L = geo.n_layers
     k_new = randn((L, n, geo.n_kv_heads, geo.head_dim)); v_new = randn((L, n, geo.n_kv_heads, geo.head_dim))
     q = randn((L, n, geo.n_q_heads, geo.head_dim))
     out = torch.empty(q.shape, dtype=torch.float32, device=device)
     stream = torch.cuda.current_stream(device)
 
+    sh = stream.cuda_stream                   # the stream's handle, looked up once
+
     def step():
-        pool.step_begin(reqs, thr, ones)
-        pool.kv_append(k_new, v_new)
-        pool.decode_attn(q, out)
+        pool.step_begin(reqs, thr, ones, stream=sh)
+        pool.kv_append(k_new, v_new, stream=sh)
+        pool.decode_attn(q, out, stream=sh)
 
     for _ in range(max(args.warmup, 3)):
         step()

@@ -74,11 +74,13 @@ def _check(code: int, where: str) -> None:
 
 
 def _i32(a) -> np.ndarray:
+    if isinstance(a, np.ndarray) and a.dtype == np.int32 and a.flags.c_contiguous:
+        return a                                  # callers that step in a loop convert once and pass arrays
     return np.ascontiguousarray(np.asarray(a, dtype=np.int32))
 
 
 def _ptr(a: Optional[np.ndarray]):
-    return None if a is None else a.ctypes.data_as(C.POINTER(C.c_int32))
+    return None if a is None else C.c_void_p(a.ctypes.data)
 
 
 def _dev(t) -> C.c_void_p:
@@ -110,7 +112,7 @@ class Pool:
         self.host_only = bool(flags & FLAG_HOST_ONLY)
         L = lib()
         order = None if free_order is None else _i32(free_order)
-        cfg.free_order = _ptr(order) if order is not None else C.POINTER(C.c_int32)()
+        cfg.free_order = order.ctypes.data_as(C.POINTER(C.c_int32)) if order is not None else C.POINTER(C.c_int32)()
         self.kv = self.workspace = None
         if not self.host_only:
             import torch
