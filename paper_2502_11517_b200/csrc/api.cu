@@ -15,6 +15,7 @@ using namespace pasta;
 namespace {
 
 constexpr int kStaging = 4;           // pinned upload buffers in rotation
+constexpr size_t kSmallPlanWords = 2048;   // plans up to this size are uploaded in the caller's stream
 constexpr int kProfCalls = 512;        // timed pasta_decode_attn launches kept between two profile reads
 constexpr int kRunChunk = 8192;       // tokens whose slots are uploaded at once by pasta_kv_append_run
 int32_t g_last_cuda_error = 0;
@@ -350,11 +351,18 @@ pasta_status_t pasta_step_begin(pasta_pool_t *p, int32_t n, const int32_t *req_i
     const int64_t i = p->step_index++;
     const int b = static_cast<int>(i & 1);
     PASTA_CUDA(cudaEventRecord(p->work_mark[b], st));
-    if (i >= 1) PASTA_CUDA(cudaStreamWaitEvent(p->copy_stream, p->work_mark[b ^ 1], 0));
-    s = upload(p, p->plan.data(), p->plan.size(), p->plan_dev[b], p->copy_stream);
-    if (s != PASTA_OK) return s;
-    PASTA_CUDA(cudaEventRecord(p->plan_ready[b], p->copy_stream));
-    PASTA_CUDA(cudaStreamWaitEvent(st, p->plan_ready[b], 0));
+    if (p->plan.size() <= kSmallPlanWords) {
+      // a small plan is copied in the caller's stream: it is ordered behind the kernels of step i - 2 there anyway,
+      // and a few microseconds of copy are not worth two more events and two stream waits on the host
+      s = upload(p, p->plan.data(), p->plan.size(), p->plan_dev[b], st);
+      if (s != PASTA_OK) return s;
+    } else {
+      if (i >= 1) PASTA_CUDA(cudaStreamWaitEvent(p->copy_stream, p->work_mark[b ^ 1], 0));
+      s = upload(p, p->plan.data(), p->plan.size(), p->plan_dev[b], p->copy_stream);
+      if (s != PASTA_OK) return s;
+      PASTA_CUDA(cudaEventRecord(p->plan_ready[b], p->copy_stream));
+      PASTA_CUDA(cudaStreamWaitEvent(st, p->plan_ready[b], 0));
+    }
     p->pv.plan = p->plan_dev[b];
   }
   p->plan_valid = true;
