@@ -280,10 +280,8 @@ def run_ours(args):
 
     sh = stream.cuda_stream                   # the stream's handle, looked up once
 
-    def step():
-        pool.step_begin(reqs, thr, ones, stream=sh)
-        pool.kv_append(k_new, v_new, stream=sh)
-        pool.decode_attn(q, out, stream=sh)
+    def step():                               # plan + append + attention of all layers, one library call
+        pool.step_device(reqs, thr, ones, k_new, v_new, q, out, stream=sh)
 
     for _ in range(max(args.warmup, 3)):
         step()

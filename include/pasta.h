@@ -216,6 +216,17 @@ pasta_status_t pasta_kv_append_run_rope(pasta_pool_t *pool, int32_t req, int32_t
                                         float theta, void *stream);
 
 /*
+ * One whole step with DEVICE tensors in one call: pasta_step_begin, pasta_kv_append and pasta_decode_attn for all
+ * layers (Section 3: a decoding step of every active thread).  Arguments as in those three calls: k_new, v_new
+ * device bf16 [n_layers, appended tokens, n_kv_heads, head_dim]; q device bf16 [n_layers, queries, n_q_heads,
+ * head_dim]; out device fp32 like q; lse optional.  Saves the caller two library calls per step, which is what
+ * bounds small steps.  Errors as in the three calls; after a failure of the first nothing is enqueued.
+ */
+pasta_status_t pasta_step_device(pasta_pool_t *pool, int32_t n, const int32_t *req_ids, const int32_t *thread_ids,
+                                 const int32_t *n_new, const void *k_new, const void *v_new, const void *q, void *out,
+                                 float *lse, float scale, void *stream);
+
+/*
  * One whole step with HOST tensors: step_begin, copy k_new / v_new / q to the device, kv_append
  * and decode_attn for all layers, copy `out` back, synchronise the stream.  k_new, v_new:
  * host bf16 [n_layers, n_app, n_kv_heads, head_dim]; q: host bf16 [n_layers, n, n_q_heads, head_dim];

@@ -26,7 +26,7 @@ EXPORTS = [
     "pasta_pool_dump", "pasta_plan_dump", "pasta_pool_status", "pasta_launch_count",
     "pasta_profile_enable", "pasta_profile_read", "pasta_decode_attn_noalloc",
     "pasta_thread_spawn_predicted", "pasta_step_positions", "pasta_kv_append_rope", "pasta_rope_queries",
-    "pasta_kv_append_run_rope",
+    "pasta_kv_append_run_rope", "pasta_step_device",
     "pasta_last_cuda_error",
 ]
 
@@ -233,6 +233,15 @@ class Pool:
         st = C.c_void_p(0) if (self.host_only or cnt == 0) else _stream(stream)
         _check(lib().pasta_kv_append_run(self._h, req, thread, m, layer_begin, cnt, _dev(k), _dev(v), st),
                "pasta_kv_append_run")
+
+    def step_device(self, req_ids, thread_ids, n_new, k_new, v_new, q, out, lse=None, scale: float = 0.0,
+                    stream=None) -> None:
+        """step_begin + kv_append + decode_attn for all layers in one library call (device tensors)."""
+        r, t = _i32(req_ids), _i32(thread_ids)
+        nn = None if n_new is None else _i32(n_new)
+        _check(lib().pasta_step_device(self._h, len(r), _ptr(r), _ptr(t), _ptr(nn), _dev(k_new), _dev(v_new), _dev(q),
+                                       _dev(out), _dev(lse), C.c_float(scale), _stream(stream)), "pasta_step_device")
+        self._last_n = len(r) if nn is None else int(np.maximum(nn, 1).sum())
 
     def step_host_bytes(self, n: int) -> int:
         out = C.c_size_t()

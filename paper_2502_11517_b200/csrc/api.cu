@@ -484,6 +484,18 @@ pasta_status_t pasta_kv_append_run_rope(pasta_pool_t *p, int32_t req, int32_t th
   return append_run_impl(p, req, thread, m, layer_begin, layer_count, k, v, theta, stream);
 }
 
+pasta_status_t pasta_step_device(pasta_pool_t *p, int32_t n, const int32_t *req_ids, const int32_t *thread_ids,
+                                 const int32_t *n_new, const void *k_new, const void *v_new, const void *q, void *out,
+                                 float *lse, float scale, void *stream) {
+  if (!p) return PASTA_ERR_INVALID_ARG;
+  if (p->host_only) return PASTA_ERR_BAD_STATE;
+  pasta_status_t s = pasta_step_begin(p, n, req_ids, thread_ids, n_new, stream);
+  if (s != PASTA_OK) return s;
+  s = pasta_kv_append(p, 0, p->cfg.n_layers, k_new, v_new, stream);
+  if (s != PASTA_OK) return s;
+  return pasta_decode_attn(p, 0, p->cfg.n_layers, q, out, lse, scale, stream);
+}
+
 pasta_status_t pasta_step_host_bytes(pasta_pool_t *p, int32_t n, size_t *out) {
   if (!p || !out || n < 0) return PASTA_ERR_INVALID_ARG;
   const size_t L = p->cfg.n_layers, d = p->cfg.head_dim;

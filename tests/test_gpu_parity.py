@@ -174,6 +174,35 @@ def test_page_placement_does_not_change_the_result(lib):
         assert torch.equal(a, b)
 
 
+def test_step_device_entry_point_equals_the_three_calls(lib):
+    import torch
+    from lib_replay import LibReplay, make_pool
+    outs = []
+    for fused in (False, True):
+        script = cfg2_single_request("b")
+        pool = make_pool(script)
+        rep = LibReplay(script, pool)
+        first = next(i for i, op in enumerate(script.ops) if op[0] == "step")
+        for i in range(first):
+            rep.apply(i)
+        op = script.ops[first]
+        L = range(script.geometry.n_layers)
+        ks, vs, qs = zip(*[step_tensors(script, first, l) for l in L])
+        k = torch.stack(ks).cuda(); v = torch.stack(vs).cuda(); q = torch.stack(qs).cuda()
+        out = torch.empty(q.shape, dtype=torch.float32, device="cuda")
+        lse = torch.empty(q.shape[:3], dtype=torch.float32, device="cuda")
+        reqs = [e[0] for e in op[1]]; thr = [e[1] for e in op[1]]; nn = [e[2] for e in op[1]]
+        if fused:
+            pool.step_device(reqs, thr, nn, k, v, q, out, lse)
+        else:
+            pool.step_begin(reqs, thr, nn); pool.kv_append(k, v); pool.decode_attn(q, out, lse)
+        torch.cuda.synchronize()
+        assert pool.status() == 0
+        outs.append((out.cpu(), lse.cpu(), pool.dump()))
+        pool.close()
+    assert torch.equal(outs[0][0], outs[1][0]) and torch.equal(outs[0][1], outs[1][1]) and outs[0][2] == outs[1][2]
+
+
 def test_step_host_entry_point(lib):
     """The host-buffer entry point (copies inside the call) gives the same numbers as the device one."""
     import torch
