@@ -163,3 +163,45 @@ def test_prompt_fed_in_chunks_ends_in_the_same_state():
     assert [len(f) for f in fed7[:3]] == [7, 7, 7] and [tok for _t, tok in sum(fed7[:3], [])] == prompt
     assert fed7[3:] == fed1[1:]
     assert st7[2:] == st1[:]          # the same states, two steps later (the state after the whole prompt included)
+
+
+def test_several_responses_decode_side_by_side():
+    """Three responses in one pool, stepped together: every response follows its own timeline (same tokens fed at
+    the same step, same views, cut-offs and position ids as when it runs alone); only page numbers differ, since
+    the responses draw from one free list."""
+    scripts = [random_threads(s) for s in (2, 5, 9)]
+
+    def strip(dump_req):
+        return {"streams": {s: v["len"] for s, v in dump_req["streams"].items()},
+                "threads": {t: {k: v for k, v in th.items() if k != "state"} for t, th in dump_req["threads"].items()}}
+
+    alone = []
+    for prompt, emissions in scripts:
+        pool = binding.Pool(1, 4, 2, 64, 256, 1, 16, 64, flags=binding.FLAG_HOST_ONLY)
+        it = Interpreter(pool, Tags(PROMISE, OPEN, CLOSE, SYNC))
+        it.add_request(prompt)
+        fake = Scripted(emissions)
+        log = []
+        for _ in range(60):
+            entries = it.begin_step()
+            log.append(([(t, tok) for _r, t, tok in entries], strip(pool.dump()["requests"][0])))
+            it.end_step(fake(entries))
+        alone.append(log)
+        pool.close()
+
+    pool = binding.Pool(1, 4, 2, 64, 256, 3, 16, 64, flags=binding.FLAG_HOST_ONLY, max_step_queries=64)
+    it = Interpreter(pool, Tags(PROMISE, OPEN, CLOSE, SYNC))
+    fakes = {}
+    for prompt, emissions in scripts:
+        fakes[it.add_request(prompt)] = Scripted(emissions)
+    for step in range(60):
+        entries = it.begin_step()
+        dump = pool.dump()["requests"]
+        answers = [None] * len(entries)
+        for req in fakes:
+            mine = [(i, e) for i, e in enumerate(entries) if e[0] == req]
+            assert ([(t, tok) for _i, (_r, t, tok) in mine], strip(dump[req])) == alone[req][step], (req, step)
+            for (i, _e), tok in zip(mine, fakes[req]([(0, e[1], e[2]) for _i, e in mine])):
+                answers[i] = tok
+        it.end_step(answers)
+    pool.close()
