@@ -226,8 +226,9 @@ attn_tensor_kernel(PoolView pv, TensorArgs a, const __nv_bfloat16 *__restrict__ 
   const int32_t *plan = pv.plan;
   const int u0 = plan[a.off_tcta + 2 * blockIdx.x], u1 = plan[a.off_tcta + 2 * blockIdx.x + 1];
 
-  // ---- set-up: zero the operand buffers (stale bytes meet zero weights, so they must be finite)
-  for (int i = tid; i < OFF_BAR / 16; i += T_THREADS) reinterpret_cast<uint4 *>(sm)[i] = make_uint4(0, 0, 0, 0);
+  // ---- set-up.  Operand bytes that no copy fills meet zero weights, so they only have to be finite: the Q builder
+  // writes all 128 rows of every unit, and the producer clears the page slots a partial tile leaves empty the first
+  // time each stage is used (afterwards they hold an earlier tile's keys and values).
   if (tid == 0) {
     for (int s = 0; s < T_STAGES; ++s) { mbar_init(bar + 8 * (B_FULL + s), 1); mbar_init(bar + 8 * (B_EMPTY + s), 1); }
     for (int b = 0; b < 2; ++b) {
@@ -275,6 +276,12 @@ attn_tensor_kernel(PoolView pv, TensorArgs a, const __nv_bfloat16 *__restrict__ 
               if (page < 0 || page >= pv.n_pages) { report(pv.status, PASTA_ERR_DEVICE_CHECK); page = 0; meta = -1; }
             }
             meta_s[s * PASTA_TILE_PAGES + lane] = meta;
+          }
+          if (it < T_STAGES && n_valid < PASTA_TILE_PAGES) {     // first use of this stage and some slots stay empty
+            uint4 *slot = reinterpret_cast<uint4 *>(sm + OFF_STAGE + s * T_STAGE_BYTES + n_valid * T_BLOCK);
+            for (int i = lane; i < (PASTA_TILE_PAGES - n_valid) * (T_BLOCK / 16); i += 32) slot[i] = make_uint4(0, 0, 0, 0);
+            fence_proxy_async();
+            __syncwarp();
           }
           if (lane == 0) mbar_expect_tx(bar + 8 * (B_FULL + s), n_valid * T_BLOCK);
           __syncwarp();
