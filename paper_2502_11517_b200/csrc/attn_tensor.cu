@@ -195,13 +195,13 @@ struct UnitInfo {
 };
 
 __device__ __forceinline__ UnitInfo load_unit(const int32_t *plan, int off_tunit, int off_treq, int u) {
-  const int32_t *U = plan + off_tunit + u * PU_WORDS;
+  (void)off_treq;
+  const int4 *U = reinterpret_cast<const int4 *>(plan + off_tunit + u * PU_WORDS);   // tables start 16-byte aligned
+  const int4 a = U[0], b = U[1], c = U[2];
   UnitInfo x;
-  x.treq = U[PU_TREQ]; x.g = U[PU_KV_HEAD]; x.tile_begin = U[PU_TILE_BEGIN]; x.tile_end = U[PU_TILE_END];
-  x.row_base = U[PU_ROW_BASE];
-  const int32_t *T = plan + off_treq + x.treq * PT_WORDS;
-  x.page_off = T[PT_PAGE_OFF]; x.n_pages = T[PT_N_PAGES]; x.n_threads = T[PT_N_THREADS];
-  x.n_streams = T[PT_N_STREAMS]; x.vis_off = T[PT_VIS_OFF]; x.tq_off = T[PT_TQ_OFF];
+  x.treq = a.x; x.g = a.y; x.tile_begin = a.z; x.tile_end = a.w;
+  x.row_base = b.x; x.page_off = b.y; x.n_pages = b.z; x.n_threads = b.w;
+  x.n_streams = c.x; x.vis_off = c.y; x.tq_off = c.z;
   return x;
 }
 

@@ -77,15 +77,24 @@ enum {
   PT_WORDS
 };
 
-// per t-unit
+// per t-unit.  The t-request's fields are repeated here so that a kernel role learns everything about its next unit
+// from one record (12 words, three 16-byte loads issued together) instead of following a second pointer.
 enum {
   PU_TREQ = 0,
   PU_KV_HEAD,
   PU_TILE_BEGIN,
   PU_TILE_END,
   PU_ROW_BASE,
+  PU_PAGE_OFF,        // = PT_PAGE_OFF of the t-request, and so on
+  PU_N_PAGES,
+  PU_N_THREADS,
+  PU_N_STREAMS,
+  PU_VIS_OFF,
+  PU_TQ_OFF,
+  PU_PAD,
   PU_WORDS
 };
+static_assert(PU_WORDS == 12, "t-unit records are read as three int4");
 
 // per w-unit
 enum {

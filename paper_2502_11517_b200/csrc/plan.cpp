@@ -280,7 +280,9 @@ pasta_status_t build_plan(const HostPool &pool, const std::vector<StepQuery> &en
     ttab.insert(ttab.end(), rec, rec + PT_WORDS);
   }
   for (const TUnit &u : tunits) {
-    const int32_t rec[PU_WORDS] = {u.treq, u.g, u.tile_begin, u.tile_end, u.row_base};
+    const TReq &t = treqs[u.treq];
+    const int32_t rec[PU_WORDS] = {u.treq, u.g, u.tile_begin, u.tile_end, u.row_base, t.page_off, t.n_pages,
+                                   t.n_threads, t.n_streams, t.vis_off, t.tq_off, 0};
     utab.insert(utab.end(), rec, rec + PU_WORDS);
   }
   w[PH_MAGIC] = PASTA_PLAN_MAGIC;

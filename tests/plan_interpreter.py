@@ -7,7 +7,7 @@ import numpy as np
 (PH_MAGIC, PH_N_QUERIES, PH_N_APPEND, PH_N_TREQ, PH_N_TUNITS, PH_N_WUNITS, PH_T_ROWS, PH_ROWS, PH_T_GRID,
  PH_OFF_APPEND, PH_OFF_QUERY, PH_OFF_TREQ, PH_OFF_TRANGE, PH_OFF_TUNIT, PH_OFF_TCTA, PH_OFF_WUNIT, PH_OFF_PAGES,
  PH_OFF_PMETA, PH_OFF_VIS, PH_OFF_TQ, PH_OFF_APOS, PH_OFF_QPOS, PH_TOTAL_WORDS) = range(23)
-PQ, PT, PU, PW = 4, 6, 5, 4
+PQ, PT, PU, PW = 4, 6, 12, 4
 TILE_PAGES, PAGE = 8, 16
 STATS = {'flagged': 0, 'pages': 0}    # pages the plans marked as visible in full to every thread, of all pages walked
 
@@ -30,9 +30,11 @@ def run_plan(w, K, V, q, n_kv_heads):
         assert np.all(cta[1:, 0] == cta[:-1, 1]) and np.all(cta[:, 1] > cta[:, 0])
 
     for u in range(w[PH_N_TUNITS]):
-        treq, g, tb, te, row_base = w[w[PH_OFF_TUNIT] + u * PU: w[PH_OFF_TUNIT] + (u + 1) * PU]
+        rec = w[w[PH_OFF_TUNIT] + u * PU: w[PH_OFF_TUNIT] + (u + 1) * PU]
+        treq, g, tb, te, row_base = rec[:5]
         T = w[PH_OFF_TREQ] + treq * PT
         page_off, n_pages, n_thr, n_str, vis_off, tq_off = w[T:T + PT]
+        assert list(rec[5:11]) == [page_off, n_pages, n_thr, n_str, vis_off, tq_off]     # the unit repeats its t-request
         assert 0 <= tb < te <= -(-n_pages // TILE_PAGES)
         vis = w[w[PH_OFF_VIS] + vis_off: w[PH_OFF_VIS] + vis_off + n_thr * n_str].reshape(n_thr, n_str)
         tq = w[w[PH_OFF_TQ] + tq_off: w[PH_OFF_TQ] + tq_off + n_thr]
