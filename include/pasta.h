@@ -61,7 +61,7 @@ typedef struct {
   int32_t max_requests;             /* requests alive at the same time */
   int32_t max_threads_per_request;  /* main thread + every fork ever spawned by one request (ids are not reused) */
   int32_t max_segments_per_thread;  /* longest segment list of one thread */
-  int32_t max_step_queries;         /* most (request, thread) entries in one step; 0 = max_requests * 17 */
+  int32_t max_step_queries;         /* most queries in one step (one per entry, or per new token); 0 = max_requests * 17 */
   int32_t max_partial_rows;         /* split/segment partial results per layer; 0 = derived from max_step_queries */
   int32_t max_layers_per_launch;    /* layers whose partials fit the workspace at once; 0 = min(n_layers, 8) */
   int32_t flags;                    /* PASTA_FLAG_* */
