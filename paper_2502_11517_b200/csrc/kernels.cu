@@ -65,7 +65,17 @@ __global__ void kv_read_kernel(PoolView pv, const int32_t *__restrict__ slots, i
 // One thread handles the 16-byte chunk c of the low half together with chunk c of the high half.
 // Angles are evaluated in double precision so that the stored bf16 keys agree with a float64 reference.
 // =============================================================================================
-__device__ __forceinline__ void rope_pairs(uint4 &lo, uint4 &hi, int pos, int first_i, int D, double log2_theta) {
+// Sines and cosines of the 8 angles of chunk c (elements first_i .. first_i + 7 of the low half): they depend on
+// the token's position only, so a thread evaluates them once and applies them to every head of the token.
+__device__ __forceinline__ void rope_angles(int pos, int first_i, int D, double log2_theta, double *sn, double *cs) {
+#pragma unroll
+  for (int e = 0; e < 8; ++e) {
+    const double ang = static_cast<double>(pos) * exp2(-2.0 * (first_i + e) / D * log2_theta);
+    sincos(ang, &sn[e], &cs[e]);
+  }
+}
+
+__device__ __forceinline__ void rope_apply(uint4 &lo, uint4 &hi, const double *sn, const double *cs) {
   uint32_t *l = reinterpret_cast<uint32_t *>(&lo), *h = reinterpret_cast<uint32_t *>(&hi);
 #pragma unroll
   for (int w = 0; w < 4; ++w) {
@@ -73,12 +83,9 @@ __device__ __forceinline__ void rope_pairs(uint4 &lo, uint4 &hi, int pos, int fi
     float yl[2], yh[2];
 #pragma unroll
     for (int e = 0; e < 2; ++e) {
-      const int i = first_i + 2 * w + e;
-      const double ang = static_cast<double>(pos) * exp2(-2.0 * i / D * log2_theta);
-      double sn, cs;
-      sincos(ang, &sn, &cs);
-      yl[e] = static_cast<float>(static_cast<double>(xl[e]) * cs - static_cast<double>(xh[e]) * sn);
-      yh[e] = static_cast<float>(static_cast<double>(xh[e]) * cs + static_cast<double>(xl[e]) * sn);
+      const double c = cs[2 * w + e], s_ = sn[2 * w + e];
+      yl[e] = static_cast<float>(static_cast<double>(xl[e]) * c - static_cast<double>(xh[e]) * s_);
+      yh[e] = static_cast<float>(static_cast<double>(xh[e]) * c + static_cast<double>(xl[e]) * s_);
     }
     __nv_bfloat162 pl = __floats2bfloat162_rn(yl[0], yl[1]), ph = __floats2bfloat162_rn(yh[0], yh[1]);
     l[w] = *reinterpret_cast<uint32_t *>(&pl);
@@ -86,19 +93,22 @@ __device__ __forceinline__ void rope_pairs(uint4 &lo, uint4 &hi, int pos, int fi
   }
 }
 
+// Threads [0, n_k) rotate and store K: one thread per (layer, token, chunk pair), all kv heads of the token in turn.
+// Threads [n_k, n_k + n_v) copy V: one thread per (layer, token, kv head, chunk pair).
 __global__ void kv_append_rope_kernel(PoolView pv, const int32_t *__restrict__ slots, const int32_t *__restrict__ pos,
                                       int32_t pos0, int32_t n_tok, int32_t layer_begin, int32_t layer_count,
                                       const uint4 *__restrict__ k_new, const uint4 *__restrict__ v_new, double log2_theta) {
   const int chunks = pv.head_dim >> 3, half_chunks = chunks >> 1;
-  const int64_t total = static_cast<int64_t>(layer_count) * n_tok * pv.n_kv_heads * 2 * half_chunks;
-  const int64_t idx = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
-  if (idx >= total) return;
+  const int64_t n_k = static_cast<int64_t>(layer_count) * n_tok * half_chunks;
+  const int64_t n_v = n_k * pv.n_kv_heads;
+  int64_t idx = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (idx >= n_k + n_v) return;
+  const bool is_k = idx < n_k;
+  if (!is_k) idx -= n_k;
   const int c = static_cast<int>(idx % half_chunks);
   int64_t rest = idx / half_chunks;
-  const int kv = static_cast<int>(rest & 1);
-  rest >>= 1;
-  const int g = static_cast<int>(rest % pv.n_kv_heads);
-  rest /= pv.n_kv_heads;
+  int g = 0;
+  if (!is_k) { g = static_cast<int>(rest % pv.n_kv_heads); rest /= pv.n_kv_heads; }
   const int a = static_cast<int>(rest % n_tok);
   const int ll = static_cast<int>(rest / n_tok);
   const int page = slots[2 * a], off = slots[2 * a + 1];
@@ -106,36 +116,55 @@ __global__ void kv_append_rope_kernel(PoolView pv, const int32_t *__restrict__ s
     report(pv.status, PASTA_ERR_DEVICE_CHECK);
     return;
   }
-  const uint4 *src = (kv ? v_new : k_new) + ((static_cast<int64_t>(ll) * n_tok + a) * pv.n_kv_heads + g) * chunks;
-  uint4 lo = __ldg(src + c), hi = __ldg(src + c + half_chunks);
-  if (kv == 0) rope_pairs(lo, hi, pos ? pos[a] : pos0 + a, c * 8, pv.head_dim, log2_theta);
-  uint8_t *block = pv.kv_base + (layer_begin + ll) * pv.layer_stride +
-                   (static_cast<int64_t>(page) * pv.n_kv_heads + g) * kv_block_bytes(pv.head_dim);
-  *reinterpret_cast<uint4 *>(block + kv_chunk_offset(pv.head_dim >> 6, kv, off, c)) = lo;
-  *reinterpret_cast<uint4 *>(block + kv_chunk_offset(pv.head_dim >> 6, kv, off, c + half_chunks)) = hi;
+  uint8_t *layer = pv.kv_base + (layer_begin + ll) * pv.layer_stride;
+  if (is_k) {
+    double sn[8], cs[8];
+    rope_angles(pos ? pos[a] : pos0 + a, c * 8, pv.head_dim, log2_theta, sn, cs);
+#pragma unroll 1
+    for (g = 0; g < pv.n_kv_heads; ++g) {
+      const uint4 *src = k_new + ((static_cast<int64_t>(ll) * n_tok + a) * pv.n_kv_heads + g) * chunks;
+      uint4 lo = __ldg(src + c), hi = __ldg(src + c + half_chunks);
+      rope_apply(lo, hi, sn, cs);
+      uint8_t *block = layer + (static_cast<int64_t>(page) * pv.n_kv_heads + g) * kv_block_bytes(pv.head_dim);
+      *reinterpret_cast<uint4 *>(block + kv_chunk_offset(pv.head_dim >> 6, 0, off, c)) = lo;
+      *reinterpret_cast<uint4 *>(block + kv_chunk_offset(pv.head_dim >> 6, 0, off, c + half_chunks)) = hi;
+    }
+  } else {
+    const uint4 *src = v_new + ((static_cast<int64_t>(ll) * n_tok + a) * pv.n_kv_heads + g) * chunks;
+    uint8_t *block = layer + (static_cast<int64_t>(page) * pv.n_kv_heads + g) * kv_block_bytes(pv.head_dim);
+    *reinterpret_cast<uint4 *>(block + kv_chunk_offset(pv.head_dim >> 6, 1, off, c)) = __ldg(src + c);
+    *reinterpret_cast<uint4 *>(block + kv_chunk_offset(pv.head_dim >> 6, 1, off, c + half_chunks)) = __ldg(src + c + half_chunks);
+  }
 }
 
-// rotates the step's queries in place: q [layer_count, n, Hq, D], positions from the plan
+// rotates the step's queries in place: q [layer_count, n, Hq, D], positions from the plan; one thread per
+// (layer, query, chunk pair), all heads of the query in turn
 __global__ void rope_queries_kernel(const int32_t *__restrict__ pos, int32_t n, int32_t n_q_heads, int32_t D,
                                     int32_t layer_count, uint4 *__restrict__ q, double log2_theta) {
   const int chunks = D >> 3, half_chunks = chunks >> 1;
-  const int64_t total = static_cast<int64_t>(layer_count) * n * n_q_heads * half_chunks;
+  const int64_t total = static_cast<int64_t>(layer_count) * n * half_chunks;
   const int64_t idx = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
   if (idx >= total) return;
   const int c = static_cast<int>(idx % half_chunks);
-  const int64_t vec = idx / half_chunks;                 // (layer, query, head)
-  const int i = static_cast<int>((vec / n_q_heads) % n);
-  uint4 *row = q + vec * chunks;
-  uint4 lo = row[c], hi = row[c + half_chunks];
-  rope_pairs(lo, hi, pos[i], c * 8, D, log2_theta);
-  row[c] = lo;
-  row[c + half_chunks] = hi;
+  const int64_t tok = idx / half_chunks;                 // (layer, query)
+  const int i = static_cast<int>(tok % n);
+  double sn[8], cs[8];
+  rope_angles(pos[i], c * 8, D, log2_theta, sn, cs);
+#pragma unroll 1
+  for (int h = 0; h < n_q_heads; ++h) {
+    uint4 *row = q + (tok * n_q_heads + h) * chunks;
+    uint4 lo = row[c], hi = row[c + half_chunks];
+    rope_apply(lo, hi, sn, cs);
+    row[c] = lo;
+    row[c + half_chunks] = hi;
+  }
 }
 
 cudaError_t launch_kv_append_rope(const PoolView &pv, const int32_t *slots, const int32_t *pos, int32_t pos0, int32_t n_tok,
                                   int32_t layer_begin, int32_t layer_count, const void *k_new, const void *v_new,
                                   double theta, cudaStream_t st) {
-  const int64_t total = static_cast<int64_t>(layer_count) * n_tok * pv.n_kv_heads * 2 * (pv.head_dim >> 4);
+  const int64_t n_k = static_cast<int64_t>(layer_count) * n_tok * (pv.head_dim >> 4);
+  const int64_t total = n_k * (1 + pv.n_kv_heads);        // K threads (all heads each) + V threads (one head each)
   if (total == 0) return cudaSuccess;
   const int threads = 128;
   kv_append_rope_kernel<<<static_cast<unsigned>((total + threads - 1) / threads), threads, 0, st>>>(
@@ -146,7 +175,7 @@ cudaError_t launch_kv_append_rope(const PoolView &pv, const int32_t *slots, cons
 
 cudaError_t launch_rope_queries(const PoolView &pv, const int32_t *pos, int32_t n, int32_t layer_count, void *q, double theta,
                                 cudaStream_t st) {
-  const int64_t total = static_cast<int64_t>(layer_count) * n * pv.n_q_heads * (pv.head_dim >> 4);
+  const int64_t total = static_cast<int64_t>(layer_count) * n * (pv.head_dim >> 4);
   if (total == 0) return cudaSuccess;
   const int threads = 128;
   rope_queries_kernel<<<static_cast<unsigned>((total + threads - 1) / threads), threads, 0, st>>>(
