@@ -126,7 +126,7 @@ class ClockSampler:
 
 
 # ------------------------------------------------------------------------------------------------ our arm
-def build_state(script, device, seed_offset=0, grow_tokens=640):
+def build_state(script, device, seed_offset=0, grow_tokens=640, flags=0):
     """Replays the set-up part of the script (everything before its final step) with device-generated
     bf16 N(0,1) tensors.  Returns the pool and the final step's entries."""
     import torch
@@ -139,7 +139,7 @@ def build_state(script, device, seed_offset=0, grow_tokens=640):
     pool = binding.Pool(geo.n_layers, geo.n_q_heads, geo.n_kv_heads, geo.head_dim, script.n_pages + grow_pages,
                         script.max_requests, script.max_threads_per_request, script.max_segments_per_thread,
                         free_order=order, max_step_queries=len(entries), max_layers_per_launch=geo.n_layers,
-                        device=device.index or 0)
+                        flags=flags, device=device.index or 0)
     gen = torch.Generator(device=device)
     gen.manual_seed(script.seed + 977 * seed_offset)
 
@@ -268,14 +268,17 @@ def run_ours(args):
     if args.layout == "naive_rows":
         pool, entries, randn, spawn_copy_bytes = build_state_naive_rows(script, device, seed_offset=rank, grow_tokens=grow)
     else:
-        pool, entries, randn = build_state(script, device, seed_offset=rank, grow_tokens=grow)
+        from paper_2502_11517_b200 import binding as _b
+        pool, entries, randn = build_state(script, device, seed_offset=rank, grow_tokens=grow,
+                                           flags=_b.FLAG_OUT_BF16 if args.out_dtype == "bf16" else 0)
     n = len(entries)
     reqs = np.asarray([e[0] for e in entries], dtype=np.int32); thr = np.asarray([e[1] for e in entries], dtype=np.int32)
     ones = np.ones(n, dtype=np.int32)
     L = geo.n_layers
     k_new = randn((L, n, geo.n_kv_heads, geo.head_dim)); v_new = randn((L, n, geo.n_kv_heads, geo.head_dim))
     q = randn((L, n, geo.n_q_heads, geo.head_dim))
-    out = torch.empty(q.shape, dtype=torch.float32, device=device)
+    out_dtype = torch.bfloat16 if (args.out_dtype == "bf16" and args.layout == "pool") else torch.float32
+    out = torch.empty(q.shape, dtype=out_dtype, device=device)
     stream = torch.cuda.current_stream(device)
 
     sh = stream.cuda_stream                   # the stream's handle, looked up once
@@ -316,7 +319,7 @@ def run_ours(args):
 
     # ---- end to end: the same step through the host-buffer entry point (copies inside the timed region)
     k_h = k_new.cpu().pin_memory(); v_h = v_new.cpu().pin_memory(); q_h = q.cpu().pin_memory()
-    out_h = torch.empty(q.shape, dtype=torch.float32).pin_memory()
+    out_h = torch.empty(q.shape, dtype=out_dtype).pin_memory()
     staging = torch.empty(pool.step_host_bytes(n), dtype=torch.uint8, device=device)
     for _ in range(3):
         pool.step_host(reqs, thr, ones, k_h, v_h, q_h, out_h, staging)
@@ -330,7 +333,7 @@ def run_ours(args):
     e2e_s = time.perf_counter() - t0
     e2e_tokens, e2e_s = aggregate(float(n * e2e_steps), e2e_s)
     h2d = k_h.numel() * 2 * 2 + q_h.numel() * 2
-    d2h = out_h.numel() * 4
+    d2h = out_h.numel() * out_h.element_size()
 
     # ---- host-only cost of a <sync/> merge (no kernel, no copy): a scratch pool with 16 finished forks
     merge_us = time_sync_merge()
@@ -358,7 +361,8 @@ def run_ours(args):
         "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {
-            "workload": args.workload, "size": args.size, "layout": args.layout, "script": script.name, "requests": len(set(reqs)), "thread_tokens_per_step": n,
+            "workload": args.workload, "size": args.size, "layout": args.layout, "out_dtype": args.out_dtype,
+            "script": script.name, "requests": len(set(reqs)), "thread_tokens_per_step": n,
             "layers": L, "n_q_heads": geo.n_q_heads, "n_kv_heads": geo.n_kv_heads, "head_dim": geo.head_dim,
             "page_size": geo.page_size, "unique_kv_tokens_per_layer": avg_tokens,
             "unique_kv_bytes_per_step": step_bytes, "l2": "inputs larger than L2" if step_bytes / L > 126e6 * 1.5 else
@@ -753,6 +757,8 @@ def main():
     ap.add_argument("--workload", default="long_shared_prefix")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--out-dtype", default="fp32", choices=["fp32", "bf16"],
+                    help="type of the attention output (bf16 halves the device-to-host bytes of the end-to-end path)")
     ap.add_argument("--layout", default="pool", choices=["pool", "naive_rows"],
                     help="pool: the library's shared paged pool (default).  naive_rows: the comparison layout of the "
                          "paper's Appendix B (one dense row per thread, prefix duplicated), on the same kernels")

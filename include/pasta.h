@@ -46,7 +46,10 @@ enum {
 
 enum {
   PASTA_FLAG_HOST_ONLY = 1,      /* bookkeeping only: no CUDA call is ever made, compute entry points return BAD_STATE */
-  PASTA_FLAG_NO_TENSOR_PATH = 2  /* route every stream through the warp-shuffle kernel (debugging / comparison) */
+  PASTA_FLAG_NO_TENSOR_PATH = 2, /* route every stream through the warp-shuffle kernel (debugging / comparison) */
+  PASTA_FLAG_OUT_BF16 = 4        /* `out` of pasta_decode_attn, pasta_step_device and pasta_step_host is bf16 instead of
+                                    fp32 (same shape; the sums stay fp32, one rounding at the end; lse stays fp32).
+                                    pasta_decode_attn_noalloc writes fp32 only and returns BAD_STATE on such a pool. */
 };
 
 /* thread states reported by pasta_pool_dump */

@@ -15,7 +15,7 @@ import numpy as np
 from .build import LIB
 
 OK, INVALID_ARG, OUT_OF_PAGES, BAD_STATE, CAPACITY, CUDA, DEVICE_CHECK, TIMEOUT = range(8)
-FLAG_HOST_ONLY, FLAG_NO_TENSOR_PATH = 1, 2
+FLAG_HOST_ONLY, FLAG_NO_TENSOR_PATH, FLAG_OUT_BF16 = 1, 2, 4
 _NAMES = ["OK", "INVALID_ARG", "OUT_OF_PAGES", "BAD_STATE", "CAPACITY", "CUDA", "DEVICE_CHECK", "TIMEOUT"]
 
 EXPORTS = [

@@ -146,6 +146,7 @@ namespace pasta {
 bool pool_step_view(pasta_pool_t *p, PoolView *pv, PlanHeader *hdr, int32_t *n_layers, int32_t *head_dim,
                     int32_t *device) {
   if (p->host_only || !p->plan_valid) return false;
+  if (p->cfg.flags & PASTA_FLAG_OUT_BF16) return false;      // that entry point writes fp32 only
   *pv = p->pv;
   *hdr = p->hdr;
   *n_layers = p->cfg.n_layers;
@@ -407,7 +408,8 @@ pasta_status_t pasta_decode_attn(pasta_pool_t *p, int32_t layer_begin, int32_t l
   for (int32_t done = 0; done < layer_count; done += p->d.layers_per_launch) {
     const int32_t cnt = std::min(p->d.layers_per_launch, layer_count - done);
     const uint16_t *qg = static_cast<const uint16_t *>(q) + size_t(done) * q_layer;
-    float *og = static_cast<float *>(out) + size_t(done) * q_layer;
+    const bool out_bf16 = (p->cfg.flags & PASTA_FLAG_OUT_BF16) != 0;
+    void *og = static_cast<uint8_t *>(out) + size_t(done) * q_layer * (out_bf16 ? 2 : 4);
     float *lg = lse ? lse + size_t(done) * n * p->cfg.n_q_heads : nullptr;
     const bool timed = p->profiling && p->prof_calls < kProfCalls;
     cudaEvent_t *ev = timed ? &p->prof_events[4 * p->prof_calls] : nullptr;
@@ -425,7 +427,7 @@ pasta_status_t pasta_decode_attn(pasta_pool_t *p, int32_t layer_begin, int32_t l
       mask |= 2;
     }
     if (timed) PASTA_CUDA(cudaEventRecord(ev[2], st));
-    PASTA_CUDA(launch_merge(p->pv, p->hdr, cnt, og, lg, st));
+    PASTA_CUDA(launch_merge(p->pv, p->hdr, cnt, og, lg, st, out_bf16));
     p->launches += 1;
     mask |= 4;
     if (timed) {
@@ -539,7 +541,8 @@ pasta_status_t pasta_step_host(pasta_pool_t *p, int32_t n, const int32_t *req_id
   if (s != PASTA_OK) return s;
   s = pasta_decode_attn(p, 0, p->cfg.n_layers, q_dev, o_dev, nullptr, scale, stream);
   if (s != PASTA_OK) return s;
-  PASTA_CUDA(cudaMemcpyAsync(out, o_dev, q_bytes * 2, cudaMemcpyDeviceToHost, st));
+  const size_t out_bytes = (p->cfg.flags & PASTA_FLAG_OUT_BF16) ? q_bytes : q_bytes * 2;
+  PASTA_CUDA(cudaMemcpyAsync(out, o_dev, out_bytes, cudaMemcpyDeviceToHost, st));
   PASTA_CUDA(cudaStreamSynchronize(st));
   return PASTA_OK;
 }

@@ -428,9 +428,10 @@ cudaError_t launch_attn_warp(const PoolView &pv, const PlanHeader &h, int32_t la
 // Which partial rows belong to a (query, head) is the same for every layer, so the look-ups in the plan are made
 // once per warp, and the (m, l) pairs of the next layer are fetched while this layer's outputs are summed.
 // =============================================================================================
+template <bool kOutBf16>
 __global__ void __launch_bounds__(256)
 merge_kernel(PoolView pv, int32_t n_queries, int32_t layer_count, int32_t off_query, int32_t off_trange,
-             int32_t off_tunit, int32_t t_rows, int32_t layers_per_warp, float *__restrict__ out,
+             int32_t off_tunit, int32_t t_rows, int32_t layers_per_warp, void *__restrict__ out_raw,
              float *__restrict__ lse) {
   const int D = pv.head_dim, Hq = pv.n_q_heads, G = Hq / pv.n_kv_heads;
   const int64_t gw = (static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x) >> 5;
@@ -504,16 +505,28 @@ merge_kernel(PoolView pv, int32_t n_queries, int32_t layer_count, int32_t off_qu
       }
     }
     const float inv = L > 0.f ? 1.f / L : 0.f;
-    float *dst = out + ((static_cast<int64_t>(ll) * n_queries + n) * Hq + h) * D + lane * E;
-    if (E == 4) *reinterpret_cast<float4 *>(dst) = make_float4(acc[0] * inv, acc[1] * inv, acc[2] * inv, acc[3] * inv);
-    else *reinterpret_cast<float2 *>(dst) = make_float2(acc[0] * inv, acc[1] * inv);
+    const int64_t at = ((static_cast<int64_t>(ll) * n_queries + n) * Hq + h) * D + lane * E;
+    if (kOutBf16) {
+      __nv_bfloat16 *dst = static_cast<__nv_bfloat16 *>(out_raw) + at;
+      const __nv_bfloat162 p0 = __floats2bfloat162_rn(acc[0] * inv, acc[1] * inv);
+      if (E == 4) {
+        const __nv_bfloat162 p1 = __floats2bfloat162_rn(acc[2] * inv, acc[3] * inv);
+        *reinterpret_cast<uint2 *>(dst) = make_uint2(*reinterpret_cast<const uint32_t *>(&p0), *reinterpret_cast<const uint32_t *>(&p1));
+      } else {
+        *reinterpret_cast<__nv_bfloat162 *>(dst) = p0;
+      }
+    } else {
+      float *dst = static_cast<float *>(out_raw) + at;
+      if (E == 4) *reinterpret_cast<float4 *>(dst) = make_float4(acc[0] * inv, acc[1] * inv, acc[2] * inv, acc[3] * inv);
+      else *reinterpret_cast<float2 *>(dst) = make_float2(acc[0] * inv, acc[1] * inv);
+    }
     if (lse && lane == 0)
       lse[(static_cast<int64_t>(ll) * n_queries + n) * Hq + h] = (mstar + log2f(L)) * 0.6931471805599453f;
   }
 }
 
-cudaError_t launch_merge(const PoolView &pv, const PlanHeader &h, int32_t layer_count, float *out, float *lse,
-                         cudaStream_t st) {
+cudaError_t launch_merge(const PoolView &pv, const PlanHeader &h, int32_t layer_count, void *out, float *lse,
+                         cudaStream_t st, bool out_bf16) {
   const int64_t per_group = static_cast<int64_t>(h.w[PH_N_QUERIES]) * pv.n_q_heads;
   if (per_group == 0 || layer_count == 0) return cudaSuccess;
   // enough warps to fill the machine a few times over; beyond that, more layers per warp (its plan look-ups are shared)
@@ -522,9 +535,14 @@ cudaError_t launch_merge(const PoolView &pv, const PlanHeader &h, int32_t layer_
   const int32_t layers_per_warp = static_cast<int32_t>((layer_count + groups - 1) / groups);
   const int64_t warps = per_group * ((layer_count + layers_per_warp - 1) / layers_per_warp);
   const int64_t blocks = (warps * 32 + 255) / 256;
-  merge_kernel<<<static_cast<unsigned>(blocks), 256, 0, st>>>(pv, h.w[PH_N_QUERIES], layer_count, h.w[PH_OFF_QUERY],
-                                                              h.w[PH_OFF_TRANGE], h.w[PH_OFF_TUNIT], h.w[PH_T_ROWS],
-                                                              layers_per_warp, out, lse);
+  if (out_bf16)
+    merge_kernel<true><<<static_cast<unsigned>(blocks), 256, 0, st>>>(pv, h.w[PH_N_QUERIES], layer_count, h.w[PH_OFF_QUERY],
+                                                                      h.w[PH_OFF_TRANGE], h.w[PH_OFF_TUNIT], h.w[PH_T_ROWS],
+                                                                      layers_per_warp, out, lse);
+  else
+    merge_kernel<false><<<static_cast<unsigned>(blocks), 256, 0, st>>>(pv, h.w[PH_N_QUERIES], layer_count, h.w[PH_OFF_QUERY],
+                                                                       h.w[PH_OFF_TRANGE], h.w[PH_OFF_TUNIT], h.w[PH_T_ROWS],
+                                                                       layers_per_warp, out, lse);
   return cudaGetLastError();
 }
 

@@ -33,7 +33,8 @@ cudaError_t launch_attn_tensor(const PoolView &pv, const PlanHeader &h, int32_t 
                                const void *q, float scale_log2, cudaStream_t st);
 bool tensor_path_available();       // false while the tensor-core kernel is compiled out
 // K4: log-sum-exp merge of all partial rows of every (query, head)
-cudaError_t launch_merge(const PoolView &pv, const PlanHeader &h, int32_t layer_count, float *out, float *lse,
-                         cudaStream_t st);
+// out: device fp32 [layer_count, n, Hq, D], or bf16 of the same shape when out_bf16
+cudaError_t launch_merge(const PoolView &pv, const PlanHeader &h, int32_t layer_count, void *out, float *lse,
+                         cudaStream_t st, bool out_bf16 = false);
 
 }  // namespace pasta

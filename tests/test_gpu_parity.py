@@ -203,6 +203,33 @@ def test_step_device_entry_point_equals_the_three_calls(lib):
     assert torch.equal(outs[0][0], outs[1][0]) and torch.equal(outs[0][1], outs[1][1]) and outs[0][2] == outs[1][2]
 
 
+def test_bf16_output_option(lib):
+    """The same step with fp32 and with bf16 outputs: the bf16 result is the fp32 one rounded once."""
+    import torch
+    from lib_replay import LibReplay, make_pool
+    outs = {}
+    for flag in (0, lib.FLAG_OUT_BF16):
+        script = cfg2_single_request("b")
+        pool = make_pool(script, flags=flag)
+        rep = LibReplay(script, pool)
+        first = next(i for i, op in enumerate(script.ops) if op[0] == "step")
+        for i in range(first):
+            rep.apply(i)
+        op = script.ops[first]
+        L = range(script.geometry.n_layers)
+        ks, vs, qs = zip(*[step_tensors(script, first, l) for l in L])
+        k = torch.stack(ks).cuda(); v = torch.stack(vs).cuda(); q = torch.stack(qs).cuda()
+        out = torch.empty(q.shape, dtype=torch.bfloat16 if flag else torch.float32, device="cuda")
+        lse = torch.empty(q.shape[:3], dtype=torch.float32, device="cuda")
+        pool.step_device([e[0] for e in op[1]], [e[1] for e in op[1]], [e[2] for e in op[1]], k, v, q, out, lse)
+        torch.cuda.synchronize()
+        assert pool.status() == 0
+        outs[flag] = (out.cpu(), lse.cpu())
+        pool.close()
+    assert torch.equal(outs[0][0].to(torch.bfloat16), outs[lib.FLAG_OUT_BF16][0])
+    assert torch.equal(outs[0][1], outs[lib.FLAG_OUT_BF16][1])
+
+
 def test_step_host_entry_point(lib):
     """The host-buffer entry point (copies inside the call) gives the same numbers as the device one."""
     import torch
