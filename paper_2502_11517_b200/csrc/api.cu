@@ -518,25 +518,30 @@ pasta_status_t pasta_step_host(pasta_pool_t *p, int32_t n, const int32_t *req_id
   if (s != PASTA_OK) return s;
   if (staging_bytes < need || (reinterpret_cast<uintptr_t>(staging) & 255)) return PASTA_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  if (n_new)
-    for (int32_t i = 0; i < n; ++i)
-      if (n_new[i] > 1) return PASTA_ERR_INVALID_ARG;   // the staging layout is one query per entry
-  s = pasta_step_begin(p, n, req_ids, thread_ids, n_new, stream);
-  if (s != PASTA_OK) return s;
+  size_t n_app = static_cast<size_t>(n);
+  if (n_new) {
+    n_app = 0;
+    for (int32_t i = 0; i < n; ++i) {
+      if (n_new[i] < 0 || n_new[i] > 1) return PASTA_ERR_INVALID_ARG;   // the staging layout is one query per entry
+      n_app += static_cast<size_t>(n_new[i]);
+    }
+  }
   const size_t L = p->cfg.n_layers, d = p->cfg.head_dim;
-  const size_t n_app = p->hdr.w[PH_N_APPEND];
   const size_t kv_full = align_up(L * n * p->cfg.n_kv_heads * d * 2, 256);
   const size_t kv_bytes = L * n_app * p->cfg.n_kv_heads * d * 2;
   const size_t q_bytes = L * n * p->cfg.n_q_heads * d * 2;
   uint8_t *base = static_cast<uint8_t *>(staging);
   uint8_t *k_dev = base, *v_dev = base + kv_full, *q_dev = base + 2 * kv_full;
   uint8_t *o_dev = q_dev + align_up(q_bytes, 256);
+  if (n_app > 0 && (!k_new || !v_new)) return PASTA_ERR_INVALID_ARG;
+  // the input copies go first: the host plans the step while they are in flight
   if (n_app > 0) {
-    if (!k_new || !v_new) return PASTA_ERR_INVALID_ARG;
     PASTA_CUDA(cudaMemcpyAsync(k_dev, k_new, kv_bytes, cudaMemcpyHostToDevice, st));
     PASTA_CUDA(cudaMemcpyAsync(v_dev, v_new, kv_bytes, cudaMemcpyHostToDevice, st));
   }
   PASTA_CUDA(cudaMemcpyAsync(q_dev, q, q_bytes, cudaMemcpyHostToDevice, st));
+  s = pasta_step_begin(p, n, req_ids, thread_ids, n_new, stream);
+  if (s != PASTA_OK) return s;
   s = pasta_kv_append(p, 0, p->cfg.n_layers, k_dev, v_dev, stream);
   if (s != PASTA_OK) return s;
   s = pasta_decode_attn(p, 0, p->cfg.n_layers, q_dev, o_dev, nullptr, scale, stream);
