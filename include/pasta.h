@@ -230,8 +230,9 @@ pasta_status_t pasta_step_device(pasta_pool_t *pool, int32_t n, const int32_t *r
                                  float *lse, float scale, void *stream);
 
 /*
- * One whole step with HOST tensors: step_begin, copy k_new / v_new / q to the device, kv_append
- * and decode_attn for all layers, copy `out` back, synchronise the stream.  k_new, v_new:
+ * One whole step with HOST tensors: the copies of k_new / v_new / q to the device are enqueued, the step is
+ * planned while they are in flight (step_begin), then kv_append and decode_attn for all layers, `out` is copied
+ * back and the stream synchronised.  k_new, v_new:
  * host bf16 [n_layers, n_app, n_kv_heads, head_dim]; q: host bf16 [n_layers, n, n_q_heads, head_dim];
  * out: host fp32 like q.  staging: device scratch of at least pasta_step_host_bytes(pool, n)
  * bytes, caller-owned.  Pinned host memory makes the copies asynchronous; pageable works too.
