@@ -189,6 +189,14 @@ __device__ __forceinline__ bool wait_or_abort(uint32_t bar, uint32_t parity, vol
   }
 }
 
+// bulk copy whose lines are the first to leave L2: every page is read once per launch
+__device__ __forceinline__ void bulk_g2s_stream(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar, uint64_t policy) {
+  asm volatile(
+      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
+      ::"r"(dst), "l"(src), "r"(bytes), "r"(bar), "l"(policy)
+      : "memory");
+}
+
 struct UnitInfo {
   int treq, g, tile_begin, tile_end, row_base;
   int page_off, n_pages, n_threads, n_streams, vis_off, tq_off;
@@ -259,6 +267,8 @@ attn_tensor_kernel(PoolView pv, TensorArgs a, const __nv_bfloat16 *__restrict__ 
     // ================================================================ producer
     uint32_t it = 0;
     bool ok = true;
+    uint64_t policy;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
     for (int ll = 0; ll < a.layer_count && ok; ++ll) {
       const uint8_t *kv_layer = pv.kv_base + (a.layer_begin + ll) * pv.layer_stride;
       for (int u = u0; u < u1 && ok; ++u) {
@@ -286,9 +296,9 @@ attn_tensor_kernel(PoolView pv, TensorArgs a, const __nv_bfloat16 *__restrict__ 
           if (lane == 0) mbar_expect_tx(bar + 8 * (B_FULL + s), n_valid * T_BLOCK);
           __syncwarp();
           if (lane < n_valid)
-            bulk_g2s(base + OFF_STAGE + s * T_STAGE_BYTES + lane * T_BLOCK,
-                     kv_layer + (static_cast<int64_t>(page) * pv.n_kv_heads + x.g) * T_BLOCK, T_BLOCK,
-                     bar + 8 * (B_FULL + s));
+            bulk_g2s_stream(base + OFF_STAGE + s * T_STAGE_BYTES + lane * T_BLOCK,
+                            kv_layer + (static_cast<int64_t>(page) * pv.n_kv_heads + x.g) * T_BLOCK, T_BLOCK,
+                            bar + 8 * (B_FULL + s), policy);
         }
       }
     }
