@@ -40,7 +40,7 @@ SEED_EXTRAS = 2502115
 FALLBACK_HBM_GBS = 6650.0
 # dram bytes (read + write) of one launch of the dominant kernel from an ncu capture of this workload,
 # or None when no capture matches the current kernel
-NCU_TRAFFIC_BYTES = {}   # (workload, size) -> DRAM bytes per launch of the dominant kernel, from profiles/
+NCU_TRAFFIC_BYTES = {("long_shared_prefix", "full"): 1.2111e9, ("long_shared_prefix", "small"): 3.945e8}   # see profiles/
 
 
 def make_script(workload: str, size: str = "full"):
