@@ -17,7 +17,9 @@
 //
 // Warp roles: warp 0 producer (eight lanes issue the bulk copies of a tile's (page, kv head) blocks into a
 // 3-stage ring of 64 KB), warp 1 MMA issue (one thread), warps 2-3 build the stacked, swizzled Q operand of each
-// unit, warps 4-7 and 8-11 the two softmax groups (thread i of a group owns row i = TMEM lane i).
+// unit, warps 4-7 and 8-11 the two softmax groups (a thread owns the row held in its TMEM lane: row i is in lane i
+// when the unit's MMAs have M = 128; a unit with at most 64 rows uses M = 64, which puts row i in lane
+// 32 (i / 16) + i % 16).
 // Every wait is bounded; on expiry the CTA reports PASTA_ERR_TIMEOUT, drains and leaves.
 #include "device_common.cuh"
 #include "kernels.hpp"
@@ -53,10 +55,13 @@ static_assert(T_SMEM_BYTES <= 232448, "shared memory budget");
 constexpr uint32_t TMEM_COLS = 512;
 constexpr uint32_t COL_S = 0, COL_O = 256;   // S[b] at 128 b (group g: columns 64 g .. 64 g + 63; its P reuses the first 32), O_g at 256 + 128 g
 
-// instruction descriptors: D fp32, A/B bf16, M = 128
-constexpr uint32_t IDESC_BASE = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 4) << 24);
+// instruction descriptors: D fp32, A/B bf16; M = 128, or M = 64 for a unit with at most 64 stacked rows (half the
+// tensor-core work per tile: long runs are power-limited, and the tensor cores are what draws the power)
+constexpr uint32_t IDESC_BASE = (1u << 4) | (1u << 7) | (1u << 10);
+constexpr uint32_t IDESC_M128 = (128u >> 4) << 24, IDESC_M64 = (64u >> 4) << 24;
 constexpr uint32_t IDESC_QK = IDESC_BASE | ((128u >> 3) << 17);                // N = 128, both operands K-major
 constexpr uint32_t IDESC_PV = IDESC_BASE | ((128u >> 3) << 17) | (1u << 16);   // N = 128, B (= V) MN-major
+constexpr int T_M64_ROWS = 64;
 
 __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
   return static_cast<uint64_t>((addr & 0x3FFFFu) >> 4) | (static_cast<uint64_t>(lbo_bytes >> 4) << 16) |
@@ -317,6 +322,7 @@ attn_tensor_kernel(PoolView pv, TensorArgs a, const __nv_bfloat16 *__restrict__ 
         for (int u = u0; u < u1 && ok; ++u, ++uc) {
           const UnitInfo x = load_unit(plan, a.off_tunit, a.off_treq, u);
           const int nt = x.tile_end - x.tile_begin;
+          const uint32_t m_bits = x.n_threads * G <= T_M64_ROWS ? IDESC_M64 : IDESC_M128;
           if (!wait_or_abort(bar + 8 * B_QFULL, uc & 1, abort_flag)) { ok = false; break; }
           tc_fence_after();
           for (int k = 0; k <= nt && ok; ++k) {
@@ -330,7 +336,7 @@ attn_tensor_kernel(PoolView pv, TensorArgs a, const __nv_bfloat16 *__restrict__ 
               for (int ks = 0; ks < 8; ++ks) {
                 const uint32_t half = ks >> 2, kk = ks & 3;
                 mma_ss(tmem + COL_S + b * T_TILE, smem_desc(q_addr + half * 16384 + kk * 32, 16, 1024),
-                       smem_desc(k_addr + half * 1024 + kk * 32, 16, 4096), IDESC_QK, ks > 0);
+                       smem_desc(k_addr + half * 1024 + kk * 32, 16, 4096), IDESC_QK | m_bits, ks > 0);
               }
               mma_commit(bar + 8 * (B_SFULL + b));
               if (k == nt - 1) mma_commit(bar + 8 * B_QFREE);   // the Q operand may be replaced once these finish
@@ -349,7 +355,8 @@ attn_tensor_kernel(PoolView pv, TensorArgs a, const __nv_bfloat16 *__restrict__ 
 #pragma unroll
                 for (int pg = 0; pg < T_HALF_PAGES; ++pg)
                   mma_ts(tmem + COL_O + g2 * 128, tmem + COL_S + b * T_TILE + g2 * T_HALF + pg * 8,
-                         smem_desc(v_addr + (g2 * T_HALF_PAGES + pg) * T_BLOCK, 1024, 4096), IDESC_PV, (k > 1) || (pg > 0));
+                         smem_desc(v_addr + (g2 * T_HALF_PAGES + pg) * T_BLOCK, 1024, 4096), IDESC_PV | m_bits,
+                         (k > 1) || (pg > 0));
               }
               if (!ok) break;
               mma_commit(bar + 8 * (B_EMPTY + s));
@@ -400,7 +407,7 @@ attn_tensor_kernel(PoolView pv, TensorArgs a, const __nv_bfloat16 *__restrict__ 
   } else {
     // ================================================================ softmax + epilogue (2 groups of 128 threads)
     const int grp = (warp - 4) >> 2;                // this group's half of every tile: pages 4 grp .. 4 grp + 3
-    const int row = (tid - 128) & 127;              // = TMEM lane
+    const int wq = warp & 3;                        // the TMEM lanes this warp reaches: 32 wq .. 32 wq + 31
     const uint32_t lane_addr = static_cast<uint32_t>((warp & 3) * 32) << 16;
     const uint32_t col_o = COL_O + grp * 128;
     float2 *ml1 = reinterpret_cast<float2 *>(sm + OFF_ML1);
@@ -411,8 +418,12 @@ attn_tensor_kernel(PoolView pv, TensorArgs a, const __nv_bfloat16 *__restrict__ 
         const UnitInfo x = load_unit(plan, a.off_tunit, a.off_treq, u);
         const int nt = x.tile_end - x.tile_begin;
         const int rows = x.n_threads * G;
+        // M = 128: row i of the score matrix sits in TMEM lane i.  M = 64: row i sits in lane 32 (i / 16) + i % 16, so
+        // a warp owns 16 rows and its upper 16 lanes hold nothing (whatever they compute is never read or written out)
+        const bool m64 = rows <= T_M64_ROWS;
+        const int row = m64 ? (lane < 16 ? wq * 16 + lane : 128) : wq * 32 + lane;
         const bool active = row < rows;
-        const bool warp_active = ((warp - 4) & 3) * 32 < rows;
+        const bool warp_active = (m64 ? wq * 16 : wq * 32) < rows;
         const int32_t *visrow = plan + a.off_vis + x.vis_off + (active ? row / G : 0) * x.n_streams;
         // the row's visible lengths of the first four local streams stay in registers for the whole unit: a global
         // load per page would otherwise sit between two tiles of this group
@@ -484,7 +495,7 @@ attn_tensor_kernel(PoolView pv, TensorArgs a, const __nv_bfloat16 *__restrict__ 
             }
             const float mt = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * a.scale_log2;
             const bool need = mt > m_ref + 8.f;       // also true for the first visible tile (m_ref = -inf)
-            const bool rescale = need && l > 0.f;
+            const bool rescale = active && need && l > 0.f;
             if (__any_sync(0xffffffffu, rescale)) {
               // O_g and l are relative to m_ref: move them to the new reference.  The accumulator is quiet once the
               // P.V of the previous tile has finished, which is what releases that tile's stage.

@@ -1,6 +1,7 @@
 """GPU parity on the edges of the method and of the kernels' limits: empty steps, one-token contexts, ragged page
 and tile boundaries, exactly as many stacked rows as the tensor-core tile holds and one thread more, every supported
-group size, more streams than the tensor-core path takes, forks with empty chunks."""
+group size, row counts on both sides of the half-height MMA tile, more streams than the tensor-core path takes, forks
+with empty chunks."""
 import numpy as np
 import pytest
 
@@ -54,6 +55,22 @@ def test_as_many_rows_as_the_tile_holds_and_one_thread_more(lib, n_forks, tensor
     assert (w[4] > 0) == tensor_units and (w[5] > 0) == (not tensor_units)     # t-units / w-units of the plan
     pool.close()
     run_script(lib, script, max_step_queries=64)
+
+
+@pytest.mark.parametrize("n_forks", [0, 3, 4, 7, 8, 11, 15, 16])
+def test_row_counts_around_the_half_height_tile(lib, n_forks):
+    """Units of at most 64 stacked rows run their MMAs with M = 64 (another row-to-lane layout in tensor memory), larger
+    ones with M = 128: 1, 4, 5, 8, 9, 12, 16 and 17 threads of group 4 cover every warp's first and last row on both
+    sides of the switch; a second request with 20 threads puts both kinds of unit into one launch."""
+    geo = Geometry(1, 32, 8, 128, 16)
+    ops = [("begin", 0), ("run", 0, 0, 333), ("begin", 1), ("run", 1, 0, 150)]
+    for t in range(1, n_forks + 1):
+        ops += [("spawn", 0, t), ("run", 0, t, 1 + (7 * t) % 40)]
+    for t in range(1, 20):
+        ops += [("spawn", 1, t), ("run", 1, t, 2 + t % 9)]
+    ops.append(("step", tuple((0, t, 1) for t in range(n_forks + 1)) + tuple((1, t, 1) for t in range(20))))
+    ops.append(("step", tuple((0, t, 1) for t in range(n_forks + 1))))
+    run_script(lib, manual(ops, geo, n_pages=400, max_threads=24), max_step_queries=64)
 
 
 @pytest.mark.parametrize("hq,hkv,d", [(8, 8, 128), (8, 4, 128), (16, 2, 128), (8, 8, 64), (16, 2, 64)])
