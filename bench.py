@@ -351,7 +351,14 @@ def run_ours(args):
     timed_steps = max(1, max(kernel_launches))                 # one launch of each kernel per step
     dom = 0 if kernel_launches[0] else 1                       # tensor-core kernel when the workload has shared streams
     dom_name = ["attn_tensor_kernel", "attn_warp_kernel"][dom]
-    dom_bytes_per_launch = shared_bytes if dom == 0 else step_bytes - shared_bytes
+    # the per-kernel events cover the first `timed_steps` steps of the timed region (the library keeps a bounded
+    # number of them), and every step lengthens each stream by one token: bytes of the average step among those
+    frac_timed = min(1.0, timed_steps / max(1, args.steps))
+    tok_p = tok0 + (tok1 - tok0) * frac_timed
+    shared_p = shared0 + (shared1 - shared0) * frac_timed
+    prof_step_bytes = ((tok0 + tok_p) / 2.0 + n / 2.0) * B_tok * L
+    prof_shared_bytes = (shared0 + shared_p) / 2.0 * B_tok * L
+    dom_bytes_per_launch = prof_shared_bytes if dom == 0 else prof_step_bytes - prof_shared_bytes
     dom_ms = kernel_ms[dom] / max(1, kernel_launches[dom])
     achieved = dom_bytes_per_launch / (dom_ms * 1e-3) / 1e9 if dom_ms > 0 else 0.0
     value = all_tokens / (ms * 1e-3)
