@@ -125,10 +125,13 @@ pasta_status_t build_plan(const HostPool &pool, const std::vector<StepQuery> &en
         const int32_t np = (u.max_vis + P - 1) / P;
         int32_t min_vis = u.max_vis;             // what EVERY thread of the request sees of this stream
         for (int32_t ti = 0; ti < T; ++ti) min_vis = std::min(min_vis, q_vis[ti][ui]);
-        for (int32_t k = 0; k < np; ++k) {
-          pages.push_back(sp[k]);
-          pmeta.push_back((k << 8) | u.local | ((k + 1) * P <= min_vis ? PASTA_PMETA_ALL_VISIBLE : 0));
-        }
+        pages.insert(pages.end(), sp.begin(), sp.begin() + np);
+        const size_t m0 = pmeta.size();
+        pmeta.resize(m0 + np);
+        int32_t *pm = pmeta.data() + m0;
+        const int32_t n_all = std::min(np, min_vis / P);     // pages every thread of the request sees in full
+        for (int32_t k = 0; k < n_all; ++k) pm[k] = (k << 8) | u.local | PASTA_PMETA_ALL_VISIBLE;
+        for (int32_t k = n_all; k < np; ++k) pm[k] = (k << 8) | u.local;
       }
       t.n_pages = static_cast<int32_t>(pages.size()) - t.page_off;
       for (int32_t ti = 0; ti < T; ++ti) {
@@ -255,6 +258,10 @@ pasta_status_t build_plan(const HostPool &pool, const std::vector<StepQuery> &en
   int32_t n_app = 0;
   for (const Slot &s : slots) n_app += s.page >= 0;
   std::vector<int32_t> &w = *out;
+  w.clear();
+  w.reserve(PH_WORDS + pages.size() + pmeta.size() + vis_tab.size() + tq_tab.size() + trange.size() + tcta.size() +
+            wunits.size() + tunits.size() * PU_WORDS + treqs.size() * PT_WORDS + static_cast<size_t>(n) * (PQ_WORDS + 4) +
+            64);
   w.assign(PH_WORDS, 0);
   auto put = [&](int off_field, const std::vector<int32_t> &v) {
     w[off_field] = static_cast<int32_t>(w.size());
