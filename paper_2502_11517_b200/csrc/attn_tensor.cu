@@ -599,11 +599,10 @@ bool tensor_path_available() { return true; }
 cudaError_t launch_attn_tensor(const PoolView &pv, const PlanHeader &h, int32_t layer_begin, int32_t layer_count,
                                const void *q, float scale_log2, cudaStream_t st) {
   if (pv.head_dim != 128) return cudaErrorInvalidValue;
-  static bool prepared = false;
-  if (!prepared) {
-    cudaError_t e = cudaFuncSetAttribute(attn_tensor_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, T_SMEM_BYTES);
+  static uint64_t prepared = 0;
+  {
+    cudaError_t e = raise_smem_limit(reinterpret_cast<const void *>(attn_tensor_kernel), T_SMEM_BYTES, &prepared);
     if (e != cudaSuccess) return e;
-    prepared = true;
   }
   const int grid = h.w[PH_T_GRID];
   if (grid == 0 || layer_count == 0) return cudaSuccess;

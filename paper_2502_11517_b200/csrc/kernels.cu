@@ -396,11 +396,10 @@ template <int D, int G>
 static cudaError_t launch_warp_t(const PoolView &pv, const PlanHeader &h, int32_t layer_begin, int32_t layer_count,
                                  const void *q, float scale_log2, cudaStream_t st) {
   using S = WarpSmem<D, G>;
-  static bool prepared = false;
-  if (!prepared) {
-    cudaError_t e = cudaFuncSetAttribute(attn_warp_kernel<D, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, S::TOTAL);
+  static uint64_t prepared = 0;
+  {
+    cudaError_t e = raise_smem_limit(reinterpret_cast<const void *>(attn_warp_kernel<D, G>), S::TOTAL, &prepared);
     if (e != cudaSuccess) return e;
-    prepared = true;
   }
   const int64_t warps = static_cast<int64_t>(h.w[PH_N_WUNITS]) * layer_count;
   if (warps == 0) return cudaSuccess;

@@ -12,6 +12,19 @@ struct PlanHeader {            // host copy of the plan's header words
   int32_t w[32];
 };
 
+// Raises a kernel's dynamic shared-memory limit once per device of the process (the attribute belongs to the device's
+// context, so a second pool on another GPU needs it again).  `done` holds one bit per device ordinal.
+inline cudaError_t raise_smem_limit(const void *kernel, int bytes, uint64_t *done) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev >= 0 && dev < 64 && ((*done >> dev) & 1)) return cudaSuccess;
+  e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  if (e != cudaSuccess) return e;
+  if (dev >= 0 && dev < 64) *done |= 1ull << dev;
+  return cudaSuccess;
+}
+
 // K1: copies the new tokens of `layer_count` layers into their slots.  slots: device, 2 words per token.
 cudaError_t launch_kv_append(const PoolView &pv, const int32_t *slots, int32_t n_tok, int32_t layer_begin,
                              int32_t layer_count, const void *k_new, const void *v_new, cudaStream_t st);
