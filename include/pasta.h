@@ -302,8 +302,11 @@ pasta_status_t pasta_pool_status(pasta_pool_t *pool, void *stream);
 pasta_status_t pasta_launch_count(pasta_pool_t *pool, int64_t *out);
 
 /*
- * Kernel timing for benchmarks.  While enabled, pasta_decode_attn brackets each of its kernels with
- * CUDA events on the launching stream (at most 512 launches are kept between two reads).
+ * Kernel timing for benchmarks.  on = 0 switches it off; on = k >= 1 makes every k-th pasta_decode_attn launch group
+ * (the first one included) bracket each of its kernels with CUDA events on the launching stream (at most 512 timed
+ * groups are kept between two reads; on < 0 is INVALID_ARG).  A timing event between two kernels keeps the second from
+ * starting until its time stamp is written, which costs a few microseconds per event: time every launch (k = 1) only
+ * where that does not matter, and sample (k = 8, say) inside a region whose total time is being measured.
  * pasta_profile_read waits for the recorded events and returns, accumulated since the previous read:
  * out_ms[0..2] = device milliseconds of the tensor-core pass, the warp-shuffle pass and the merge,
  * out_launches[0..2] = how many launches of each were timed.  Both arrays are host memory.

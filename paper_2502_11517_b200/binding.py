@@ -310,7 +310,8 @@ class Pool:
         st = C.c_void_p(0) if self.host_only else _stream(stream)
         return lib().pasta_pool_status(self._h, st)
 
-    def profile_enable(self, on: bool = True) -> None:
+    def profile_enable(self, on=True) -> None:
+        """False / 0: off; True / 1: time every launch group; k > 1: time every k-th one."""
         _check(lib().pasta_profile_enable(self._h, int(on)), "pasta_profile_enable")
 
     def profile_read(self):

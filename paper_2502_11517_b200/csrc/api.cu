@@ -92,6 +92,8 @@ struct pasta_pool {
   int64_t step_index = 0;
   // kernel timing (pasta_profile_*): events[4 * i .. 4 * i + 3] bracket the three kernels of call i
   bool profiling = false;
+  int prof_stride = 1;                  // every prof_stride-th pasta_decode_attn launch group is timed
+  int64_t prof_seen = 0;                // launch groups since profiling was enabled
   std::vector<cudaEvent_t> prof_events;
   std::vector<uint8_t> prof_mask;       // per call: bit k set if kernel k was launched
   int prof_calls = 0;
@@ -411,7 +413,7 @@ pasta_status_t pasta_decode_attn(pasta_pool_t *p, int32_t layer_begin, int32_t l
     const bool out_bf16 = (p->cfg.flags & PASTA_FLAG_OUT_BF16) != 0;
     void *og = static_cast<uint8_t *>(out) + size_t(done) * q_layer * (out_bf16 ? 2 : 4);
     float *lg = lse ? lse + size_t(done) * n * p->cfg.n_q_heads : nullptr;
-    const bool timed = p->profiling && p->prof_calls < kProfCalls;
+    const bool timed = p->profiling && p->prof_calls < kProfCalls && (p->prof_seen++ % p->prof_stride) == 0;
     cudaEvent_t *ev = timed ? &p->prof_events[4 * p->prof_calls] : nullptr;
     uint8_t mask = 0;
     if (timed) PASTA_CUDA(cudaEventRecord(ev[0], st));
@@ -621,7 +623,10 @@ pasta_status_t pasta_profile_enable(pasta_pool_t *p, int32_t on) {
     p->prof_mask.assign(kProfCalls, 0);
     for (cudaEvent_t &e : p->prof_events) PASTA_CUDA(cudaEventCreate(&e));
   }
+  if (on < 0) return PASTA_ERR_INVALID_ARG;
   p->profiling = on != 0;
+  p->prof_stride = on > 0 ? on : 1;
+  p->prof_seen = 0;
   p->prof_calls = 0;
   return PASTA_OK;
 }

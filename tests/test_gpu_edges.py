@@ -97,3 +97,30 @@ def test_fork_spawned_before_any_token(lib):
     ops = [("begin", 0), ("spawn", 0, 1), ("run", 0, 1, 5), ("run", 0, 0, 9),
            ("step", ((0, 1, 1), (0, 0, 1))), ("finish", 0, 1), ("merge", 0, (1,)), ("step", ((0, 0, 1),))]
     run_script(lib, manual(ops, geo))
+
+
+def test_kernel_timing_can_sample_every_kth_step(lib):
+    """pasta_profile_enable(k): every k-th attention launch group is bracketed by events, the first one included."""
+    import torch
+    geo = Geometry(1, 8, 2, 128, 16)
+    pool = lib.Pool(geo.n_layers, geo.n_q_heads, geo.n_kv_heads, geo.head_dim, 64, 1, 2, 4)
+    r = pool.request_begin()
+    g = torch.Generator(device="cuda"); g.manual_seed(5)
+    rnd = lambda *shape: torch.randn(shape, generator=g, device="cuda").to(torch.bfloat16)
+    pool.kv_append_run(r, 0, 40, rnd(1, 40, 2, 128), rnd(1, 40, 2, 128))
+    q, out = rnd(1, 1, 8, 128), torch.empty((1, 1, 8, 128), dtype=torch.float32, device="cuda")
+    for stride, steps, want in ((1, 5, 5), (3, 7, 3), (8, 8, 1)):
+        pool.profile_enable(stride)
+        for _ in range(steps):
+            pool.step_begin([r], [0], [1])
+            pool.kv_append(rnd(1, 1, 2, 128), rnd(1, 1, 2, 128))
+            pool.decode_attn(q, out)
+        ms, launches = pool.profile_read()
+        assert launches[0] == want and launches[2] == want and launches[1] == 0
+        assert ms[0] > 0 and ms[2] > 0
+    pool.profile_enable(False)
+    with pytest.raises(Exception):
+        pool.profile_enable(-1)
+    torch.cuda.synchronize()
+    assert pool.status() == 0
+    pool.close()
