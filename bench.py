@@ -294,7 +294,7 @@ def run_ours(args):
     torch.cuda.synchronize(device)
     tok0, shared0 = unique_tokens(pool, entries)
     launches0 = pool.launch_count()
-    stride = PROFILE_STRIDE if args.steps >= 8 * PROFILE_STRIDE else 1
+    stride = min(PROFILE_STRIDE, max(1, args.steps // 4))      # short runs still get at least four timed steps
     pool.profile_enable(stride)
     sampler = ClockSampler(local) if rank == 0 else None
     if world > 1:
