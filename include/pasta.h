@@ -258,6 +258,8 @@ pasta_status_t pasta_step_host(pasta_pool_t *pool, int32_t n, const int32_t *req
  *     PASTA_ERR_CAPACITY; use pasta_decode_attn for those.
  *   - The first call on a device looks up the array's device address (a runtime query, no allocation).
  *     Make that first call outside any stream capture.  The pool's device must be the current device.
+ *     The address is kept for the life of the device's primary context: after cudaDeviceReset the library
+ *     has to be reloaded before this entry point is used again.
  *   - All calls, from all pools, share the one array per GPU and each overwrites what the previous one
  *     left: two calls whose kernels may run at the same time on one GPU (different streams, different
  *     pools or processes' threads) race on it and corrupt each other's results.  Serialise them.
@@ -297,6 +299,19 @@ pasta_status_t pasta_plan_dump(pasta_pool_t *pool, int32_t *host_buf, size_t cap
 /* Synchronises `stream`, returns and clears the status word the kernels write
  * (PASTA_OK, PASTA_ERR_DEVICE_CHECK or PASTA_ERR_TIMEOUT). */
 pasta_status_t pasta_pool_status(pasta_pool_t *pool, void *stream);
+
+/*
+ * Test hooks for the bounded waits inside the kernels (no counterpart in the paper, whose only wait is the
+ * interpreter's, on the host, at <sync/>).  Every wait of one kernel role for another gives up after a number of SM
+ * clock cycles, the kernel then returns early and pasta_pool_status reports PASTA_ERR_TIMEOUT.
+ * pasta_debug_set_wait_limit sets that number for the kernels this pool launches from now on (cycles <= 0 restores
+ * the default of 3e9, about 1.5 s).  pasta_debug_wait_expiry enqueues a one-warp kernel that waits, with the pool's
+ * limit, for a barrier nobody completes: with a short limit it returns after that many cycles and leaves
+ * PASTA_ERR_TIMEOUT in the status word, which is how the tests see the limit, the report and the recovery work.
+ * With the default limit it occupies one warp for 1.5 s.  Neither touches the pool's bookkeeping or KV memory.
+ */
+pasta_status_t pasta_debug_set_wait_limit(pasta_pool_t *pool, int64_t cycles);
+pasta_status_t pasta_debug_wait_expiry(pasta_pool_t *pool, void *stream);
 
 /* Number of kernels this pool has launched so far (for launch accounting). */
 pasta_status_t pasta_launch_count(pasta_pool_t *pool, int64_t *out);

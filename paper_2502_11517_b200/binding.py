@@ -27,7 +27,7 @@ EXPORTS = [
     "pasta_profile_enable", "pasta_profile_read", "pasta_decode_attn_noalloc",
     "pasta_thread_spawn_predicted", "pasta_step_positions", "pasta_kv_append_rope", "pasta_rope_queries",
     "pasta_kv_append_run_rope", "pasta_step_device",
-    "pasta_last_cuda_error",
+    "pasta_last_cuda_error", "pasta_debug_set_wait_limit", "pasta_debug_wait_expiry",
 ]
 
 
@@ -320,6 +320,12 @@ class Pool:
         cnt = (C.c_int64 * 3)()
         _check(lib().pasta_profile_read(self._h, ms, cnt), "pasta_profile_read")
         return list(ms), list(cnt)
+
+    def debug_set_wait_limit(self, cycles: int) -> None:
+        _check(lib().pasta_debug_set_wait_limit(self._h, C.c_int64(cycles)), "pasta_debug_set_wait_limit")
+
+    def debug_wait_expiry(self, stream=None) -> None:
+        _check(lib().pasta_debug_wait_expiry(self._h, _stream(stream)), "pasta_debug_wait_expiry")
 
     def launch_count(self) -> int:
         out = C.c_int64()

@@ -233,6 +233,7 @@ pasta_status_t pasta_pool_create(const pasta_pool_config_t *cfg, pasta_pool_t **
     p->pv.part_ml = reinterpret_cast<float2 *>(ws + d.off_ml);
     p->pv.part_o = reinterpret_cast<float *>(ws + d.off_o);
     p->pv.rows_per_layer = d.max_rows;
+    p->pv.wait_limit = kWaitLimitCycles;
   }
   *out = p;
   return PASTA_OK;
@@ -646,6 +647,21 @@ pasta_status_t pasta_profile_read(pasta_pool_t *p, double *out_ms, int64_t *out_
     }
   }
   p->prof_calls = 0;
+  return PASTA_OK;
+}
+
+pasta_status_t pasta_debug_set_wait_limit(pasta_pool_t *p, int64_t cycles) {
+  if (!p) return PASTA_ERR_INVALID_ARG;
+  if (p->host_only) return PASTA_ERR_BAD_STATE;
+  p->pv.wait_limit = cycles > 0 ? static_cast<long long>(cycles) : kWaitLimitCycles;
+  return PASTA_OK;
+}
+
+pasta_status_t pasta_debug_wait_expiry(pasta_pool_t *p, void *stream) {
+  if (!p) return PASTA_ERR_INVALID_ARG;
+  if (p->host_only) return PASTA_ERR_BAD_STATE;
+  PASTA_CUDA(launch_wait_expiry(p->pv, static_cast<cudaStream_t>(stream)));
+  p->launches += 1;
   return PASTA_OK;
 }
 

@@ -44,7 +44,9 @@ constexpr int OFF_BAR = OFF_STAGE + T_STAGES * T_STAGE_BYTES;
 constexpr int B_FULL = 0, B_EMPTY = B_FULL + T_STAGES, B_SFULL = B_EMPTY + T_STAGES, B_PFULL = B_SFULL + 2,
               B_QFULL = B_PFULL + 4,   // PFULL[2 * b + group]
               B_QFREE = B_QFULL + 1, B_OFULL = B_QFREE + 1,
-              B_OFREE = B_OFULL + 1, B_MLFULL = B_OFREE + 1, B_COUNT = B_MLFULL + 1;
+              B_OFREE = B_OFULL + 1, B_MLFULL = B_OFREE + 1,
+              B_DRAIN = B_MLFULL + 1,  // only used when a role gave up: completion of the MMAs still in flight
+              B_COUNT = B_DRAIN + 1;
 constexpr int OFF_META = OFF_BAR + 8 * ((B_COUNT + 1) & ~1);   // per stage: 8 page metas
 constexpr int OFF_MISC = OFF_META + T_STAGES * 32;             // tmem base, abort flag
 constexpr int OFF_ML1 = OFF_MISC + 16;                         // (m_ref, l) of group 1's rows, for the epilogue
@@ -181,8 +183,8 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   return r;
 }
 
-// Bounded wait that also gives up when another role of the CTA has already given up.
-__device__ __forceinline__ bool wait_or_abort(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
+// Bounded wait of one role for another that also gives up when some role of the CTA has already given up.
+__device__ __forceinline__ bool wait_or_abort(uint32_t bar, uint32_t parity, volatile int *abort_flag, long long limit) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   for (;;) {
@@ -190,8 +192,13 @@ __device__ __forceinline__ bool wait_or_abort(uint32_t bar, uint32_t parity, vol
     for (int i = 0; i < 128; ++i)
       if (mbar_try_wait(bar, parity)) return true;
     if (*abort_flag) return false;
-    if (clock64() - t0 > kWaitLimitCycles) { *abort_flag = 1; return false; }
+    if (clock64() - t0 > limit) { *abort_flag = 1; return false; }
   }
+}
+// The same for a whole warp whose lanes go on to warp-wide instructions (tcgen05.ld / st, votes, __syncwarp): the
+// lanes poll on their own, so the warp takes the decision as one.
+__device__ __forceinline__ bool warp_wait_or_abort(uint32_t bar, uint32_t parity, volatile int *abort_flag, long long limit) {
+  return __all_sync(0xffffffffu, wait_or_abort(bar, parity, abort_flag, limit));
 }
 
 // bulk copy whose lines are the first to leave L2: every page is read once per launch
@@ -254,6 +261,7 @@ attn_tensor_kernel(PoolView pv, TensorArgs a, const __nv_bfloat16 *__restrict__ 
     mbar_init(bar + 8 * B_OFULL, 1);
     mbar_init(bar + 8 * B_OFREE, 4);
     mbar_init(bar + 8 * B_MLFULL, 4);
+    mbar_init(bar + 8 * B_DRAIN, 1);
     misc[1] = 0;
     mbar_init_fence();
   }
@@ -267,6 +275,8 @@ attn_tensor_kernel(PoolView pv, TensorArgs a, const __nv_bfloat16 *__restrict__ 
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = misc[0];
+  const long long limit = pv.wait_limit;
+  uint32_t prod_it = 0;       // warp 0: tiles whose copies have been issued
 
   if (warp == 0) {
     // ================================================================ producer
@@ -280,7 +290,7 @@ attn_tensor_kernel(PoolView pv, TensorArgs a, const __nv_bfloat16 *__restrict__ 
         const UnitInfo x = load_unit(plan, a.off_tunit, a.off_treq, u);
         for (int tile = x.tile_begin; tile < x.tile_end; ++tile, ++it) {
           const int s = it % T_STAGES;
-          if (!wait_or_abort(bar + 8 * (B_EMPTY + s), ((it / T_STAGES) & 1) ^ 1, abort_flag)) { ok = false; break; }
+          if (!warp_wait_or_abort(bar + 8 * (B_EMPTY + s), ((it / T_STAGES) & 1) ^ 1, abort_flag, limit)) { ok = false; break; }
           const int n_valid = min(PASTA_TILE_PAGES, x.n_pages - tile * PASTA_TILE_PAGES);
           int page = 0;
           if (lane < PASTA_TILE_PAGES) {
@@ -307,11 +317,7 @@ attn_tensor_kernel(PoolView pv, TensorArgs a, const __nv_bfloat16 *__restrict__ 
         }
       }
     }
-    if (!ok && lane == 0) {
-      // copies still in flight must land before the CTA leaves: bounded waits on the last stages issued
-      for (uint32_t j = (it > T_STAGES ? it - T_STAGES : 0); j < it; ++j)
-        mbar_wait_bounded(bar + 8 * (B_FULL + j % T_STAGES), (j / T_STAGES) & 1);
-    }
+    prod_it = it;
   } else if (warp == 1) {
     // ================================================================ MMA issue (one thread)
     if (lane == 0) {
@@ -323,13 +329,13 @@ attn_tensor_kernel(PoolView pv, TensorArgs a, const __nv_bfloat16 *__restrict__ 
           const UnitInfo x = load_unit(plan, a.off_tunit, a.off_treq, u);
           const int nt = x.tile_end - x.tile_begin;
           const uint32_t m_bits = x.n_threads * G <= T_M64_ROWS ? IDESC_M64 : IDESC_M128;
-          if (!wait_or_abort(bar + 8 * B_QFULL, uc & 1, abort_flag)) { ok = false; break; }
+          if (!wait_or_abort(bar + 8 * B_QFULL, uc & 1, abort_flag, limit)) { ok = false; break; }
           tc_fence_after();
           for (int k = 0; k <= nt && ok; ++k) {
             if (k < nt) {
               // ---- S[b] = Q . K^T for tile `it` (S[b] was last used by tile it - 2, whose P.V was issued before this)
               const uint32_t s = it % T_STAGES, b = it & 1;
-              if (!wait_or_abort(bar + 8 * (B_FULL + s), (it / T_STAGES) & 1, abort_flag)) { ok = false; break; }
+              if (!wait_or_abort(bar + 8 * (B_FULL + s), (it / T_STAGES) & 1, abort_flag, limit)) { ok = false; break; }
               tc_fence_after();
               const uint32_t k_addr = base + OFF_STAGE + s * T_STAGE_BYTES;
 #pragma unroll
@@ -346,11 +352,11 @@ attn_tensor_kernel(PoolView pv, TensorArgs a, const __nv_bfloat16 *__restrict__ 
               const uint32_t j = it - 1;
               const uint32_t s = j % T_STAGES, b = j & 1;
               if (k == 1 && uc > 0) {   // the unit's first P.V overwrites the accumulators: the previous unit's rows must be read out
-                if (!wait_or_abort(bar + 8 * B_OFREE, (uc - 1) & 1, abort_flag)) { ok = false; break; }
+                if (!wait_or_abort(bar + 8 * B_OFREE, (uc - 1) & 1, abort_flag, limit)) { ok = false; break; }
               }
               const uint32_t v_addr = base + OFF_STAGE + s * T_STAGE_BYTES + 2048;
               for (uint32_t g2 = 0; g2 < 2 && ok; ++g2) {
-                if (!wait_or_abort(bar + 8 * (B_PFULL + 2 * b + g2), (j >> 1) & 1, abort_flag)) { ok = false; break; }
+                if (!wait_or_abort(bar + 8 * (B_PFULL + 2 * b + g2), (j >> 1) & 1, abort_flag, limit)) { ok = false; break; }
                 tc_fence_after();
 #pragma unroll
                 for (int pg = 0; pg < T_HALF_PAGES; ++pg)
@@ -375,7 +381,7 @@ attn_tensor_kernel(PoolView pv, TensorArgs a, const __nv_bfloat16 *__restrict__ 
     for (int ll = 0; ll < a.layer_count && ok; ++ll) {
       for (int u = u0; u < u1; ++u, ++uc) {
         const UnitInfo x = load_unit(plan, a.off_tunit, a.off_treq, u);
-        if (uc > 0 && !wait_or_abort(bar + 8 * B_QFREE, (uc - 1) & 1, abort_flag)) { ok = false; break; }
+        if (uc > 0 && !warp_wait_or_abort(bar + 8 * B_QFREE, (uc - 1) & 1, abort_flag, limit)) { ok = false; break; }
         const int rows = x.n_threads * G;
         // thread t64 builds rows 2 t64 and 2 t64 + 1; the 16 loads of a row are issued together before any store
 #pragma unroll 1
@@ -437,7 +443,7 @@ attn_tensor_kernel(PoolView pv, TensorArgs a, const __nv_bfloat16 *__restrict__ 
           const uint32_t s = it % T_STAGES, b = it & 1;
           const uint32_t col_s = COL_S + b * T_TILE + grp * T_HALF;
           // the tile's page metas are in shared memory once its copies have landed: fetch the row's thresholds early
-          if (!wait_or_abort(bar + 8 * (B_FULL + s), (it / T_STAGES) & 1, abort_flag)) { ok = false; break; }
+          if (!warp_wait_or_abort(bar + 8 * (B_FULL + s), (it / T_STAGES) & 1, abort_flag, limit)) { ok = false; break; }
           int thr[T_HALF_PAGES];
           bool full = true;
           const int4 m4 = *reinterpret_cast<const int4 *>(meta_s + s * PASTA_TILE_PAGES + grp * T_HALF_PAGES);
@@ -476,7 +482,7 @@ attn_tensor_kernel(PoolView pv, TensorArgs a, const __nv_bfloat16 *__restrict__ 
               }
             }
           }
-          if (!wait_or_abort(bar + 8 * (B_SFULL + b), (it >> 1) & 1, abort_flag)) { ok = false; break; }
+          if (!warp_wait_or_abort(bar + 8 * (B_SFULL + b), (it >> 1) & 1, abort_flag, limit)) { ok = false; break; }
           tc_fence_after();
           if (warp_active) {
             float sc[T_HALF];
@@ -499,7 +505,7 @@ attn_tensor_kernel(PoolView pv, TensorArgs a, const __nv_bfloat16 *__restrict__ 
             if (__any_sync(0xffffffffu, rescale)) {
               // O_g and l are relative to m_ref: move them to the new reference.  The accumulator is quiet once the
               // P.V of the previous tile has finished, which is what releases that tile's stage.
-              if (!wait_or_abort(bar + 8 * (B_EMPTY + (it - 1) % T_STAGES), ((it - 1) / T_STAGES) & 1, abort_flag)) { ok = false; break; }
+              if (!warp_wait_or_abort(bar + 8 * (B_EMPTY + (it - 1) % T_STAGES), ((it - 1) / T_STAGES) & 1, abort_flag, limit)) { ok = false; break; }
               tc_fence_after();
               const float f = rescale ? fast_exp2(m_ref - mt) : 1.f;
 #pragma unroll 1
@@ -523,10 +529,13 @@ attn_tensor_kernel(PoolView pv, TensorArgs a, const __nv_bfloat16 *__restrict__ 
               fma2(x0, x1, sc[j], sc[j + 1], a.scale_log2, -ref);
               fma2(x2, x3, sc[j + 2], sc[j + 3], a.scale_log2, -ref);
               const float p0 = fast_exp2(x0), p1 = fast_exp2(x1), p2 = fast_exp2(x2), p3 = fast_exp2(x3);
-              add2(ls[0], ls[1], p0, p1);
-              add2(ls[2], ls[3], p2, p3);
-              pk[j >> 1] = pack_bf16(p0, p1);
-              pk[(j >> 1) + 1] = pack_bf16(p2, p3);
+              const uint32_t w0 = pack_bf16(p0, p1), w1 = pack_bf16(p2, p3);
+              // l sums the weights as the MMA will read them (rounded to bf16), so that O / l stays a convex
+              // combination of V rows: with one dominant key the result is that key's V row whatever m_ref is
+              add2(ls[0], ls[1], bf16_lo(w0), bf16_hi(w0));
+              add2(ls[2], ls[3], bf16_lo(w1), bf16_hi(w1));
+              pk[j >> 1] = w0;
+              pk[(j >> 1) + 1] = w1;
             }
             l += (ls[0] + ls[1]) + (ls[2] + ls[3]);
             tmem_st32_u32(tmem + lane_addr + col_s, pk);      // P takes the place of the first 32 score columns
@@ -538,7 +547,7 @@ attn_tensor_kernel(PoolView pv, TensorArgs a, const __nv_bfloat16 *__restrict__ 
         }
         if (!ok) break;
         // ---- epilogue: the unit's rows leave TMEM; group 0 folds group 1's accumulator into its own
-        if (!wait_or_abort(bar + 8 * B_OFULL, uc & 1, abort_flag)) { ok = false; break; }
+        if (!warp_wait_or_abort(bar + 8 * B_OFULL, uc & 1, abort_flag, limit)) { ok = false; break; }
         tc_fence_after();
         if (grp == 1) {
           if (active) ml1[row] = make_float2(m_ref, l);
@@ -546,7 +555,7 @@ attn_tensor_kernel(PoolView pv, TensorArgs a, const __nv_bfloat16 *__restrict__ 
           if (lane == 0) mbar_arrive(bar + 8 * B_MLFULL);
           continue;
         }
-        if (!wait_or_abort(bar + 8 * B_MLFULL, uc & 1, abort_flag)) { ok = false; break; }
+        if (!warp_wait_or_abort(bar + 8 * B_MLFULL, uc & 1, abort_flag, limit)) { ok = false; break; }
         if (warp_active) {
           const float2 other = active ? ml1[row] : make_float2(-INFINITY, 0.f);
           const float m_all = fmaxf(m_ref, other.x);
@@ -584,9 +593,25 @@ attn_tensor_kernel(PoolView pv, TensorArgs a, const __nv_bfloat16 *__restrict__ 
   }
 
   // ---- tear-down
-  if (*abort_flag && tid == 0) report(pv.status, PASTA_ERR_TIMEOUT);
   tc_fence_before();
   __syncthreads();
+  if (*abort_flag) {
+    // Some role gave up, so the others left in the middle of their work.  What the hardware still has in flight for
+    // this CTA has to finish before its shared memory and TMEM are given back: the bulk copies of the last tiles
+    // issued (their barriers complete whether or not anybody consumes the tiles) and the MMAs issued last (a commit
+    // to a barrier of its own arrives once every earlier MMA of this thread has completed).  Both end on their own.
+    if (warp == 0 && lane == 0) {
+      for (uint32_t j = (prod_it > T_STAGES ? prod_it - T_STAGES : 0); j < prod_it; ++j)
+        mbar_wait_bounded(bar + 8 * (B_FULL + j % T_STAGES), (j / T_STAGES) & 1);
+    }
+    if (warp == 1 && lane == 0) {
+      mma_commit(bar + 8 * B_DRAIN);
+      mbar_wait_bounded(bar + 8 * B_DRAIN, 0);
+    }
+    if (tid == 0) report(pv.status, PASTA_ERR_TIMEOUT);
+    tc_fence_before();
+    __syncthreads();
+  }
   if (warp == 2) {
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(TMEM_COLS) : "memory");
   }

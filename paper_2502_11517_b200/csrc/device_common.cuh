@@ -39,6 +39,7 @@ struct PoolView {
   float2 *part_ml;           // partial (m, l) per row; m in log2 units of the scaled score
   float *part_o;             // partial unnormalised outputs [row][D]
   int64_t rows_per_layer;    // stride of the partial arrays between layers of one launch
+  long long wait_limit;      // SM cycles a role waits for another role before it gives up (kWaitLimitCycles by default)
 };
 
 __device__ __forceinline__ void report(int32_t *status, int32_t code) { atomicMax(status, code); }
@@ -74,19 +75,22 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-// Upper bound of every wait inside a kernel, in SM clock cycles (about 1.5 s at 2 GHz).
+// Default upper bound of every wait inside a kernel, in SM clock cycles (about 1.5 s at 2 GHz).  Waits of one role
+// for another take the pool's limit (PoolView::wait_limit, this value unless a test shortened it); waits for the
+// hardware to finish what the CTA itself started (bulk copies, MMAs in flight when a role gives up) always take
+// this constant: they end on their own.
 constexpr long long kWaitLimitCycles = 3000000000ll;
 
-// Waits for the phase with the given parity to complete, for at most kWaitLimitCycles.
+// Waits for the phase with the given parity to complete, for at most `limit` cycles.
 // Returns false when the wait was given up (the caller then reports PASTA_ERR_TIMEOUT and leaves).
-__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, long long limit = kWaitLimitCycles) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   for (;;) {
 #pragma unroll 1
     for (int i = 0; i < 256; ++i)
       if (mbar_try_wait(bar, parity)) return true;
-    if (clock64() - t0 > kWaitLimitCycles) return false;
+    if (clock64() - t0 > limit) return false;
   }
 }
 

@@ -160,6 +160,27 @@ __global__ void rope_queries_kernel(const int32_t *__restrict__ pos, int32_t n, 
   }
 }
 
+// =============================================================================================
+// Test kernel for the bounded waits: one warp waits, with the pool's limit, for an mbarrier phase that nobody
+// completes, reports PASTA_ERR_TIMEOUT when the wait gives up (it always does) and returns.
+// =============================================================================================
+__global__ void wait_expiry_kernel(PoolView pv) {
+  __shared__ __align__(8) uint64_t bar_mem;
+  const uint32_t bar = smem_u32(&bar_mem);
+  if (threadIdx.x == 0) {
+    mbar_init(bar, 1);
+    mbar_init_fence();
+  }
+  __syncwarp();
+  const bool done = __all_sync(0xffffffffu, mbar_wait_bounded(bar, 0, pv.wait_limit));
+  if (!done && threadIdx.x == 0) report(pv.status, PASTA_ERR_TIMEOUT);
+}
+
+cudaError_t launch_wait_expiry(const PoolView &pv, cudaStream_t st) {
+  wait_expiry_kernel<<<1, 32, 0, st>>>(pv);
+  return cudaGetLastError();
+}
+
 cudaError_t launch_kv_append_rope(const PoolView &pv, const int32_t *slots, const int32_t *pos, int32_t pos0, int32_t n_tok,
                                   int32_t layer_begin, int32_t layer_count, const void *k_new, const void *v_new,
                                   double theta, cudaStream_t st) {
@@ -302,7 +323,8 @@ attn_warp_kernel(PoolView pv, int32_t off_wunit, int32_t off_pages, int32_t n_wu
 
   for (int i = 0; i < n_pg; ++i) {
     const int s = i % W_STAGES;
-    if (!mbar_wait_bounded(bar0 + 8 * s, (i / W_STAGES) & 1)) { ok = false; consumed = i; break; }
+    // the lanes poll on their own: the warp gives up as one, or the shuffles below would meet half a warp
+    if (!__all_sync(0xffffffffu, mbar_wait_bounded(bar0 + 8 * s, (i / W_STAGES) & 1, pv.wait_limit))) { ok = false; consumed = i; break; }
     const uint8_t *sp = stages + s * S::BLOCK;
     const int nv = min(PASTA_PAGE, n_tok - i * PASTA_PAGE);
 

@@ -45,6 +45,8 @@ cudaError_t launch_attn_warp(const PoolView &pv, const PlanHeader &h, int32_t la
 cudaError_t launch_attn_tensor(const PoolView &pv, const PlanHeader &h, int32_t layer_begin, int32_t layer_count,
                                const void *q, float scale_log2, cudaStream_t st);
 bool tensor_path_available();       // false while the tensor-core kernel is compiled out
+// test kernel: a bounded wait that runs out (one warp, PoolView::wait_limit cycles), reported as PASTA_ERR_TIMEOUT
+cudaError_t launch_wait_expiry(const PoolView &pv, cudaStream_t st);
 // K4: log-sum-exp merge of all partial rows of every (query, head)
 // out: device fp32 [layer_count, n, Hq, D], or bf16 of the same shape when out_bf16
 cudaError_t launch_merge(const PoolView &pv, const PlanHeader &h, int32_t layer_count, void *out, float *lse,
