@@ -311,6 +311,14 @@ pasta_status_t pasta_pool_status(pasta_pool_t *pool, void *stream);
  * With the default limit it occupies one warp for 1.5 s.  Neither touches the pool's bookkeeping or KV memory.
  */
 pasta_status_t pasta_debug_set_wait_limit(pasta_pool_t *pool, int64_t cycles);
+/*
+ * Makes the wait of a role of the tensor-core attention kernel run out for real: the roles whose bit is set in
+ * role_mask (1 page producer, 2 MMA issue, 4 query-operand builder, 8 / 16 the two softmax groups) do not start in
+ * the launches that follow, the roles that wait for them give up after the pool's wait limit, every CTA drains what
+ * it has in flight, frees its tensor memory and returns, and the status word holds PASTA_ERR_TIMEOUT.  The outputs
+ * of such a launch are undefined.  Set a short limit first (pasta_debug_set_wait_limit); 0 switches the hook off.
+ */
+pasta_status_t pasta_debug_hold_roles(pasta_pool_t *pool, int32_t role_mask);
 pasta_status_t pasta_debug_wait_expiry(pasta_pool_t *pool, void *stream);
 
 /* Number of kernels this pool has launched so far (for launch accounting). */

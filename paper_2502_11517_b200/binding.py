@@ -27,7 +27,7 @@ EXPORTS = [
     "pasta_profile_enable", "pasta_profile_read", "pasta_decode_attn_noalloc",
     "pasta_thread_spawn_predicted", "pasta_step_positions", "pasta_kv_append_rope", "pasta_rope_queries",
     "pasta_kv_append_run_rope", "pasta_step_device",
-    "pasta_last_cuda_error", "pasta_debug_set_wait_limit", "pasta_debug_wait_expiry",
+    "pasta_last_cuda_error", "pasta_debug_set_wait_limit", "pasta_debug_wait_expiry", "pasta_debug_hold_roles",
 ]
 
 
@@ -323,6 +323,9 @@ class Pool:
 
     def debug_set_wait_limit(self, cycles: int) -> None:
         _check(lib().pasta_debug_set_wait_limit(self._h, C.c_int64(cycles)), "pasta_debug_set_wait_limit")
+
+    def debug_hold_roles(self, role_mask: int) -> None:
+        _check(lib().pasta_debug_hold_roles(self._h, role_mask), "pasta_debug_hold_roles")
 
     def debug_wait_expiry(self, stream=None) -> None:
         _check(lib().pasta_debug_wait_expiry(self._h, _stream(stream)), "pasta_debug_wait_expiry")

@@ -234,6 +234,7 @@ pasta_status_t pasta_pool_create(const pasta_pool_config_t *cfg, pasta_pool_t **
     p->pv.part_o = reinterpret_cast<float *>(ws + d.off_o);
     p->pv.rows_per_layer = d.max_rows;
     p->pv.wait_limit = kWaitLimitCycles;
+    p->pv.debug_hold = 0;
   }
   *out = p;
   return PASTA_OK;
@@ -654,6 +655,13 @@ pasta_status_t pasta_debug_set_wait_limit(pasta_pool_t *p, int64_t cycles) {
   if (!p) return PASTA_ERR_INVALID_ARG;
   if (p->host_only) return PASTA_ERR_BAD_STATE;
   p->pv.wait_limit = cycles > 0 ? static_cast<long long>(cycles) : kWaitLimitCycles;
+  return PASTA_OK;
+}
+
+pasta_status_t pasta_debug_hold_roles(pasta_pool_t *p, int32_t role_mask) {
+  if (!p || role_mask < 0 || role_mask > 31) return PASTA_ERR_INVALID_ARG;
+  if (p->host_only) return PASTA_ERR_BAD_STATE;
+  p->pv.debug_hold = role_mask;
   return PASTA_OK;
 }
 

@@ -278,7 +278,10 @@ attn_tensor_kernel(PoolView pv, TensorArgs a, const __nv_bfloat16 *__restrict__ 
   const long long limit = pv.wait_limit;
   uint32_t prod_it = 0;       // warp 0: tiles whose copies have been issued
 
-  if (warp == 0) {
+  // test hook: a held role goes straight to the tear-down, so that the roles waiting for it run into their limits
+  const int role = warp == 0 ? 0 : warp == 1 ? 1 : warp < 4 ? 2 : 3 + ((warp - 4) >> 2);
+  if ((pv.debug_hold >> role) & 1) {
+  } else if (warp == 0) {
     // ================================================================ producer
     uint32_t it = 0;
     bool ok = true;

@@ -40,6 +40,7 @@ struct PoolView {
   float *part_o;             // partial unnormalised outputs [row][D]
   int64_t rows_per_layer;    // stride of the partial arrays between layers of one launch
   long long wait_limit;      // SM cycles a role waits for another role before it gives up (kWaitLimitCycles by default)
+  int32_t debug_hold;        // test hook, 0 in normal use: bit r set = role r of the tensor-core kernel never starts
 };
 
 __device__ __forceinline__ void report(int32_t *status, int32_t code) { atomicMax(status, code); }
