@@ -38,12 +38,22 @@ UNIT = "thread-tokens/s"
 NOMINAL_HBM_GBS = 8000.0
 SEED_EXTRAS = 2502115
 FALLBACK_HBM_GBS = 6650.0
-# dram bytes (read + write) of one launch of the dominant kernel from an ncu capture of this workload,
-# or None when no capture matches the current kernel
-# Per-kernel events inside the timed region: a timing event between two kernels delays the second by a few microseconds
-# (10 % of a 0.2 ms step with all four events on every step), so only every eighth step carries them.
-PROFILE_STRIDE = 8
-NCU_TRAFFIC_BYTES = {("long_shared_prefix", "full"): 1.2111e9, ("long_shared_prefix", "small"): 3.945e8}   # see profiles/
+# The per-kernel events are kept out of the timed region (a timing event between two kernels holds the second back
+# by a few microseconds): the kernels are timed in a loop of their own right after it, every launch, at least this many.
+PROFILE_STEPS = 24
+# DRAM bytes (read + write) of one launch of the tensor-core kernel from the ncu captures summarised under profiles/,
+# as a ratio to the launch's algorithmic bytes (reads grow with the bytes read; the partial-row writes are added as
+# they are).  Valid for the kernel source it was captured from only: its hash is checked at run time.
+NCU_TRAFFIC = {"attn_tensor_sha256_16": None, "read_ratio": 1.0135, "write_bytes": 3.9e6}
+
+
+def kernel_source_hash() -> str:
+    import hashlib
+    h = hashlib.sha256()
+    for name in ("attn_tensor.cu", "device_common.cuh", "pasta_plan.h"):
+        with open(os.path.join(ROOT, "paper_2502_11517_b200", "csrc", name), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()[:16]
 
 
 def make_script(workload: str, size: str = "full"):
@@ -72,60 +82,109 @@ def measured_peak():
 
 # ------------------------------------------------------------------------------------------------ clocks
 class ClockSampler:
+    """SM clock, power and throttle reasons of one GPU while a region runs: read through NVML from a thread of this
+    process every millisecond or so (reading only; no setting is touched), or, without the NVML module, from an
+    `nvidia-smi` child that samples every 20 ms."""
+    REASONS = {0x4: "sw_power_cap", 0x8: "hw_slowdown", 0x20: "sw_thermal_slowdown", 0x40: "hw_thermal_slowdown",
+               0x80: "hw_power_brake_slowdown"}
     QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
              "clocks_event_reasons.sw_power_cap")
 
     def __init__(self, device_index: int):
-        self.file = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
-        self.proc = None
+        import threading
+        self.rows = []          # (wall time, sm MHz, reasons bit mask, watts)
+        self.now = lambda: None  # one reading taken by the caller's thread (NVML only)
+        self.sm_max = None
+        self.proc = self.file = self.thread = None
+        self._stop = threading.Event()
         try:
-            self.proc = subprocess.Popen(
-                ["nvidia-smi", "-i", str(device_index), f"--query-gpu=timestamp,{self.QUERY}",
-                 "--format=csv,noheader,nounits", "-lms", "20"], stdout=self.file, stderr=subprocess.DEVNULL)
-        except Exception:
-            self.proc = None
+            import pynvml
+            pynvml.nvmlInit()
+            visible = os.environ.get("CUDA_VISIBLE_DEVICES")
+            index = int(visible.split(",")[device_index]) if visible and visible.split(",")[device_index].isdigit() else device_index
+            handle = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.sm_max = float(pynvml.nvmlDeviceGetMaxClockInfo(handle, pynvml.NVML_CLOCK_SM))
+            reasons = getattr(pynvml, "nvmlDeviceGetCurrentClocksEventReasons", None) or pynvml.nvmlDeviceGetCurrentClocksThrottleReasons
 
-    def stop(self, t0: float, t1: float):
-        """Samples whose wall-clock time lies in [t0, t1] (the timed region); falls back to all samples."""
-        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
-        if self.proc is None:
-            return out
-        time.sleep(0.05)
-        self.proc.terminate()
-        try:
-            self.proc.wait(timeout=5)
+            def loop():
+                while not self._stop.is_set():
+                    try:
+                        self.rows.append((time.time(), float(pynvml.nvmlDeviceGetClockInfo(handle, pynvml.NVML_CLOCK_SM)),
+                                          int(reasons(handle)), pynvml.nvmlDeviceGetPowerUsage(handle) / 1000.0))
+                    except Exception:
+                        pass
+                    time.sleep(0.001)
+
+            def now():
+                self.rows.append((time.time(), float(pynvml.nvmlDeviceGetClockInfo(handle, pynvml.NVML_CLOCK_SM)),
+                                  int(reasons(handle)), pynvml.nvmlDeviceGetPowerUsage(handle) / 1000.0))
+
+            self.now = now
+            self.thread = threading.Thread(target=loop, daemon=True)
+            self.thread.start()
+            self.how = "nvml: a thread about 1 ms apart, plus one reading as the region's last kernel ends"
         except Exception:
-            self.proc.kill()
-        self.file.flush()
-        rows = []
-        import datetime
-        for line in open(self.file.name):
-            parts = [p.strip() for p in line.split(",")]
-            if len(parts) < 9:
-                continue
+            self.how = "nvidia-smi, 20 ms apart"
+            self.file = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
             try:
-                ts = datetime.datetime.strptime(parts[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
-                rows.append((ts, float(parts[1]), float(parts[2]), parts[4:9]))
+                self.proc = subprocess.Popen(
+                    ["nvidia-smi", "-i", str(device_index), f"--query-gpu=timestamp,{self.QUERY}",
+                     "--format=csv,noheader,nounits", "-lms", "20"], stdout=self.file, stderr=subprocess.DEVNULL)
             except Exception:
-                continue
-        os.unlink(self.file.name)
+                self.proc = None
+
+    def _finish(self):
+        if self.thread is not None:
+            self._stop.set()
+            self.thread.join(timeout=2)
+            self.thread = None
+        if self.proc is not None:
+            import datetime
+            time.sleep(0.05)
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except Exception:
+                self.proc.kill()
+            self.proc = None
+            self.file.flush()
+            bits = {v: k for k, v in self.REASONS.items()}
+            names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+            for line in open(self.file.name):
+                parts = [p.strip() for p in line.split(",")]
+                if len(parts) < 9:
+                    continue
+                try:
+                    ts = datetime.datetime.strptime(parts[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+                    mask = sum(bits[n] for n, flag in zip(names, parts[5:9]) if flag.lower().startswith("active"))
+                    self.rows.append((ts, float(parts[1]), mask, float(parts[3])))
+                    self.sm_max = max(self.sm_max or 0.0, float(parts[2]))
+                except Exception:
+                    continue
+            os.unlink(self.file.name)
+
+    def window(self, t0: float, t1: float):
+        """Summary of the samples taken in [t0, t1] (wall clock); all samples so far when none fell inside."""
+        out = {"sm_mhz": None, "sm_max_mhz": self.sm_max, "reasons": [], "samples": 0, "how": self.how}
+        rows = list(self.rows)
         inside = [r for r in rows if t0 <= r[0] <= t1]
-        out["window"] = "timed region" if inside else "whole run (timed region shorter than the sampling period)"
+        out["window"] = "timed region" if inside else "whole run (no sample fell inside the timed region)"
         use = inside or rows
         if not use:
             return out
         out["samples"] = len(use)
         out["sm_mhz"] = float(np.median([r[1] for r in use]))
-        out["sm_max_mhz"] = float(max(r[2] for r in use))
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        out["power_w"] = float(np.median([r[3] for r in use]))
         seen = set()
         for r in use:
-            for name, flag in zip(names, r[3][1:]):
-                if flag.lower().startswith("active"):
-                    seen.add(name)
+            seen.update(name for bit, name in self.REASONS.items() if r[2] & bit)
         out["reasons"] = sorted(seen)
         return out
+
+    def stop(self, t0: float, t1: float):
+        self._finish()
+        return self.window(t0, t1)
 
 
 # ------------------------------------------------------------------------------------------------ our arm
@@ -222,7 +281,7 @@ def build_state_naive_rows(script, device, seed_offset=0, grow_tokens=640):
     return pool, row_entries, randn, rows.bytes_copied_at_spawn
 
 
-def unique_tokens(pool, entries):
+def unique_tokens(pool, entries, tensor=True):
     """Per request, the union of what the step's threads see (a shared prefix counts once); and the part of
     it that the tensor-core kernel reads: everything, for requests whose stacked query rows fit one MMA tile."""
     dump = pool.dump()
@@ -238,13 +297,181 @@ def unique_tokens(pool, entries):
                 vis[s] = max(vis.get(s, 0), a + n)
             for s, v in vis.items():
                 seen.setdefault(s, []).append(v)
-        on_tensor = (pool.head_dim == 128 and len(threads) * (pool.n_q_heads // pool.n_kv_heads) <= 128
+        on_tensor = (tensor and pool.head_dim == 128 and len(threads) * (pool.n_q_heads // pool.n_kv_heads) <= 128
                      and len(seen) <= 255)
         for s, vs in seen.items():
             total += max(vs)
             if on_tensor:
                 shared += max(vs)
     return total, shared
+
+
+def measure_steady(args, workload, size, steps, warmup, device, rank, world, local, *, layout="pool",
+                   out_dtype_name="fp32", with_e2e=True, flags=0):
+    """One workload whose step repeats (every entry appends a token and attends): builds the state, times `steps`
+    steps after `warmup`, then times the kernels in a loop of their own and, if asked, the host-buffer path."""
+    import torch
+    import torch.distributed as dist
+    from paper_2502_11517_b200 import binding as _b
+    from paper_2502_11517_b200.sharding import aggregate
+    script = make_script(workload, size)
+    geo = script.geometry
+    warmup = max(warmup, 3)
+    prof_steps = PROFILE_STEPS
+    e2e_steps = max(8, min(steps, 50)) if with_e2e else 0
+    grow = steps + warmup + prof_steps + 2 * e2e_steps + 16
+    spawn_copy_bytes = None
+    if layout == "naive_rows":
+        pool, entries, randn, spawn_copy_bytes = build_state_naive_rows(script, device, seed_offset=rank, grow_tokens=grow)
+    else:
+        pool, entries, randn = build_state(script, device, seed_offset=rank, grow_tokens=grow,
+                                           flags=flags | (_b.FLAG_OUT_BF16 if out_dtype_name == "bf16" else 0))
+    n = len(entries)
+    reqs = np.asarray([e[0] for e in entries], dtype=np.int32); thr = np.asarray([e[1] for e in entries], dtype=np.int32)
+    ones = np.ones(n, dtype=np.int32)
+    L = geo.n_layers
+    k_new = randn((L, n, geo.n_kv_heads, geo.head_dim)); v_new = randn((L, n, geo.n_kv_heads, geo.head_dim))
+    q = randn((L, n, geo.n_q_heads, geo.head_dim))
+    out_dtype = torch.bfloat16 if (out_dtype_name == "bf16" and layout == "pool") else torch.float32
+    out = torch.empty(q.shape, dtype=out_dtype, device=device)
+    stream = torch.cuda.current_stream(device)
+    sh = stream.cuda_stream                   # the stream's handle, looked up once
+
+    def step():                               # plan + append + attention of all layers, one library call
+        pool.step_device(reqs, thr, ones, k_new, v_new, q, out, stream=sh)
+
+    sampler = ClockSampler(local) if rank == 0 else None      # started early: its first readings take a while
+    for _ in range(warmup):
+        step()
+    torch.cuda.synchronize(device)
+    on_tensor = not (flags & _b.FLAG_NO_TENSOR_PATH)
+    tok0, _ = unique_tokens(pool, entries, on_tensor)
+    launches0 = pool.launch_count()
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize(device)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t_wall0 = time.time()
+    ev0.record(stream)
+    for _ in range(steps):
+        step()
+    ev1.record(stream)
+    torch.cuda.synchronize(device)
+    if sampler:
+        sampler.now()                         # the GPU was under load until a few microseconds ago
+    t_wall1 = time.time()
+    if world > 1:
+        dist.barrier()
+    ms = ev0.elapsed_time(ev1)
+    clocks = sampler.window(t_wall0, t_wall1) if sampler else None
+    launches = pool.launch_count() - launches0
+    tok1, shared1 = unique_tokens(pool, entries, on_tensor)
+    all_tokens, worst_s = aggregate(float(n * steps), ms * 1e-3)    # every rank runs its own requests
+    ms = worst_s * 1e3
+
+    # ---- the kernels, timed one by one (events around every launch) in the steps that follow the timed region
+    pool.profile_enable(1)
+    t_prof0 = time.time()
+    for _ in range(prof_steps):
+        step()
+    torch.cuda.synchronize(device)
+    if sampler:
+        sampler.now()
+    t_prof1 = time.time()
+    kernel_ms, kernel_launches = pool.profile_read()
+    pool.profile_enable(False)
+    prof_clocks = sampler.window(t_prof0, t_prof1) if sampler else None
+    tok2, shared2 = unique_tokens(pool, entries, on_tensor)
+    assert pool.status() == 0, "a kernel reported an error"
+
+    # ---- what a read-only kernel gets on this GPU, same run: the pool's KV memory read by bulk copies and by loads
+    ceilings = {}
+    if layout == "pool" and pool.kv.numel() > 256e6:
+        for name, mode in (("bulk_copy", 1), ("bulk_copy_scattered_8k", 2), ("vector_loads", 0)):
+            for _ in range(2):
+                nbytes = pool.debug_stream_read(None, mode, stream=sh)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            reps = 8
+            e0.record(stream)
+            for _ in range(reps):
+                pool.debug_stream_read(None, mode, stream=sh)
+            e1.record(stream)
+            torch.cuda.synchronize(device)
+            ceilings[name] = nbytes * reps / (e0.elapsed_time(e1) * 1e-3) / 1e9
+        assert pool.status() == 0
+
+    # ---- end to end: the same step through the host-buffer entry points (copies inside the timed region)
+    e2e = None
+    if with_e2e:
+        k_h = k_new.cpu().pin_memory(); v_h = v_new.cpu().pin_memory(); q_h = q.cpu().pin_memory()
+        out_h = [torch.empty(q.shape, dtype=out_dtype).pin_memory() for _ in range(2)]
+        staging = torch.empty(2 * pool.step_host_bytes(n), dtype=torch.uint8, device=device)
+        for _ in range(3):
+            pool.step_host(reqs, thr, ones, k_h, v_h, q_h, out_h[0], staging)
+        torch.cuda.synchronize(device)
+        if world > 1:
+            dist.barrier()
+        # (a) one step after the other, each waited for before the next begins
+        t0 = time.perf_counter()
+        for _ in range(e2e_steps):
+            pool.step_host(reqs, thr, ones, k_h, v_h, q_h, out_h[0], staging)
+        serial_s = time.perf_counter() - t0
+        # (b) two steps in flight: the copies of a step overlap the kernels of its neighbour
+        torch.cuda.synchronize(device)
+        t0 = time.perf_counter()
+        pool.step_host_begin(reqs, thr, ones, k_h, v_h, q_h, out_h[0], staging)
+        for i in range(1, e2e_steps):
+            pool.step_host_begin(reqs, thr, ones, k_h, v_h, q_h, out_h[i & 1], staging)
+            pool.step_host_wait()
+        pool.step_host_wait()
+        piped_s = time.perf_counter() - t0
+        torch.cuda.synchronize(device)
+        assert pool.status() == 0
+        e2e_tokens, piped_s = aggregate(float(n * e2e_steps), piped_s)
+        _, serial_s = aggregate(float(n * e2e_steps), serial_s)
+        e2e = {"value": e2e_tokens / piped_s, "unit": UNIT, "h2d_bytes_per_step": k_h.numel() * 2 * 2 + q_h.numel() * 2,
+               "d2h_bytes_per_step": out_h[0].numel() * out_h[0].element_size(), "steps": e2e_steps,
+               "how": "pasta_step_host_begin / _wait, two steps in flight, pinned host buffers",
+               "one_step_at_a_time": e2e_tokens / serial_s}
+    if sampler:
+        sampler.stop(0, 0)
+
+    B_tok = geo.kv_bytes_per_token
+    avg_tokens = (tok0 + tok1) / 2.0 + n / 2.0                 # unique KV tokens of the average timed step
+    step_bytes = avg_tokens * B_tok * L
+    timed = max(1, max(kernel_launches))
+    dom = 0 if kernel_launches[0] else 1                       # tensor-core kernel when the plan has t-units
+    prof_tokens = (tok1 + tok2) / 2.0 + n / 2.0
+    prof_shared = (shared1 + shared2) / 2.0
+    dom_bytes = (prof_shared if dom == 0 else prof_tokens - prof_shared) * B_tok * L
+    dom_ms = kernel_ms[dom] / max(1, kernel_launches[dom])
+    res = {
+        "script": script, "geo": geo, "n": n, "L": L, "requests": len(set(reqs.tolist())),
+        "value": all_tokens / (ms * 1e-3), "ms_per_step": ms / steps, "steps": steps, "warmup": warmup,
+        "launches": launches, "clocks": clocks, "avg_tokens": avg_tokens, "step_bytes": step_bytes,
+        "step_gbs": step_bytes / (ms / steps * 1e-3) / 1e9,
+        "kernel_ms_per_step": {"tensor": kernel_ms[0] / timed, "warp": kernel_ms[1] / timed, "merge": kernel_ms[2] / timed,
+                               "launches_timed": timed, "where": "every launch of the %d steps after the timed region" % prof_steps,
+                               "clocks": prof_clocks},
+        "dom": ["attn_tensor_kernel", "attn_warp_kernel"][dom], "dom_bytes": dom_bytes, "dom_ms": dom_ms,
+        "dom_gbs": dom_bytes / (dom_ms * 1e-3) / 1e9 if dom_ms > 0 else 0.0,
+        "ceilings": ceilings, "e2e": e2e, "spawn_copy_bytes": spawn_copy_bytes,
+    }
+    pool.close()
+    del pool, out, q, k_new, v_new
+    torch.cuda.empty_cache()
+    return res
+
+
+def summary_of(m, peak):
+    """The figures of a secondary workload that go under config.other_workloads."""
+    return {"workload": m["script"].name, "thread_tokens_per_step": m["n"], "layers": m["L"], "steps": m["steps"],
+            "warmup": m["warmup"], "ms_per_step": m["ms_per_step"], "thread_tokens_per_s": m["value"],
+            "unique_kv_bytes_per_step": m["step_bytes"],
+            "l2": "inputs larger than L2" if m["step_bytes"] / m["L"] > 126e6 * 1.5 else "working set fits L2 (latency case)",
+            "step_hbm_gbs": m["step_gbs"], "step_frac_of_measured_peak": m["step_gbs"] / peak,
+            "kernel": m["dom"], "kernel_gbs": m["dom_gbs"], "kernel_frac_of_measured_peak": m["dom_gbs"] / peak,
+            "kernel_ms_per_step": m["kernel_ms_per_step"], "clocks": m["clocks"], "gpu_launches": m["launches"]}
 
 
 def run_ours(args):
@@ -263,137 +490,62 @@ def run_ours(args):
         dist.barrier()
     device = torch.device("cuda", local)
     torch.cuda.set_device(device)
-    script = make_script(args.workload, args.size)
-    geo = script.geometry
-    e2e_steps = max(3, min(args.steps, 50))
-    grow = args.steps + max(args.warmup, 3) + e2e_steps + 3
-    spawn_copy_bytes = None
-    if args.layout == "naive_rows":
-        pool, entries, randn, spawn_copy_bytes = build_state_naive_rows(script, device, seed_offset=rank, grow_tokens=grow)
-    else:
-        from paper_2502_11517_b200 import binding as _b
-        pool, entries, randn = build_state(script, device, seed_offset=rank, grow_tokens=grow,
-                                           flags=_b.FLAG_OUT_BF16 if args.out_dtype == "bf16" else 0)
-    n = len(entries)
-    reqs = np.asarray([e[0] for e in entries], dtype=np.int32); thr = np.asarray([e[1] for e in entries], dtype=np.int32)
-    ones = np.ones(n, dtype=np.int32)
-    L = geo.n_layers
-    k_new = randn((L, n, geo.n_kv_heads, geo.head_dim)); v_new = randn((L, n, geo.n_kv_heads, geo.head_dim))
-    q = randn((L, n, geo.n_q_heads, geo.head_dim))
-    out_dtype = torch.bfloat16 if (args.out_dtype == "bf16" and args.layout == "pool") else torch.float32
-    out = torch.empty(q.shape, dtype=out_dtype, device=device)
-    stream = torch.cuda.current_stream(device)
-
-    sh = stream.cuda_stream                   # the stream's handle, looked up once
-
-    def step():                               # plan + append + attention of all layers, one library call
-        pool.step_device(reqs, thr, ones, k_new, v_new, q, out, stream=sh)
-
-    for _ in range(max(args.warmup, 3)):
-        step()
-    torch.cuda.synchronize(device)
-    tok0, shared0 = unique_tokens(pool, entries)
-    launches0 = pool.launch_count()
-    stride = min(PROFILE_STRIDE, max(1, args.steps // 4))      # short runs still get at least four timed steps
-    pool.profile_enable(stride)
-    sampler = ClockSampler(local) if rank == 0 else None
-    if world > 1:
-        dist.barrier()
-    torch.cuda.synchronize(device)
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    t_wall0 = time.time()
-    ev0.record(stream)
-    for _ in range(args.steps):
-        step()
-    ev1.record(stream)
-    torch.cuda.synchronize(device)
-    t_wall1 = time.time()
-    if world > 1:
-        dist.barrier()
-    ms = ev0.elapsed_time(ev1)
-    clocks = sampler.stop(t_wall0, t_wall1) if sampler else None
-    kernel_ms, kernel_launches = pool.profile_read()
-    pool.profile_enable(False)
-    launches = pool.launch_count() - launches0
-    tok1, shared1 = unique_tokens(pool, entries)
-    assert pool.status() == 0, "a kernel reported an error"
-    from paper_2502_11517_b200.sharding import aggregate
-    all_tokens, worst_s = aggregate(float(n * args.steps), ms * 1e-3)    # every rank runs its own requests
-    ms = worst_s * 1e3
-
-    # ---- end to end: the same step through the host-buffer entry point (copies inside the timed region)
-    k_h = k_new.cpu().pin_memory(); v_h = v_new.cpu().pin_memory(); q_h = q.cpu().pin_memory()
-    out_h = torch.empty(q.shape, dtype=out_dtype).pin_memory()
-    staging = torch.empty(pool.step_host_bytes(n), dtype=torch.uint8, device=device)
-    for _ in range(3):
-        pool.step_host(reqs, thr, ones, k_h, v_h, q_h, out_h, staging)
-    torch.cuda.synchronize(device)
-    if world > 1:
-        dist.barrier()
-    t0 = time.perf_counter()
-    for _ in range(e2e_steps):
-        pool.step_host(reqs, thr, ones, k_h, v_h, q_h, out_h, staging)
-    torch.cuda.synchronize(device)
-    e2e_s = time.perf_counter() - t0
-    e2e_tokens, e2e_s = aggregate(float(n * e2e_steps), e2e_s)
-    h2d = k_h.numel() * 2 * 2 + q_h.numel() * 2
-    d2h = out_h.numel() * out_h.element_size()
-
-    # ---- host-only cost of a <sync/> merge (no kernel, no copy): a scratch pool with 16 finished forks
-    merge_us = time_sync_merge()
-
+    from paper_2502_11517_b200 import binding as _b
+    flags = _b.FLAG_NO_TENSOR_PATH if args.kernel == "warp" else 0
+    m = measure_steady(args, args.workload, args.size, args.steps, args.warmup, device, rank, world, local,
+                       layout=args.layout, out_dtype_name=args.out_dtype, flags=flags)
+    merge_us = time_sync_merge()              # host-only cost of a <sync/> merge (no kernel, no copy)
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
         return
-    B_tok = geo.kv_bytes_per_token
-    # unique KV bytes of the average step (every step adds one token per entry); all layers
-    avg_tokens = (tok0 + tok1) / 2.0 + n / 2.0
-    step_bytes = avg_tokens * B_tok * L
-    shared_bytes = (shared0 + shared1) / 2.0 * B_tok * L      # what one tensor-core launch... per step
     peak, peak_kind = measured_peak()
-    timed_steps = max(1, max(kernel_launches))                 # one launch of each kernel per step
-    dom = 0 if kernel_launches[0] else 1                       # tensor-core kernel when the workload has shared streams
-    dom_name = ["attn_tensor_kernel", "attn_warp_kernel"][dom]
-    # the per-kernel events bracket every PROFILE_STRIDE-th step of the timed region, up to a bounded number of them,
-    # and every step lengthens each stream by one token: bytes of the average step of the range they cover
-    frac_timed = min(1.0, timed_steps * stride / max(1, args.steps))
-    tok_p = tok0 + (tok1 - tok0) * frac_timed
-    shared_p = shared0 + (shared1 - shared0) * frac_timed
-    prof_step_bytes = ((tok0 + tok_p) / 2.0 + n / 2.0) * B_tok * L
-    prof_shared_bytes = (shared0 + shared_p) / 2.0 * B_tok * L
-    dom_bytes_per_launch = prof_shared_bytes if dom == 0 else prof_step_bytes - prof_shared_bytes
-    dom_ms = kernel_ms[dom] / max(1, kernel_launches[dom])
-    achieved = dom_bytes_per_launch / (dom_ms * 1e-3) / 1e9 if dom_ms > 0 else 0.0
-    value = all_tokens / (ms * 1e-3)
-    step_gbs = step_bytes / (ms / args.steps * 1e-3) / 1e9
+    others = []
+    if world == 1 and args.others and args.workload == "long_shared_prefix" and args.layout == "pool" and args.kernel == "auto":
+        # the other configurations, same protocol, shorter: their figures ride along under config.other_workloads
+        for wl, size, st, wu in (("batched", "full", 12, 3), ("single_request", "full", 200, 10)):
+            try:
+                others.append(summary_of(measure_steady(args, wl, size, st, wu, device, rank, world, local, with_e2e=False), peak))
+            except Exception as exc:           # e.g. not enough free memory on a shared GPU
+                others.append({"workload": wl, "error": repr(exc)[:200]})
+        try:
+            tr = trace_measure(device, rank, world, local, size="small", steps=40, warmup=4)
+            others.append({k: tr[k] for k in ("workload", "steps", "warmup", "ms_per_step", "thread_tokens_per_s", "layers",
+                                              "requests", "step_hbm_gbs", "step_frac_of_measured_peak", "kernel_ms_per_step",
+                                              "clocks", "gpu_launches", "sync_merges_timed")})
+        except Exception as exc:
+            others.append({"workload": "trace", "error": repr(exc)[:200]})
+    geo, L = m["geo"], m["L"]
+    traffic = None
+    if m["dom"] == "attn_tensor_kernel" and args.layout == "pool" and NCU_TRAFFIC["attn_tensor_sha256_16"] == kernel_source_hash():
+        traffic = m["dom_bytes"] * NCU_TRAFFIC["read_ratio"] + NCU_TRAFFIC["write_bytes"]
     result = {
-        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-        "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps, "higher_is_better": True,
+        "metric": METRIC, "value": m["value"], "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": m["warmup"], "ms_per_step": m["ms_per_step"], "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {
             "workload": args.workload, "size": args.size, "layout": args.layout, "out_dtype": args.out_dtype,
-            "script": script.name, "requests": len(set(reqs)), "thread_tokens_per_step": n,
+            "kernel_path": args.kernel,
+            "script": m["script"].name, "requests": m["requests"], "thread_tokens_per_step": m["n"],
             "layers": L, "n_q_heads": geo.n_q_heads, "n_kv_heads": geo.n_kv_heads, "head_dim": geo.head_dim,
-            "page_size": geo.page_size, "unique_kv_tokens_per_layer": avg_tokens,
-            "unique_kv_bytes_per_step": step_bytes, "l2": "inputs larger than L2" if step_bytes / L > 126e6 * 1.5 else
-            "working set fits L2 (latency case)",
-            "step_hbm_gbs": step_gbs, "step_frac_of_measured_peak": step_gbs / peak,
-            "step_frac_of_nominal_8TBs": step_gbs / NOMINAL_HBM_GBS,
-            "kernel_ms_per_step": {"tensor": kernel_ms[0] / timed_steps, "warp": kernel_ms[1] / timed_steps,
-                                   "merge": kernel_ms[2] / timed_steps, "steps_timed": timed_steps,
-                                   "every": stride},
+            "page_size": geo.page_size, "unique_kv_tokens_per_layer": m["avg_tokens"],
+            "unique_kv_bytes_per_step": m["step_bytes"],
+            "l2": "inputs larger than L2" if m["step_bytes"] / L > 126e6 * 1.5 else "working set fits L2 (latency case)",
+            "step_hbm_gbs": m["step_gbs"], "step_frac_of_measured_peak": m["step_gbs"] / peak,
+            "step_frac_of_nominal_8TBs": m["step_gbs"] / NOMINAL_HBM_GBS,
+            "kernel_ms_per_step": m["kernel_ms_per_step"],
+            "read_ceiling_gbs": m["ceilings"],
             "sync_merge_host_us": merge_us,
-            **({"bytes_duplicated_at_spawn": spawn_copy_bytes} if spawn_copy_bytes is not None else {}),
+            **({"bytes_duplicated_at_spawn": m["spawn_copy_bytes"]} if m["spawn_copy_bytes"] is not None else {}),
+            **({"other_workloads": others} if others else {}),
         },
-        "clocks": clocks,
-        "e2e": {"value": e2e_tokens / e2e_s, "unit": UNIT, "h2d_bytes_per_step": h2d,
-                "d2h_bytes_per_step": d2h, "steps": e2e_steps},
-        "gpu_launches": launches,
-        "roofline": {"bound": "hbm", "kernel": dom_name, "achieved": achieved, "peak": peak, "peak_kind": peak_kind,
-                     "unit": "GB/s", "frac": achieved / peak, "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
-                     "traffic": NCU_TRAFFIC_BYTES.get((args.workload, args.size)) if dom == 0 and args.layout == "pool" else None, "bytes_per_launch": dom_bytes_per_launch,
-                     "ms_per_launch": dom_ms},
+        "clocks": m["clocks"],
+        "e2e": m["e2e"],
+        "gpu_launches": m["launches"],
+        "roofline": {"bound": "hbm", "kernel": m["dom"], "achieved": m["dom_gbs"], "peak": peak, "peak_kind": peak_kind,
+                     "unit": "GB/s", "frac": m["dom_gbs"] / peak, "frac_of_nominal_8TBs": m["dom_gbs"] / NOMINAL_HBM_GBS,
+                     "traffic": traffic, "bytes_per_launch": m["dom_bytes"], "ms_per_launch": m["dom_ms"],
+                     "launches_timed": m["kernel_ms_per_step"]["launches_timed"]},
         "cpu_baseline": oracle_sample(args.workload, budget_s=20.0) if world == 1 and not args.no_cpu_baseline else None,
     }
     print(json.dumps(result))
@@ -435,25 +587,17 @@ def unique_tokens_per_step(script):
     return out
 
 
-def run_trace(args):
+def trace_measure(device, rank, world, local, size="full", steps=200, warmup=3):
+    """Replays the synthetic interpreter trace op by op (step plan, append, attention of every layer, spawn, finish,
+    sync merge) and times `steps` decode steps after `warmup`.  Returns the figures as a dict."""
     import torch
+    import torch.distributed as dist
     from paper_2502_11517_b200 import binding
-    from paper_2502_11517_b200.build import build
     from paper_2502_11517_b200.sharding import aggregate
     from pasta_workloads import cfg5_trace
-    import torch.distributed as dist
-    rank = int(os.environ.get("RANK", "0")); world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
-    if rank == 0:
-        build()
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local)); dist.barrier()
-    device = torch.device("cuda", local); torch.cuda.set_device(device)
-    warm = max(args.warmup, 3)
-    n_req, n_layers = (256, 32) if args.size == "full" else (64, 8)
-    script = cfg5_trace(n_requests=n_req, n_steps=args.steps + warm, n_layers=n_layers)
+    warm = max(warmup, 3)
+    n_req, n_layers = (256, 32) if size == "full" else (64, 8)
+    script = cfg5_trace(n_requests=n_req, n_steps=steps + warm, n_layers=n_layers)
     geo = script.geometry
     uniq = unique_tokens_per_step(script)
     max_n = max(len(op[1]) for op in script.ops if op[0] == "step")
@@ -495,7 +639,7 @@ def run_trace(args):
                 if world > 1:
                     dist.barrier()
                 launches0 = pool.launch_count()
-                pool.profile_enable(True)
+                pool.profile_enable(8)
                 sampler = ClockSampler(local) if rank == 0 else None
                 t_wall0 = time.time(); ev0.record(stream)
             n = len(op[1])
@@ -518,25 +662,56 @@ def run_trace(args):
     timed_calls = max(1, max(kernel_launches))
     assert pool.status() == 0, "a kernel reported an error"
     all_tokens, worst_s = aggregate(float(tokens), ms * 1e-3)
+    peak, peak_kind = measured_peak()
+    gbs = bytes_ / (ms * 1e-3) / 1e9
+    res = {"workload": script.name, "size": size, "script": script, "steps": steps, "warmup": warm,
+           "value": all_tokens / worst_s, "thread_tokens_per_s": all_tokens / worst_s, "ms_per_step": worst_s * 1e3 / steps,
+           "requests": n_req, "layers": L, "thread_tokens_timed": tokens, "max_thread_tokens_per_step": max_n,
+           "sync_merges_timed": int(merges), "pool_pages": script.n_pages, "pool_gb": script.n_pages * 65536 * L / 1e9,
+           "unique_kv_bytes_timed": bytes_, "step_hbm_gbs": gbs, "step_frac_of_measured_peak": gbs / peak,
+           "kernel_ms_per_step": {"tensor": kernel_ms[0] / timed_calls, "warp": kernel_ms[1] / timed_calls,
+                                  "merge": kernel_ms[2] / timed_calls, "launches_timed": timed_calls,
+                                  "where": "every eighth step of the timed region"},
+           "step_begin_call_ms": host_s * 1e3 / steps, "clocks": clocks, "gpu_launches": launches, "peak": peak,
+           "peak_kind": peak_kind}
+    pool.close()
+    del pool, out, kv_pool, kv_pool2, q_pool
+    torch.cuda.empty_cache()
+    return res
+
+
+def run_trace(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2502_11517_b200.build import build
+    rank = int(os.environ.get("RANK", "0")); world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
     if rank == 0:
-        peak, peak_kind = measured_peak()
-        gbs = bytes_ / (ms * 1e-3) / 1e9
+        build()
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local)); dist.barrier()
+    device = torch.device("cuda", local); torch.cuda.set_device(device)
+    r = trace_measure(device, rank, world, local, size=args.size, steps=args.steps, warmup=args.warmup)
+    if rank == 0:
+        peak, gbs = r["peak"], r["step_hbm_gbs"]
         print(json.dumps({
-            "metric": METRIC, "value": all_tokens / worst_s, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": warm,
-            "ms_per_step": worst_s * 1e3 / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "metric": METRIC, "value": r["value"], "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": r["warmup"],
+            "ms_per_step": r["ms_per_step"], "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": "trace", "size": args.size, "script": script.name, "requests": n_req, "layers": L,
-                       "thread_tokens_timed": tokens, "max_thread_tokens_per_step": max_n, "sync_merges_timed": int(merges),
-                       "pool_pages": script.n_pages, "pool_gb": script.n_pages * 65536 * L / 1e9,
-                       "unique_kv_bytes_timed": bytes_, "l2": "inputs larger than L2",
-                       "step_hbm_gbs": gbs, "step_frac_of_measured_peak": gbs / peak, "step_frac_of_nominal_8TBs": gbs / NOMINAL_HBM_GBS,
-                       "kernel_ms_per_step": {"tensor": kernel_ms[0] / timed_calls, "warp": kernel_ms[1] / timed_calls,
-                                              "merge": kernel_ms[2] / timed_calls, "steps_timed": timed_calls},
-                       "step_begin_call_ms": host_s * 1e3 / args.steps,
+            "config": {"workload": "trace", "size": args.size, "script": r["workload"], "requests": r["requests"],
+                       "layers": r["layers"], "thread_tokens_timed": r["thread_tokens_timed"],
+                       "max_thread_tokens_per_step": r["max_thread_tokens_per_step"],
+                       "sync_merges_timed": r["sync_merges_timed"], "pool_pages": r["pool_pages"], "pool_gb": r["pool_gb"],
+                       "unique_kv_bytes_timed": r["unique_kv_bytes_timed"], "l2": "inputs larger than L2",
+                       "step_hbm_gbs": gbs, "step_frac_of_measured_peak": gbs / peak,
+                       "step_frac_of_nominal_8TBs": gbs / NOMINAL_HBM_GBS, "kernel_ms_per_step": r["kernel_ms_per_step"],
+                       "step_begin_call_ms": r["step_begin_call_ms"],
                        "step_begin_note": "wall time inside pasta_step_begin; includes waiting for the device when the host runs ahead"},
-            "clocks": clocks, "e2e": None, "gpu_launches": launches,
+            "clocks": r["clocks"], "e2e": None, "gpu_launches": r["gpu_launches"],
             "roofline": {"bound": "hbm", "kernel": "whole step (tensor + warp + merge + append)", "achieved": gbs, "peak": peak,
-                         "peak_kind": peak_kind, "unit": "GB/s", "frac": gbs / peak, "traffic": None},
+                         "peak_kind": r["peak_kind"], "unit": "GB/s", "frac": gbs / peak, "traffic": None},
             "cpu_baseline": None}))
     if world > 1:
         dist.destroy_process_group()
@@ -676,6 +851,20 @@ def time_sync_merge():
 
 # ------------------------------------------------------------------------------------------------ oracle arm
 _ORACLE_STATE = {}
+ORACLE_WORKER_GB = {"long_shared_prefix": 1.3, "batched": 1.2, "single_request": 0.3}   # resident + transient, per worker
+
+
+def _oracle_script(workload: str):
+    """The bounded sample of a workload that the oracle is timed on: (script, what it is, layers it stands for)."""
+    from pasta_workloads import cfg2_single_request, cfg3_batched, cfg4_long_prefix
+    if workload == "long_shared_prefix":
+        return (cfg4_long_prefix(n_requests=1),
+                "the 17 thread-tokens of 1 of the 8 requests (32768-token prefix, 16 forks), 1 layer", 1)
+    if workload == "batched":
+        return cfg3_batched(n_layers=1), "all thread-tokens of the 64 requests, 1 of 32 layers (time scaled by 32)", 32
+    script = cfg2_single_request("a")
+    script.ops = script.ops[:11]
+    return script, "step A: the 5 thread-tokens of the request, 1 layer", 1
 
 
 def _oracle_state(workload: str):
@@ -683,16 +872,8 @@ def _oracle_state(workload: str):
     if workload in _ORACLE_STATE:
         return _ORACLE_STATE[workload]
     from oracle import OracleReplay
-    from pasta_workloads import cfg2_single_request, cfg3_batched, cfg4_long_prefix, step_tensors
-    if workload == "long_shared_prefix":
-        script = cfg4_long_prefix(n_requests=1); passes = 4
-        sample = "the 17 thread-tokens of 1 of 8 requests (32768-token prefix, 16 forks), 1 layer, 4 passes"
-    elif workload == "batched":
-        script = cfg3_batched(n_layers=1); passes = 8
-        sample = "all thread-tokens of the 64 requests, 1 of 32 layers, 8 passes (time scaled by 32 layers)"
-    else:
-        script = cfg2_single_request("a"); script.ops = script.ops[:11]; passes = 50
-        sample = "step A: 5 thread-tokens of the request, 1 layer, 50 passes"
+    from pasta_workloads import step_tensors
+    script, _, _ = _oracle_script(workload)
     rep = OracleReplay(script)
     last = len(script.ops) - 1
     for i in range(last):
@@ -702,38 +883,112 @@ def _oracle_state(workload: str):
     slots = [s for s in rep.model.reserve(op[1]) if s is not None]
     rep.stores[0].write(slots, k, v)
     queries = [(e[0], e[1]) for e in op[1]]
-    _ORACLE_STATE[workload] = (rep, queries, q, sample, passes)
+    _ORACLE_STATE[workload] = (rep, queries, q)
     return _ORACLE_STATE[workload]
 
 
-def oracle_sample(workload: str, budget_s: float = 20.0, steps: int = 1):
-    """Times the fp64 CPU oracle, as it stands, on a bounded sample of the workload: the queries of the
-    workload's first request(s), in layer 0 (the attention is what is timed).  Returns the cpu_baseline object."""
-    from oracle import decode_attention
-    rep, queries, q, sample, passes = _oracle_state(workload)
-    steps = max(steps, passes)
-    times = []
-    t_all = time.perf_counter()
-    for _ in range(steps):
-        t0 = time.perf_counter()
-        done = 0
-        for i, qq in enumerate(queries):
-            decode_attention(rep.model, rep.stores[0], [qq], q[i:i + 1])
-            done += 1
-            if time.perf_counter() - t_all > budget_s:
-                break
-        times.append((time.perf_counter() - t0, done))
-        if time.perf_counter() - t_all > budget_s:
-            break
-    dt = sum(t for t, _ in times); done = sum(d for _, d in times)
-    layers = 32 if workload == "batched" else 1
+def _oracle_worker_init(workload, root, ready):
+    """Runs once in every worker process: one compute thread, its own copy of the oracle's state."""
+    if root not in sys.path:
+        sys.path.insert(0, root)
     try:
-        from threadpoolctl import threadpool_info
-        cores = max([p.get("num_threads", 1) for p in threadpool_info()] or [1])
+        import torch
+        torch.set_num_threads(1)
     except Exception:
-        cores = 1
-    return {"value": done / (dt * layers), "unit": UNIT, "cores": cores, "kind": "oracle",
-            "sample": f"{done} thread-tokens: {sample}", "seconds": dt}
+        pass
+    try:
+        from threadpoolctl import threadpool_limits
+        threadpool_limits(1)
+    except Exception:
+        pass
+    _oracle_state(workload)
+    with ready.get_lock():
+        ready.value += 1
+
+
+def _oracle_worker_query(task):
+    """One query of the sample through the oracle, as it stands; returns the seconds it took in this worker."""
+    workload, i = task
+    from oracle import decode_attention
+    rep, queries, q = _oracle_state(workload)
+    t0 = time.perf_counter()
+    decode_attention(rep.model, rep.stores[0], [queries[i]], q[i:i + 1])
+    return time.perf_counter() - t0
+
+
+class OraclePool:
+    """The fp64 oracle on the host's cores: one single-threaded worker process per core the process may use (fewer when
+    memory is short), each with its own copy of the state; queries of the sample are independent and are handed out one
+    by one.  Workers are spawned, not forked: this process may already hold a CUDA context."""
+
+    def __init__(self, workload: str):
+        import multiprocessing as mp
+        self.workload = workload
+        self.script, self.what, self.layers = _oracle_script(workload)
+        self.n_queries = len(self.script.ops[-1][1])
+        self.cores_available = len(os.sched_getaffinity(0))
+        workers = self.cores_available
+        try:
+            import psutil
+            room = psutil.virtual_memory().available / 2**30 * 0.5
+            workers = max(1, min(workers, int(room / ORACLE_WORKER_GB.get(workload, 1.0))))
+        except Exception:
+            workers = min(workers, 16)
+        self.workers = min(workers, 96)
+        ctx = mp.get_context("spawn")
+        ready = ctx.Value("i", 0)
+        saved = {k: os.environ.get(k) for k in ("OMP_NUM_THREADS", "OPENBLAS_NUM_THREADS", "MKL_NUM_THREADS")}
+        os.environ.update({k: "1" for k in saved})           # inherited by the workers: one thread each
+        try:
+            self.pool = ctx.Pool(self.workers, initializer=_oracle_worker_init, initargs=(workload, ROOT, ready))
+        finally:
+            for k, v in saved.items():
+                if v is None:
+                    os.environ.pop(k, None)
+                else:
+                    os.environ[k] = v
+        t0 = time.time()
+        while ready.value < self.workers and time.time() - t0 < 300:
+            time.sleep(0.05)
+        if ready.value < self.workers:
+            raise RuntimeError(f"only {ready.value} of {self.workers} oracle workers came up")
+        self.one_query_s = None
+
+    def one_core(self, repeats: int = 6) -> float:
+        """Seconds per query with a single worker busy (the fastest of a few: the first calls of a worker are cold)."""
+        ts = [self.pool.apply(_oracle_worker_query, ((self.workload, i % self.n_queries),)) for i in range(repeats)]
+        self.one_query_s = float(min(ts))
+        return self.one_query_s
+
+    def sample(self, budget_s: float):
+        """Hands whole passes over the sample's queries to the workers for about budget_s seconds of wall time."""
+        if self.one_query_s is None:
+            self.one_core()
+        per_pass = self.n_queries * self.one_query_s / min(self.workers, self.n_queries)
+        passes = int(max(1, min(256, budget_s / max(per_pass, 1e-6))))
+        # enough queries in the air to keep every worker busy
+        passes = max(passes, -(-self.workers // self.n_queries))
+        tasks = [(self.workload, i) for _ in range(passes) for i in range(self.n_queries)]
+        t0 = time.perf_counter()
+        self.pool.map(_oracle_worker_query, tasks, chunksize=1)
+        wall = time.perf_counter() - t0
+        return {"value": len(tasks) / (wall * self.layers), "unit": UNIT, "cores": self.workers,
+                "cores_available": self.cores_available, "kind": "oracle",
+                "sample": f"{len(tasks)} thread-tokens ({passes} passes over {self.what})", "seconds": wall,
+                "one_core_value": 1.0 / (self.one_query_s * self.layers), "thread_tokens": len(tasks)}
+
+    def close(self):
+        self.pool.close()
+        self.pool.join()
+
+
+def oracle_sample(workload: str, budget_s: float = 20.0):
+    """The cpu_baseline object: the oracle, as it stands, on a bounded sample of the workload, over the host's cores."""
+    pool = OraclePool(workload)
+    try:
+        return pool.sample(budget_s)
+    finally:
+        pool.close()
 
 
 def run_reference(args):
@@ -741,16 +996,20 @@ def run_reference(args):
     if rank != 0:
         return
     t0 = time.perf_counter()
-    _oracle_state(args.workload)                       # set-up once, outside the steps
-    per_step = max(0.25, min(20.0, 150.0 / max(1, args.steps + args.warmup)))
-    for _ in range(args.warmup):
-        oracle_sample(args.workload, budget_s=per_step)
-    res = [oracle_sample(args.workload, budget_s=per_step) for _ in range(args.steps)]
+    pool = OraclePool(args.workload)                   # set-up once, outside the steps
+    try:
+        per_step = max(0.5, min(20.0, 120.0 / max(1, args.steps + args.warmup)))
+        for _ in range(args.warmup):
+            pool.sample(per_step)
+        res = [pool.sample(per_step) for _ in range(args.steps)]
+    finally:
+        pool.close()
     secs = sum(r["seconds"] for r in res)
-    done = sum(float(r["sample"].split()[0]) for r in res)
-    layers = 32 if args.workload == "batched" else 1
-    value = done / (secs * layers)
-    base = dict(res[-1]); base["value"] = value
+    done = sum(r["thread_tokens"] for r in res)
+    value = done / (secs * pool.layers)
+    base = {"value": value, "unit": UNIT, "cores": pool.workers, "cores_available": pool.cores_available, "kind": "oracle",
+            "sample": f"{done} thread-tokens in {args.steps} steps, each step whole passes over {pool.what}",
+            "seconds": secs, "one_core_value": res[-1]["one_core_value"]}
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": int(os.environ.get("WORLD_SIZE", "1")),
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": secs / max(1, args.steps) * 1e3,
@@ -769,6 +1028,10 @@ def main():
     ap.add_argument("--workload", default="long_shared_prefix")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-others", dest="others", action="store_false",
+                    help="skip the shorter runs of the other configurations that ride along with the default workload")
+    ap.add_argument("--kernel", default="auto", choices=["auto", "warp"],
+                    help="warp: send every stream through the warp-shuffle kernel (PASTA_FLAG_NO_TENSOR_PATH)")
     ap.add_argument("--out-dtype", default="fp32", choices=["fp32", "bf16"],
                     help="type of the attention output (bf16 halves the device-to-host bytes of the end-to-end path)")
     ap.add_argument("--layout", default="pool", choices=["pool", "naive_rows"],

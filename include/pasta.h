@@ -239,6 +239,22 @@ pasta_status_t pasta_step_device(pasta_pool_t *pool, int32_t n, const int32_t *r
  * Entries append at most one token each here (n_new[i] > 1: INVALID_ARG, nothing reserved).
  */
 pasta_status_t pasta_step_host_bytes(pasta_pool_t *pool, int32_t n, size_t *out);
+/*
+ * The same step in two halves, so that a caller can keep two steps in flight (Section 3: the decode loop is one
+ * step after the other; what overlaps here are the copies of one step with the kernels of its neighbour).
+ * pasta_step_host_begin enqueues everything pasta_step_host does (the input copies and the copy of `out` back to
+ * the host run on streams of the pool's own, ordered with `stream` by events) and returns without waiting;
+ * pasta_step_host_wait blocks until the OLDEST step begun and not yet waited for has delivered its `out`.
+ * k_new, v_new, q and out must stay untouched between the two calls.  At most two steps may be begun and not
+ * waited for (a third begin: BAD_STATE, as is a wait with nothing begun).  With `staging_bytes` of at least twice
+ * pasta_step_host_bytes the inputs of a step are copied while the step before still computes; with less, the
+ * copies wait for that step to leave the area.  Pinned host memory is required for any overlap.
+ */
+pasta_status_t pasta_step_host_begin(pasta_pool_t *pool, int32_t n, const int32_t *req_ids,
+                                     const int32_t *thread_ids, const int32_t *n_new,
+                                     const void *k_new, const void *v_new, const void *q, void *out,
+                                     void *staging, size_t staging_bytes, float scale, void *stream);
+pasta_status_t pasta_step_host_wait(pasta_pool_t *pool);
 pasta_status_t pasta_step_host(pasta_pool_t *pool, int32_t n, const int32_t *req_ids,
                                const int32_t *thread_ids, const int32_t *n_new,
                                const void *k_new, const void *v_new, const void *q, void *out,
@@ -319,6 +335,16 @@ pasta_status_t pasta_debug_set_wait_limit(pasta_pool_t *pool, int64_t cycles);
  * of such a launch are undefined.  Set a short limit first (pasta_debug_set_wait_limit); 0 switches the hook off.
  */
 pasta_status_t pasta_debug_hold_roles(pasta_pool_t *pool, int32_t role_mask);
+/*
+ * Measurement aid (no counterpart in the paper): enqueues a kernel that reads `bytes` of device memory at `src`
+ * (16-byte aligned; NULL = the pool's own KV memory, all of it) and does nothing with them, so that a benchmark can
+ * time what a read-only kernel is given on this GPU next to the attention kernel.  mode 0: plain 16-byte loads;
+ * mode 1: bulk copies into shared memory, one CTA per SM with 3 x 64 KB in flight, the mechanism of the tensor-core
+ * attention kernel (whole 64 KB chunks only); mode 2: the same, every 8 KB piece taken from a pseudo-random place of
+ * the buffer, the way a stream's pages lie in a pool that hands pages out in random order.  Writes nothing but 8
+ * scratch bytes of the workspace.
+ */
+pasta_status_t pasta_debug_stream_read(pasta_pool_t *pool, const void *src, size_t bytes, int32_t mode, void *stream);
 pasta_status_t pasta_debug_wait_expiry(pasta_pool_t *pool, void *stream);
 
 /* Number of kernels this pool has launched so far (for launch accounting). */

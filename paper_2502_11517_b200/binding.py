@@ -28,6 +28,7 @@ EXPORTS = [
     "pasta_thread_spawn_predicted", "pasta_step_positions", "pasta_kv_append_rope", "pasta_rope_queries",
     "pasta_kv_append_run_rope", "pasta_step_device",
     "pasta_last_cuda_error", "pasta_debug_set_wait_limit", "pasta_debug_wait_expiry", "pasta_debug_hold_roles",
+    "pasta_debug_stream_read", "pasta_step_host_begin", "pasta_step_host_wait",
 ]
 
 
@@ -257,6 +258,27 @@ class Pool:
                                      _dev(out), _dev(staging), C.c_size_t(staging.numel() * staging.element_size()),
                                      C.c_float(scale), _stream(stream)), "pasta_step_host")
         self._last_n = len(r)
+
+    def step_host_begin(self, req_ids, thread_ids, n_new, k_new, v_new, q, out, staging, scale: float = 0.0,
+                        stream=None) -> None:
+        """First half of step_host: everything is enqueued, nothing is waited for (at most two steps in flight)."""
+        r, t = _i32(req_ids), _i32(thread_ids)
+        nn = None if n_new is None else _i32(n_new)
+        _check(lib().pasta_step_host_begin(self._h, len(r), _ptr(r), _ptr(t), _ptr(nn), _dev(k_new), _dev(v_new), _dev(q),
+                                           _dev(out), _dev(staging), C.c_size_t(staging.numel() * staging.element_size()),
+                                           C.c_float(scale), _stream(stream)), "pasta_step_host_begin")
+        self._last_n = len(r)
+
+    def step_host_wait(self) -> None:
+        _check(lib().pasta_step_host_wait(self._h), "pasta_step_host_wait")
+
+    def debug_stream_read(self, src=None, mode: int = 0, stream=None) -> int:
+        """Enqueues the read-only measurement kernel over `src` (a torch CUDA tensor; None = the pool's KV memory);
+        returns the number of bytes it reads."""
+        nbytes = self.kv.numel() if src is None else src.numel() * src.element_size()
+        _check(lib().pasta_debug_stream_read(self._h, _dev(src), C.c_size_t(nbytes), mode, _stream(stream)),
+               "pasta_debug_stream_read")
+        return nbytes // 65536 * 65536 if mode else nbytes // 16 * 16
 
     # ---- introspection
     def kv_read(self, layer: int, req: int, stream_id: int, start: int, m: int, stream=None):

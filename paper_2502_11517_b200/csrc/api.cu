@@ -90,6 +90,13 @@ struct pasta_pool {
   cudaEvent_t plan_ready[2] = {nullptr, nullptr};   // recorded on copy_stream after the upload of buffer b
   cudaEvent_t work_mark[2] = {nullptr, nullptr};    // recorded on the caller's stream at the start of step i (slot i % 2)
   int64_t step_index = 0;
+  // pasta_step_host_begin / _wait: at most two steps in flight; their copies run on streams of the pool
+  cudaStream_t d2h_stream = nullptr;
+  cudaEvent_t host_inputs_ready[2] = {nullptr, nullptr};   // copy_stream: k / v / q of the step are on the device
+  cudaEvent_t host_attn_done[2] = {nullptr, nullptr};      // caller's stream: the step's outputs are in the staging area
+  cudaEvent_t host_out_ready[2] = {nullptr, nullptr};      // d2h_stream: the outputs are in the caller's host buffer
+  int host_slot_of[2] = {0, 0};                            // staging slot used by the step with event slot e
+  int64_t host_submitted = 0, host_waited = 0;
   // kernel timing (pasta_profile_*): events[4 * i .. 4 * i + 3] bracket the three kernels of call i
   bool profiling = false;
   int prof_stride = 1;                  // every prof_stride-th pasta_decode_attn launch group is timed
@@ -206,9 +213,13 @@ pasta_status_t pasta_pool_create(const pasta_pool_config_t *cfg, pasta_pool_t **
     }
     if (e == cudaSuccess) e = cudaMallocHost(reinterpret_cast<void **>(&p->status_host), 64);
     if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&p->copy_stream, cudaStreamNonBlocking);
+    if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&p->d2h_stream, cudaStreamNonBlocking);
     for (int b = 0; b < 2 && e == cudaSuccess; ++b) {
       e = cudaEventCreateWithFlags(&p->plan_ready[b], cudaEventDisableTiming);
       if (e == cudaSuccess) e = cudaEventCreateWithFlags(&p->work_mark[b], cudaEventDisableTiming);
+      if (e == cudaSuccess) e = cudaEventCreateWithFlags(&p->host_inputs_ready[b], cudaEventDisableTiming);
+      if (e == cudaSuccess) e = cudaEventCreateWithFlags(&p->host_attn_done[b], cudaEventDisableTiming);
+      if (e == cudaSuccess) e = cudaEventCreateWithFlags(&p->host_out_ready[b], cudaEventDisableTiming);
     }
     uint8_t *ws = static_cast<uint8_t *>(cfg->workspace);
     if (e == cudaSuccess) e = cudaMemset(ws, 0, 256);
@@ -248,9 +259,13 @@ pasta_status_t pasta_pool_destroy(pasta_pool_t *p) {
   }
   if (p->status_host) cudaFreeHost(p->status_host);
   if (p->copy_stream) { cudaStreamSynchronize(p->copy_stream); cudaStreamDestroy(p->copy_stream); }
+  if (p->d2h_stream) { cudaStreamSynchronize(p->d2h_stream); cudaStreamDestroy(p->d2h_stream); }
   for (int b = 0; b < 2; ++b) {
     if (p->plan_ready[b]) cudaEventDestroy(p->plan_ready[b]);
     if (p->work_mark[b]) cudaEventDestroy(p->work_mark[b]);
+    if (p->host_inputs_ready[b]) cudaEventDestroy(p->host_inputs_ready[b]);
+    if (p->host_attn_done[b]) cudaEventDestroy(p->host_attn_done[b]);
+    if (p->host_out_ready[b]) cudaEventDestroy(p->host_out_ready[b]);
   }
   for (cudaEvent_t e : p->prof_events) if (e) cudaEventDestroy(e);
   delete p;
@@ -512,11 +527,12 @@ pasta_status_t pasta_step_host_bytes(pasta_pool_t *p, int32_t n, size_t *out) {
   return PASTA_OK;
 }
 
-pasta_status_t pasta_step_host(pasta_pool_t *p, int32_t n, const int32_t *req_ids, const int32_t *thread_ids,
-                               const int32_t *n_new, const void *k_new, const void *v_new, const void *q, void *out,
-                               void *staging, size_t staging_bytes, float scale, void *stream) {
+pasta_status_t pasta_step_host_begin(pasta_pool_t *p, int32_t n, const int32_t *req_ids, const int32_t *thread_ids,
+                                     const int32_t *n_new, const void *k_new, const void *v_new, const void *q, void *out,
+                                     void *staging, size_t staging_bytes, float scale, void *stream) {
   if (!p || !q || !out || !staging) return PASTA_ERR_INVALID_ARG;
   if (p->host_only) return PASTA_ERR_BAD_STATE;
+  if (p->host_submitted - p->host_waited >= 2) return PASTA_ERR_BAD_STATE;      // two steps are in flight already
   size_t need = 0;
   pasta_status_t s = pasta_step_host_bytes(p, n, &need);
   if (s != PASTA_OK) return s;
@@ -530,30 +546,63 @@ pasta_status_t pasta_step_host(pasta_pool_t *p, int32_t n, const int32_t *req_id
       n_app += static_cast<size_t>(n_new[i]);
     }
   }
+  if (n_app > 0 && (!k_new || !v_new)) return PASTA_ERR_INVALID_ARG;
+  // A staging area of twice the size holds two steps: the inputs of this step then travel while the kernels of the
+  // step before still read theirs.  With one slot the copies wait until that step has left the area.
+  const int n_slots = staging_bytes >= 2 * need ? 2 : 1;
+  const int64_t i = p->host_submitted;
+  const int e = static_cast<int>(i & 1);
+  int slot = 0;
+  if (i > p->host_waited) slot = n_slots == 2 ? p->host_slot_of[e ^ 1] ^ 1 : 0;
   const size_t L = p->cfg.n_layers, d = p->cfg.head_dim;
   const size_t kv_full = align_up(L * n * p->cfg.n_kv_heads * d * 2, 256);
   const size_t kv_bytes = L * n_app * p->cfg.n_kv_heads * d * 2;
   const size_t q_bytes = L * n * p->cfg.n_q_heads * d * 2;
-  uint8_t *base = static_cast<uint8_t *>(staging);
+  uint8_t *base = static_cast<uint8_t *>(staging) + size_t(slot) * need;
   uint8_t *k_dev = base, *v_dev = base + kv_full, *q_dev = base + 2 * kv_full;
   uint8_t *o_dev = q_dev + align_up(q_bytes, 256);
-  if (n_app > 0 && (!k_new || !v_new)) return PASTA_ERR_INVALID_ARG;
-  // the input copies go first: the host plans the step while they are in flight
+  // the input copies go first, on the pool's copy stream: the host plans the step while they are in flight.  The
+  // step in flight (if any) is done with the slot once its outputs have reached the host, when it shares the slot.
+  if (i > p->host_waited && n_slots == 1) PASTA_CUDA(cudaStreamWaitEvent(p->copy_stream, p->host_out_ready[e ^ 1], 0));
   if (n_app > 0) {
-    PASTA_CUDA(cudaMemcpyAsync(k_dev, k_new, kv_bytes, cudaMemcpyHostToDevice, st));
-    PASTA_CUDA(cudaMemcpyAsync(v_dev, v_new, kv_bytes, cudaMemcpyHostToDevice, st));
+    PASTA_CUDA(cudaMemcpyAsync(k_dev, k_new, kv_bytes, cudaMemcpyHostToDevice, p->copy_stream));
+    PASTA_CUDA(cudaMemcpyAsync(v_dev, v_new, kv_bytes, cudaMemcpyHostToDevice, p->copy_stream));
   }
-  PASTA_CUDA(cudaMemcpyAsync(q_dev, q, q_bytes, cudaMemcpyHostToDevice, st));
+  PASTA_CUDA(cudaMemcpyAsync(q_dev, q, q_bytes, cudaMemcpyHostToDevice, p->copy_stream));
+  PASTA_CUDA(cudaEventRecord(p->host_inputs_ready[e], p->copy_stream));
   s = pasta_step_begin(p, n, req_ids, thread_ids, n_new, stream);
   if (s != PASTA_OK) return s;
+  PASTA_CUDA(cudaStreamWaitEvent(st, p->host_inputs_ready[e], 0));
   s = pasta_kv_append(p, 0, p->cfg.n_layers, k_dev, v_dev, stream);
   if (s != PASTA_OK) return s;
   s = pasta_decode_attn(p, 0, p->cfg.n_layers, q_dev, o_dev, nullptr, scale, stream);
   if (s != PASTA_OK) return s;
   const size_t out_bytes = (p->cfg.flags & PASTA_FLAG_OUT_BF16) ? q_bytes : q_bytes * 2;
-  PASTA_CUDA(cudaMemcpyAsync(out, o_dev, out_bytes, cudaMemcpyDeviceToHost, st));
-  PASTA_CUDA(cudaStreamSynchronize(st));
+  PASTA_CUDA(cudaEventRecord(p->host_attn_done[e], st));
+  PASTA_CUDA(cudaStreamWaitEvent(p->d2h_stream, p->host_attn_done[e], 0));
+  PASTA_CUDA(cudaMemcpyAsync(out, o_dev, out_bytes, cudaMemcpyDeviceToHost, p->d2h_stream));
+  PASTA_CUDA(cudaEventRecord(p->host_out_ready[e], p->d2h_stream));
+  p->host_slot_of[e] = slot;
+  p->host_submitted = i + 1;
   return PASTA_OK;
+}
+
+pasta_status_t pasta_step_host_wait(pasta_pool_t *p) {
+  if (!p) return PASTA_ERR_INVALID_ARG;
+  if (p->host_only || p->host_waited == p->host_submitted) return PASTA_ERR_BAD_STATE;
+  PASTA_CUDA(cudaEventSynchronize(p->host_out_ready[p->host_waited & 1]));
+  p->host_waited += 1;
+  return PASTA_OK;
+}
+
+pasta_status_t pasta_step_host(pasta_pool_t *p, int32_t n, const int32_t *req_ids, const int32_t *thread_ids,
+                               const int32_t *n_new, const void *k_new, const void *v_new, const void *q, void *out,
+                               void *staging, size_t staging_bytes, float scale, void *stream) {
+  if (p && p->host_submitted != p->host_waited) return PASTA_ERR_BAD_STATE;     // a pasta_step_host_begin is outstanding
+  pasta_status_t s = pasta_step_host_begin(p, n, req_ids, thread_ids, n_new, k_new, v_new, q, out, staging, staging_bytes,
+                                           scale, stream);
+  if (s != PASTA_OK) return s;
+  return pasta_step_host_wait(p);
 }
 
 pasta_status_t pasta_kv_read(pasta_pool_t *p, int32_t layer, int32_t req, int32_t stream_id, int32_t start, int32_t m,
@@ -655,6 +704,17 @@ pasta_status_t pasta_debug_set_wait_limit(pasta_pool_t *p, int64_t cycles) {
   if (!p) return PASTA_ERR_INVALID_ARG;
   if (p->host_only) return PASTA_ERR_BAD_STATE;
   p->pv.wait_limit = cycles > 0 ? static_cast<long long>(cycles) : kWaitLimitCycles;
+  return PASTA_OK;
+}
+
+pasta_status_t pasta_debug_stream_read(pasta_pool_t *p, const void *src, size_t bytes, int32_t mode, void *stream) {
+  if (!p || mode < 0 || mode > 2) return PASTA_ERR_INVALID_ARG;
+  if (p->host_only) return PASTA_ERR_BAD_STATE;
+  if (!src) { src = p->cfg.kv_base; bytes = p->d.kv_bytes; }
+  if (reinterpret_cast<uintptr_t>(src) & 15) return PASTA_ERR_INVALID_ARG;
+  void *sink = reinterpret_cast<uint8_t *>(p->pv.status) + 64;      // inside the 256 status bytes of the workspace
+  PASTA_CUDA(launch_stream_read(src, bytes, mode, sink, p->pv.status, p->sm_count, static_cast<cudaStream_t>(stream)));
+  p->launches += 1;
   return PASTA_OK;
 }
 

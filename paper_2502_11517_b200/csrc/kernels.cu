@@ -176,6 +176,93 @@ __global__ void wait_expiry_kernel(PoolView pv) {
   if (!done && threadIdx.x == 0) report(pv.status, PASTA_ERR_TIMEOUT);
 }
 
+// =============================================================================================
+// Read-only streaming kernels for measurements: what this GPU delivers to a kernel that only reads, by the two
+// mechanisms the attention kernels use.  Neither computes anything worth naming.
+//   bulk:   one CTA per SM, a 3-stage ring of 64 KB filled by 8 KB bulk copies (the tensor-core kernel's producer
+//           without its consumers); chunk c goes to CTA c % grid; its 8 KB pieces are consecutive, or scattered.
+//   vector: 16-byte loads, eight in flight per thread, folded into one word so that they cannot be dropped.
+// =============================================================================================
+constexpr int R_STAGES = 3, R_STAGE_BYTES = 65536, R_PIECE = 8192;
+
+__global__ void __launch_bounds__(32, 1)
+stream_read_bulk_kernel(const uint8_t *__restrict__ src, int64_t n_chunks, int scattered, unsigned long long *sink,
+                        int32_t *status) {
+  extern __shared__ __align__(1024) uint8_t r_smem[];
+  __shared__ __align__(8) uint64_t bars[R_STAGES];
+  const int lane = threadIdx.x;
+  const uint32_t base = smem_u32(r_smem), bar = smem_u32(bars);
+  if (lane == 0) {
+    for (int s = 0; s < R_STAGES; ++s) mbar_init(bar + 8 * s, 1);
+    mbar_init_fence();
+  }
+  fence_proxy_async();
+  __syncwarp();
+  const int64_t mine = n_chunks > blockIdx.x ? (n_chunks - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
+  const uint64_t n_pieces = static_cast<uint64_t>(n_chunks) * (R_STAGE_BYTES / R_PIECE);
+  auto issue = [&](int64_t k) {
+    const int s = static_cast<int>(k % R_STAGES);
+    const uint64_t piece = static_cast<uint64_t>(blockIdx.x + k * gridDim.x) * (R_STAGE_BYTES / R_PIECE) + lane;
+    // scattered: every 8 KB piece comes from a place far from its neighbours' (its number times a large prime,
+    // modulo the number of pieces), the way the pages of a stream lie in a pool that hands out pages in random order
+    const uint64_t from_piece = scattered ? (piece * 2654435761ull) % n_pieces : piece;   // a prime: one-to-one
+    if (lane == 0) mbar_expect_tx(bar + 8 * s, R_STAGE_BYTES);
+    __syncwarp();
+    if (lane < R_STAGE_BYTES / R_PIECE)
+      bulk_g2s(base + s * R_STAGE_BYTES + lane * R_PIECE, src + from_piece * R_PIECE, R_PIECE, bar + 8 * s);
+  };
+  for (int64_t k = 0; k < R_STAGES && k < mine; ++k) issue(k);
+  int64_t landed = 0;
+  bool ok = true;
+  for (int64_t k = 0; k < mine; ++k) {
+    if (!__all_sync(0xffffffffu, mbar_wait_bounded(bar + 8 * (k % R_STAGES), (k / R_STAGES) & 1))) { ok = false; break; }
+    landed = k + 1;
+    if (k + R_STAGES < mine) issue(k + R_STAGES);
+  }
+  if (!ok) {
+    if (lane == 0) report(status, PASTA_ERR_TIMEOUT);
+    for (int64_t k = landed; k < mine && k < landed + R_STAGES; ++k)      // copies still in flight
+      mbar_wait_bounded(bar + 8 * (k % R_STAGES), (k / R_STAGES) & 1);
+    return;
+  }
+  if (lane == 0 && mine > 0) atomicAdd(sink, static_cast<unsigned long long>(r_smem[0]));
+}
+
+__global__ void __launch_bounds__(256)
+stream_read_vector_kernel(const uint4 *__restrict__ src, int64_t n_vec, unsigned long long *sink) {
+  const int64_t stride = static_cast<int64_t>(gridDim.x) * blockDim.x;
+  int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  uint32_t acc = 0;
+  for (; i + 7 * stride < n_vec; i += 8 * stride) {
+    uint4 v[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) v[j] = __ldcs(src + i + j * stride);
+#pragma unroll
+    for (int j = 0; j < 8; ++j) acc ^= v[j].x ^ v[j].y ^ v[j].z ^ v[j].w;
+  }
+  for (; i < n_vec; i += stride) { const uint4 v = __ldcs(src + i); acc ^= v.x ^ v.y ^ v.z ^ v.w; }
+  if (acc == 0x9e3779b9u) atomicAdd(sink, 1ull);        // practically never: the loads have to be made to find out
+}
+
+cudaError_t launch_stream_read(const void *src, size_t bytes, int mode, void *sink, int32_t *status, int sm_count,
+                               cudaStream_t st) {
+  if (mode == 1 || mode == 2) {
+    static uint64_t prepared = 0;
+    cudaError_t e = raise_smem_limit(reinterpret_cast<const void *>(stream_read_bulk_kernel), R_STAGES * R_STAGE_BYTES, &prepared);
+    if (e != cudaSuccess) return e;
+    const int64_t n_chunks = static_cast<int64_t>(bytes / R_STAGE_BYTES);
+    if (n_chunks == 0) return cudaSuccess;
+    stream_read_bulk_kernel<<<sm_count, 32, R_STAGES * R_STAGE_BYTES, st>>>(
+        static_cast<const uint8_t *>(src), n_chunks, mode == 2, static_cast<unsigned long long *>(sink), status);
+  } else {
+    const int64_t n_vec = static_cast<int64_t>(bytes / 16);
+    if (n_vec == 0) return cudaSuccess;
+    stream_read_vector_kernel<<<sm_count * 8, 256, 0, st>>>(static_cast<const uint4 *>(src), n_vec,
+                                                           static_cast<unsigned long long *>(sink));
+  }
+  return cudaGetLastError();
+}
+
 cudaError_t launch_wait_expiry(const PoolView &pv, cudaStream_t st) {
   wait_expiry_kernel<<<1, 32, 0, st>>>(pv);
   return cudaGetLastError();

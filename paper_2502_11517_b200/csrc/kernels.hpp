@@ -47,6 +47,10 @@ cudaError_t launch_attn_tensor(const PoolView &pv, const PlanHeader &h, int32_t 
 bool tensor_path_available();       // false while the tensor-core kernel is compiled out
 // test kernel: a bounded wait that runs out (one warp, PoolView::wait_limit cycles), reported as PASTA_ERR_TIMEOUT
 cudaError_t launch_wait_expiry(const PoolView &pv, cudaStream_t st);
+// measurement kernels: read `bytes` of device memory and do nothing with them (mode 0: vector loads, 1: bulk copies
+// into shared memory, whole 64 KB chunks only, 2: the same with every 8 KB piece taken from a scattered place); sink: 8 bytes of device memory; status: the pool's status word
+cudaError_t launch_stream_read(const void *src, size_t bytes, int mode, void *sink, int32_t *status, int sm_count,
+                               cudaStream_t st);
 // K4: log-sum-exp merge of all partial rows of every (query, head)
 // out: device fp32 [layer_count, n, Hq, D], or bf16 of the same shape when out_bf16
 cudaError_t launch_merge(const PoolView &pv, const PlanHeader &h, int32_t layer_count, void *out, float *lse,
