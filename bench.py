@@ -463,6 +463,77 @@ def measure_steady(args, workload, size, steps, warmup, device, rank, world, loc
     return res
 
 
+def run_dense_mask(args):
+    """The workload in the paper's own layout (paper_2502_11517_b200/dense_mask.py): one dense pool per response filled
+    in decode order, a boolean mask row per thread, every query reading its response's whole pool.  One layer."""
+    import torch
+    from paper_2502_11517_b200.build import build
+    from paper_2502_11517_b200.dense_mask import DensePool
+    build()
+    device = torch.device("cuda", 0); torch.cuda.set_device(device)
+    script = make_script(args.workload, args.size)
+    geo = script.geometry
+    warm = max(args.warmup, 3)
+    entries = [(r, t, 1) for r, t, _n in script.ops[-1][1]]
+    n = len(entries)
+    per_req = {}
+    for op in script.ops[:-1]:
+        if op[0] == "run":
+            per_req[op[1]] = per_req.get(op[1], 0) + op[3]
+    max_slots = max(per_req.values()) + (args.steps + warm + 2) * max(sum(e[0] == r for e in entries) for r in per_req) + 64
+    dp = DensePool(geo.n_q_heads, geo.n_kv_heads, geo.head_dim, max_slots, script.max_threads_per_request, device=device)
+    gen = torch.Generator(device=device); gen.manual_seed(script.seed)
+
+    def randn(shape):
+        return torch.randn(shape, generator=gen, device=device, dtype=torch.float32).to(torch.bfloat16)
+
+    for op in script.ops[:-1]:
+        if op[0] == "begin":
+            dp.begin(op[1])
+        elif op[0] == "spawn":
+            dp.spawn(op[1], op[2])
+        elif op[0] == "run":
+            done = 0
+            while done < op[3]:
+                cnt = min(op[3] - done, 4096)
+                dp.run(op[1], op[2], cnt, randn((cnt, geo.n_kv_heads, geo.head_dim)), randn((cnt, geo.n_kv_heads, geo.head_dim)))
+                done += cnt
+        elif op[0] == "merge":
+            dp.merge(op[1], list(op[2] or []))
+    k_new, v_new = randn((n, geo.n_kv_heads, geo.head_dim)), randn((n, geo.n_kv_heads, geo.head_dim))
+    q = randn((n, geo.n_q_heads, geo.head_dim))
+    out = torch.empty(q.shape, dtype=torch.float32, device=device)
+    for _ in range(warm):
+        dp.step(entries, k_new, v_new, q, out)
+    torch.cuda.synchronize(device)
+    sampler = ClockSampler(0)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0 = time.time(); ev0.record()
+    read = 0
+    for _ in range(args.steps):
+        dp.step(entries, k_new, v_new, q, out)
+        read += dp.bytes_read_last_step
+    ev1.record(); torch.cuda.synchronize(device); sampler.now(); t1 = time.time()
+    ms = ev0.elapsed_time(ev1)
+    clocks = sampler.stop(t0, t1)
+    peak, peak_kind = measured_peak()
+    gbs = read / (ms * 1e-3) / 1e9
+    print(json.dumps({
+        "metric": METRIC, "value": n * args.steps / (ms * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": args.steps,
+        "warmup": warm, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": args.workload, "size": args.size, "layout": "dense_mask", "script": script.name,
+                   "requests": len(per_req), "thread_tokens_per_step": n, "layers": 1,
+                   "bytes_read_per_step": read / args.steps, "l2": "inputs larger than L2",
+                   "note": "every query reads every slot of its response's pool (K, V and a mask byte per slot)"},
+        "clocks": clocks, "e2e": None, "gpu_launches": args.steps * 3 * len(per_req),
+        "roofline": {"bound": "hbm", "kernel": "dense_mask_attn_kernel", "achieved": gbs, "peak": peak, "peak_kind": peak_kind,
+                     "unit": "GB/s", "frac": gbs / peak, "traffic": None,
+                     "note": "bytes the kernel asks for per second (a response's pool is re-read by each of its threads; "
+                             "what of that the L2 serves is not DRAM traffic)"},
+        "cpu_baseline": None}))
+
+
 def summary_of(m, peak):
     """The figures of a secondary workload that go under config.other_workloads."""
     return {"workload": m["script"].name, "thread_tokens_per_step": m["n"], "layers": m["L"], "steps": m["steps"],
@@ -1034,9 +1105,11 @@ def main():
                     help="warp: send every stream through the warp-shuffle kernel (PASTA_FLAG_NO_TENSOR_PATH)")
     ap.add_argument("--out-dtype", default="fp32", choices=["fp32", "bf16"],
                     help="type of the attention output (bf16 halves the device-to-host bytes of the end-to-end path)")
-    ap.add_argument("--layout", default="pool", choices=["pool", "naive_rows"],
+    ap.add_argument("--layout", default="pool", choices=["pool", "naive_rows", "dense_mask"],
                     help="pool: the library's shared paged pool (default).  naive_rows: the comparison layout of the "
-                         "paper's Appendix B (one dense row per thread, prefix duplicated), on the same kernels")
+                         "paper's Appendix B (one dense row per thread, prefix duplicated), on the same kernels.  "
+                         "dense_mask: the paper's own layout (one dense pool per response in decode order, a boolean "
+                         "mask row per thread), one layer, plain CUDA-core kernels")
     ap.add_argument("--size", default="full", choices=["full", "small"],
                     help="small: a reduced copy of the workload for profiler captures (prefix 8192 / 4 layers)")
     args = ap.parse_args()
@@ -1048,6 +1121,8 @@ def main():
         run_trace(args)
     elif args.workload == "extras":
         run_extras(args)
+    elif args.layout == "dense_mask":
+        run_dense_mask(args)
     else:
         run_ours(args)
 

@@ -286,6 +286,34 @@ pasta_status_t pasta_step_host(pasta_pool_t *pool, int32_t n, const int32_t *req
 pasta_status_t pasta_decode_attn_noalloc(pasta_pool_t *pool, int32_t layer, const void *q, void *out,
                                          float *lse, float scale, void *stream);
 
+/* ---- comparison layout: the paper's dense pool with a boolean mask ------------------------------ */
+
+/*
+ * The layout the paper itself describes (Section 3 "Efficiency", Fig. 2b/2c): ONE dense, token-granular pool per
+ * response, filled in decode order so that the tokens of the threads interleave, and a boolean attention mask per
+ * thread over the pool's slots.  Kept here as a measured comparison for the paged pool above (next to the duplicated
+ * rows of Appendix B); these calls own no state: the caller holds the tensors (paper_2502_11517_b200/dense_mask.py).
+ *   k_pool, v_pool  device bf16 [max_slots, n_kv_heads, head_dim], slot = position in decode order
+ *   mask, own       device bytes [n_threads, mask_stride]: mask[t, s] != 0 iff thread t may attend to slot s;
+ *                   own[t, s] != 0 iff thread t decoded slot s (what <sync/> adds to the main thread's row)
+ * pasta_dense_append copies n_new (<= 64) tokens k_new / v_new [n_new, n_kv_heads, head_dim] to slots slot0 ...
+ * and sets mask and own of token i in row rows[i] (host array).  pasta_dense_mask_attn computes, for query i
+ * (q device bf16 [n_queries, n_q_heads, head_dim]; mask_row device int32 [n_queries]: its thread's mask row),
+ * softmax(q K^T scale + (mask ? 0 : -inf)) V over slots [0, n_slots) into out (device fp32 like q) and the
+ * log-sum-exp into lse (optional): every query reads every slot, whatever the mask says, as masked attention over
+ * a dense cache does.  scratch: device, 256-byte aligned, pasta_dense_mask_scratch_bytes() bytes.  head_dim 64 or
+ * 128, n_q_heads / n_kv_heads in {1, 2, 4}.  Errors: INVALID_ARG, CUDA.
+ */
+pasta_status_t pasta_dense_mask_scratch_bytes(int32_t n_queries, int32_t n_slots, int32_t n_q_heads, int32_t n_kv_heads,
+                                              int32_t head_dim, size_t *out);
+pasta_status_t pasta_dense_append(void *k_pool, void *v_pool, uint8_t *mask, uint8_t *own, int64_t mask_stride,
+                                  int32_t slot0, int32_t n_new, const int32_t *rows, const void *k_new,
+                                  const void *v_new, int32_t n_kv_heads, int32_t head_dim, void *stream);
+pasta_status_t pasta_dense_mask_attn(const void *k_pool, const void *v_pool, const uint8_t *mask, int64_t mask_stride,
+                                     const int32_t *mask_row, const void *q, void *out, float *lse, void *scratch,
+                                     size_t scratch_bytes, int32_t n_queries, int32_t n_slots, int32_t n_q_heads,
+                                     int32_t n_kv_heads, int32_t head_dim, float scale, void *stream);
+
 /* ---- introspection ---------------------------------------------------------------------------- */
 
 /*

@@ -29,6 +29,7 @@ EXPORTS = [
     "pasta_kv_append_run_rope", "pasta_step_device",
     "pasta_last_cuda_error", "pasta_debug_set_wait_limit", "pasta_debug_wait_expiry", "pasta_debug_hold_roles",
     "pasta_debug_stream_read", "pasta_step_host_begin", "pasta_step_host_wait",
+    "pasta_dense_mask_scratch_bytes", "pasta_dense_append", "pasta_dense_mask_attn",
 ]
 
 
@@ -356,3 +357,26 @@ class Pool:
         out = C.c_int64()
         _check(lib().pasta_launch_count(self._h, C.byref(out)), "pasta_launch_count")
         return out.value
+
+
+# ---- the stateless calls of the dense-pool comparison layout (tensors are held by dense_mask.DensePool)
+def dense_mask_scratch_bytes(n_queries: int, n_slots: int, n_q_heads: int, n_kv_heads: int, head_dim: int) -> int:
+    out = C.c_size_t()
+    _check(lib().pasta_dense_mask_scratch_bytes(n_queries, n_slots, n_q_heads, n_kv_heads, head_dim, C.byref(out)),
+           "pasta_dense_mask_scratch_bytes")
+    return out.value
+
+
+def dense_append(k_pool, v_pool, mask, own, slot0: int, rows, k_new, v_new, stream=None) -> None:
+    r = _i32(rows)
+    _check(lib().pasta_dense_append(_dev(k_pool), _dev(v_pool), _dev(mask), _dev(own), C.c_int64(mask.shape[1]), slot0,
+                                    len(r), _ptr(r), _dev(k_new), _dev(v_new), k_pool.shape[1], k_pool.shape[2],
+                                    _stream(stream)), "pasta_dense_append")
+
+
+def dense_mask_attn(k_pool, v_pool, mask, mask_row, q, out, lse, scratch, n_slots: int, scale: float = 0.0,
+                    stream=None) -> None:
+    _check(lib().pasta_dense_mask_attn(_dev(k_pool), _dev(v_pool), _dev(mask), C.c_int64(mask.shape[1]), _dev(mask_row),
+                                       _dev(q), _dev(out), _dev(lse), _dev(scratch), C.c_size_t(scratch.numel()),
+                                       q.shape[0], n_slots, q.shape[1], k_pool.shape[1], k_pool.shape[2], C.c_float(scale),
+                                       _stream(stream)), "pasta_dense_mask_attn")

@@ -9,7 +9,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libpasta.so")
-SOURCES = ["pool.cpp", "plan.cpp", "kernels.cu", "attn_tensor.cu", "api.cu", "noalloc.cu"]
+SOURCES = ["pool.cpp", "plan.cpp", "kernels.cu", "attn_tensor.cu", "api.cu", "noalloc.cu", "dense_mask.cu"]
 HEADERS = ["pool.hpp", "plan.hpp", "pasta_plan.h", "device_common.cuh", "kernels.hpp",
            os.path.join("..", "..", "include", "pasta.h")]
 

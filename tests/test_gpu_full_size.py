@@ -120,3 +120,93 @@ def test_batched_full_size():
     assert pool.status() == 0
     print("cfg3 full size: worst max-abs %.2e mean-abs %.2e" % worst)
     pool.close()
+
+
+def test_interpreter_trace_at_size():
+    """cfg5 with its stated statistics (promise probability 0.02, chunks of mean 80, groups of 2 to 6 forks) at
+    64 requests x 8 layers x 128 decode steps.  Indexing (slots of every step, the whole bookkeeping state after every
+    step) must equal the oracle's exactly.  Attention is checked against the oracle in layers 0 and 7: every query of
+    every 32nd step and of the last step, and, in the step that follows a spawn or a merge, every query of the
+    requests that spawned or merged."""
+    import torch
+    from paper_2502_11517_b200 import binding, build
+    from pasta_workloads import cfg5_trace
+    build()
+    script = cfg5_trace(n_requests=64, n_steps=128, n_layers=8)
+    geo = script.geometry
+    layers = [0, geo.n_layers - 1]
+    pool = binding.Pool(geo.n_layers, geo.n_q_heads, geo.n_kv_heads, geo.head_dim, script.n_pages,
+                        script.max_requests, script.max_threads_per_request, script.max_segments_per_thread,
+                        free_order=script.free_order, max_layers_per_launch=geo.n_layers,
+                        max_step_queries=max(len(op[1]) for op in script.ops if op[0] == "step"))
+    model = PoolModel(script.n_pages, geo.page_size, script.free_order, script.max_requests,
+                      script.max_threads_per_request, script.max_segments_per_thread)
+    stores = {l: KVStore(script.n_pages, geo.page_size, geo.n_kv_heads, geo.head_dim) for l in layers}
+    gen = torch.Generator(device="cuda"); gen.manual_seed(5)
+
+    def noise(shape):
+        t = torch.empty(shape, dtype=torch.bfloat16, device="cuda")
+        t.copy_(torch.randn(shape, generator=gen, device="cuda", dtype=torch.float32))
+        return t
+
+    n_steps = sum(op[0] == "step" for op in script.ops)
+    step_no = queries_checked = steps_checked = spawns = merges = 0
+    touched = set()
+    worst = (0.0, 0.0)
+    for i, op in enumerate(script.ops):
+        kind = op[0]
+        if kind == "begin":
+            assert pool.request_begin() == op[1] == model.request_begin()
+        elif kind == "spawn":
+            assert pool.thread_spawn(op[1]) == op[2] == model.thread_spawn(op[1], 0, 0)
+            touched.add(op[1]); spawns += 1
+        elif kind == "finish":
+            pool.thread_finish(op[1], op[2]); model.thread_finish(op[1], op[2])
+        elif kind == "merge":
+            pool.sync_merge(op[1], list(op[2])); model.sync_merge(op[1], list(op[2]))
+            touched.add(op[1]); merges += 1
+        elif kind == "run":
+            m = op[3]
+            slots = model.append_run(op[1], op[2], m)
+            k, v = noise((geo.n_layers, m, geo.n_kv_heads, geo.head_dim)), noise((geo.n_layers, m, geo.n_kv_heads, geo.head_dim))
+            for l in layers:
+                kc, vc = run_tensors(script, i, l)
+                k[l].copy_(kc); v[l].copy_(vc)
+                stores[l].write(slots, kc, vc)
+            pool.kv_append_run(op[1], op[2], m, k, v)
+        elif kind == "step":
+            entries = op[1]
+            n = len(entries)
+            slots = [s for s in model.reserve(entries) if s is not None]
+            k, v = noise((geo.n_layers, n, geo.n_kv_heads, geo.head_dim)), noise((geo.n_layers, n, geo.n_kv_heads, geo.head_dim))
+            q = noise((geo.n_layers, n, geo.n_q_heads, geo.head_dim))
+            q_cpu = {}
+            for l in layers:
+                kc, vc, qc = step_tensors(script, i, l)
+                k[l].copy_(kc); v[l].copy_(vc); q[l].copy_(qc); q_cpu[l] = qc
+                stores[l].write(slots, kc, vc)
+            pool.step_begin([e[0] for e in entries], [e[1] for e in entries], [e[2] for e in entries])
+            assert [(int(s[0]), int(s[1])) for s in pool.step_slots()] == slots, ("slots", step_no)
+            pool.kv_append(k, v)
+            out = torch.empty(q.shape, dtype=torch.float32, device="cuda")
+            lse = torch.empty(q.shape[:3], dtype=torch.float32, device="cuda")
+            pool.decode_attn(q, out, lse)
+            assert pool.dump() == model.dump(), ("bookkeeping", step_no)
+            if step_no % 32 == 0 or step_no == n_steps - 1:
+                sample = list(range(n))
+            else:
+                sample = [j for j, e in enumerate(entries) if e[0] in touched]
+            if sample:
+                w = _check_sample(model, stores, entries, q_cpu, out, lse, sample, layers)
+                worst = (max(worst[0], w[0]), max(worst[1], w[1]))
+                queries_checked += len(sample) * len(layers); steps_checked += 1
+            touched.clear()
+            step_no += 1
+        else:
+            raise AssertionError(kind)
+    assert pool.status() == 0
+    assert step_no == 128 and spawns >= 100 and merges >= 10 and steps_checked >= 60
+    print("cfg5 at size: %d steps, %d spawns, %d merges; attention checked on %d (query, layer) pairs in %d steps, "
+          "worst max-abs %.2e mean-abs %.2e; bookkeeping equal after every step"
+          % (step_no, spawns, merges, queries_checked, steps_checked, worst[0], worst[1]))
+    pool.close()
