@@ -282,13 +282,15 @@ def build_state_naive_rows(script, device, seed_offset=0, grow_tokens=640):
 
 
 def unique_tokens(pool, entries, tensor=True):
-    """Per request, the union of what the step's threads see (a shared prefix counts once); and the part of
-    it that the tensor-core kernel reads: everything, for requests whose stacked query rows fit one MMA tile."""
+    """Tokens of the step, three ways: (a) per request, the union of what the step's threads see (a shared prefix counts
+    once); (b) the part of (a) that the tensor-core kernel reads: everything, for requests whose stacked query rows fit
+    one MMA tile; (c) what the warp-shuffle kernel reads for the other requests: every query's own visible tokens,
+    a shared prefix once per thread that sees it (that kernel shares nothing between queries)."""
     dump = pool.dump()
     by_req = {}
     for req, t, _ in entries:
         by_req.setdefault(req, []).append(t)
-    total = shared = 0
+    total = shared = per_query = 0
     for req, threads in by_req.items():
         seen = {}
         for t in threads:
@@ -298,12 +300,14 @@ def unique_tokens(pool, entries, tensor=True):
             for s, v in vis.items():
                 seen.setdefault(s, []).append(v)
         on_tensor = (tensor and pool.head_dim == 128 and len(threads) * (pool.n_q_heads // pool.n_kv_heads) <= 128
-                     and len(seen) <= 255)
+                     and len(seen) <= 4095)
         for s, vs in seen.items():
             total += max(vs)
             if on_tensor:
                 shared += max(vs)
-    return total, shared
+            else:
+                per_query += sum(vs)
+    return total, shared, per_query
 
 
 def measure_steady(args, workload, size, steps, warmup, device, rank, world, local, *, layout="pool",
@@ -345,7 +349,7 @@ def measure_steady(args, workload, size, steps, warmup, device, rank, world, loc
         step()
     torch.cuda.synchronize(device)
     on_tensor = not (flags & _b.FLAG_NO_TENSOR_PATH)
-    tok0, _ = unique_tokens(pool, entries, on_tensor)
+    tok0, _, _ = unique_tokens(pool, entries, on_tensor)
     launches0 = pool.launch_count()
     if world > 1:
         dist.barrier()
@@ -365,7 +369,7 @@ def measure_steady(args, workload, size, steps, warmup, device, rank, world, loc
     ms = ev0.elapsed_time(ev1)
     clocks = sampler.window(t_wall0, t_wall1) if sampler else None
     launches = pool.launch_count() - launches0
-    tok1, shared1 = unique_tokens(pool, entries, on_tensor)
+    tok1, shared1, warp1 = unique_tokens(pool, entries, on_tensor)
     all_tokens, worst_s = aggregate(float(n * steps), ms * 1e-3)    # every rank runs its own requests
     ms = worst_s * 1e3
 
@@ -381,7 +385,7 @@ def measure_steady(args, workload, size, steps, warmup, device, rank, world, loc
     kernel_ms, kernel_launches = pool.profile_read()
     pool.profile_enable(False)
     prof_clocks = sampler.window(t_prof0, t_prof1) if sampler else None
-    tok2, shared2 = unique_tokens(pool, entries, on_tensor)
+    tok2, shared2, warp2 = unique_tokens(pool, entries, on_tensor)
     assert pool.status() == 0, "a kernel reported an error"
 
     # ---- what a read-only kernel gets on this GPU, same run: the pool's KV memory read by bulk copies and by loads
@@ -443,7 +447,9 @@ def measure_steady(args, workload, size, steps, warmup, device, rank, world, loc
     dom = 0 if kernel_launches[0] else 1                       # tensor-core kernel when the plan has t-units
     prof_tokens = (tok1 + tok2) / 2.0 + n / 2.0
     prof_shared = (shared1 + shared2) / 2.0
-    dom_bytes = (prof_shared if dom == 0 else prof_tokens - prof_shared) * B_tok * L
+    # the warp-shuffle kernel's algorithmic bytes are per query (it is the path for what is not shared): K and V of
+    # every token each of its queries sees; the tensor-core kernel's are the unique tokens of its requests
+    dom_bytes = (prof_shared if dom == 0 else (warp1 + warp2) / 2.0 + n / 2.0) * B_tok * L
     dom_ms = kernel_ms[dom] / max(1, kernel_launches[dom])
     res = {
         "script": script, "geo": geo, "n": n, "L": L, "requests": len(set(reqs.tolist())),

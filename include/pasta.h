@@ -150,8 +150,9 @@ pasta_status_t pasta_sync_merge(pasta_pool_t *pool, int32_t req, int32_t n_threa
  * per-query array of the calls below (q, out, lse, slots, positions) has one row per query, and k_new / v_new
  * one row per appended token in the same order.  The number of queries is bounded by max_step_queries
  * (CAPACITY, nothing reserved).
- * If the bookkeeping succeeds but the step cannot be planned within the pool's capacities, the call
- * returns CAPACITY with the tokens already reserved (the one exception to "unchanged on failure").
+ * If the bookkeeping succeeds but the step cannot be planned within the pool's capacities (partial rows, plan
+ * words), the call returns CAPACITY and takes the reservation back: the pool is as it was, only the previous
+ * step's plan is no longer valid.
  * The plan is uploaded on `stream`; it is used by the pasta_kv_append and pasta_decode_attn calls
  * that follow, for every layer, until the next pasta_step_begin.
  */
@@ -195,7 +196,7 @@ pasta_status_t pasta_kv_append(pasta_pool_t *pool, int32_t layer_begin, int32_t 
  * the scaled scores), may be NULL; scale 0 means 1/sqrt(head_dim).
  * With head_dim 128, the streams a request's threads read are staged into shared memory once per kv
  * head and scored against all those threads' queries on tensor cores (rows that may not see a page are
- * masked), as long as threads x (n_q_heads / n_kv_heads) <= 128 and the request has at most 255 streams;
+ * masked), as long as threads x (n_q_heads / n_kv_heads) <= 128 and the request has at most 4095 streams;
  * other requests and head sizes take a warp-shuffle kernel; a merge kernel combines the partial results
  * (fp32 throughout).
  */

@@ -48,7 +48,7 @@ pasta_status_t derive(const pasta_pool_config_t &c, Derived *d) {
   const int64_t nq = d->max_queries, nr = c.max_requests;
   d->max_words = PH_WORDS + 2 * nq + PQ_WORDS * nq + PT_WORDS * nr + 2 * nr * c.n_kv_heads +
                  PU_WORDS * (nr * c.n_kv_heads + grid) + 2 * grid + PW_WORDS * (int64_t(d->max_rows) / d->group + 1) +
-                 2 * int64_t(c.n_pages) + nq * std::min(255, c.max_threads_per_request) + nq + 64;
+                 2 * int64_t(c.n_pages) + nq * std::min(PASTA_MAX_STREAMS, c.max_threads_per_request) + nq + 64;
   d->staging_words = std::max<int64_t>(d->max_words, 2 * kRunChunk);
   d->layer_stride = size_t(c.n_pages) * c.n_kv_heads * kv_block_bytes(c.head_dim);
   d->kv_bytes = d->layer_stride * c.n_layers;
@@ -355,13 +355,19 @@ pasta_status_t pasta_step_begin(pasta_pool_t *p, int32_t n, const int32_t *req_i
   if (n_queries > p->d.max_queries) return PASTA_ERR_CAPACITY;
   std::vector<Slot> slots;
   std::vector<StepQuery> queries;
-  pasta_status_t s = p->host.reserve_step(entries, &queries, &slots);
+  std::vector<StepUndo> undo;
+  pasta_status_t s = p->host.reserve_step(entries, &queries, &slots, &undo);
   if (s != PASTA_OK) return s;
   p->plan_valid = false;
   p->queries.swap(queries);
   p->slots.swap(slots);
   s = build_plan(p->host, p->queries, p->slots, limits_of(p), &p->plan);
-  if (s != PASTA_OK) return s;   // the tokens stay reserved; only the attention of this step cannot be planned
+  if (s != PASTA_OK) {           // the step does not fit the pool's capacities: take the reservation back
+    p->host.undo_step(undo);
+    p->queries.clear();
+    p->slots.clear();
+    return s;
+  }
   std::memcpy(p->hdr.w, p->plan.data(), sizeof(p->hdr.w));
   if (!p->host_only) {
     // Buffer b = i % 2 was last read by the kernels of step i - 2.  Everything the caller had enqueued when step

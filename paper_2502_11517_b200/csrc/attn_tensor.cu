@@ -454,12 +454,12 @@ attn_tensor_kernel(PoolView pv, TensorArgs a, const __nv_bfloat16 *__restrict__ 
           const bool no_mask = (m4.x | m4.y | m4.z | m4.w) >= 0 && ((m4.x & m4.y & m4.z & m4.w) & PASTA_PMETA_ALL_VISIBLE);
           if (warp_active && !no_mask) {
             const int base_meta = m4.x & ~PASTA_PMETA_ALL_VISIBLE;
-            const bool run = m4.x >= 0 && m4.w >= 0 && (m4.y & ~PASTA_PMETA_ALL_VISIBLE) == base_meta + (1 << 8) &&
-                             (m4.z & ~PASTA_PMETA_ALL_VISIBLE) == base_meta + (2 << 8) &&
-                             (m4.w & ~PASTA_PMETA_ALL_VISIBLE) == base_meta + (3 << 8);
+            const bool run = m4.x >= 0 && m4.w >= 0 && (m4.y & ~PASTA_PMETA_ALL_VISIBLE) == base_meta + (1 << PASTA_PMETA_STREAM_BITS) &&
+                             (m4.z & ~PASTA_PMETA_ALL_VISIBLE) == base_meta + (2 << PASTA_PMETA_STREAM_BITS) &&
+                             (m4.w & ~PASTA_PMETA_ALL_VISIBLE) == base_meta + (3 << PASTA_PMETA_STREAM_BITS);
             if (run) {
               // four consecutive pages of one stream (the usual case): one look-up of the row's visible length
-              const int sl = base_meta & 255;
+              const int sl = PASTA_PMETA_STREAM(base_meta);
               int vis;
               if (sl < 4) vis = sl == 0 ? vis0 : sl == 1 ? vis1 : sl == 2 ? vis2 : vis3;
               else vis = visrow[sl];
@@ -474,7 +474,7 @@ attn_tensor_kernel(PoolView pv, TensorArgs a, const __nv_bfloat16 *__restrict__ 
                 const int meta = metas[pg];
                 int t = 0;
                 if (active && meta >= 0) {
-                  const int sl = meta & 255;
+                  const int sl = PASTA_PMETA_STREAM(meta);
                   int vis;
                   if (sl < 4) vis = sl == 0 ? vis0 : sl == 1 ? vis1 : sl == 2 ? vis2 : vis3;
                   else vis = visrow[sl];

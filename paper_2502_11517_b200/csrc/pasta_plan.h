@@ -7,7 +7,7 @@
 //   stream     one page list: a request's main-thread tokens (id 0) or one fork's chunk (id = fork id).
 //              Every thread sees a PREFIX [0, vis) of every stream (vis may be 0).
 //   t-request  a request served by the tensor-core kernel: head_dim 128, its queries times `group` fit
-//              PASTA_MAX_ROWS rows, at most 255 streams.  The pages of every stream its queries read (the prefix
+//              PASTA_MAX_ROWS rows, at most PASTA_MAX_STREAMS streams.  The pages of every stream its queries read (the prefix
 //              they share and each fork's own chunk alike) are concatenated into one page list that is cut into
 //              tiles of PASTA_TILE_PAGES pages; rows of the score matrix are the request's queries
 //              times the `group` query heads of one kv head: row = t_idx * group + h_local.
@@ -24,10 +24,14 @@
 #define PASTA_TILE_PAGES 8          // pages per tensor-core tile (128 tokens)
 #define PASTA_PAGE 16               // tokens per page
 #define PASTA_MAX_ROWS 128          // rows of the stacked-query matrix (threads * group)
-// a page's meta word: bits 0-7 local stream, bits 8-29 page index within the stream, bit 30 set when every thread
+// a page's meta word: bits 0-11 local stream, bits 12-29 page index within the stream, bit 30 set when every thread
 // of the t-request sees the whole page (no row needs a mask there); -1 marks an unused slot of a tile
+#define PASTA_PMETA_STREAM_BITS 12
+#define PASTA_MAX_STREAMS ((1 << PASTA_PMETA_STREAM_BITS) - 1)      // streams one t-request may read
+#define PASTA_MAX_STREAM_PAGES (1 << 18)                             // pages of one stream (4 M tokens)
 #define PASTA_PMETA_ALL_VISIBLE (1 << 30)
-#define PASTA_PMETA_PAGE(meta) (((meta) >> 8) & 0x3FFFFF)
+#define PASTA_PMETA_STREAM(meta) ((meta) & PASTA_MAX_STREAMS)
+#define PASTA_PMETA_PAGE(meta) (((meta) >> PASTA_PMETA_STREAM_BITS) & (PASTA_MAX_STREAM_PAGES - 1))
 
 // header words
 enum {
@@ -48,7 +52,7 @@ enum {
   PH_OFF_TCTA,        // per CTA: first t-unit, one past the last
   PH_OFF_WUNIT,       // PW_WORDS per w-unit
   PH_OFF_PAGES,       // page ids
-  PH_OFF_PMETA,       // parallel to pages (t-request lists only): (page index in its stream << 8) | local stream
+  PH_OFF_PMETA,       // parallel to pages (t-request lists only): (page index in its stream << 12) | local stream
   PH_OFF_VIS,         // per t-request: [n_threads][n_streams] visible length of local stream for thread
   PH_OFF_TQ,          // per t-request: [n_threads] query index of each row-thread
   PH_OFF_APOS,        // position id of every appended token (parallel to the append table)

@@ -104,9 +104,10 @@ pasta_status_t build_plan(const HostPool &pool, const std::vector<StepQuery> &en
     bool tensor = lim.tensor_path && T >= 1 && T * G <= PASTA_MAX_ROWS;
     int32_t n_shared = 0;
     if (tensor) {
+      bool too_long = false;                 // a page's meta word has 18 bits for its index within the stream
       for (StreamUse &u : uses)
-        if (u.n_seen >= 1) u.local = n_shared++;
-      if (n_shared == 0 || n_shared > 255) {
+        if (u.n_seen >= 1) { u.local = n_shared++; too_long = too_long || (u.max_vis + P - 1) / P > PASTA_MAX_STREAM_PAGES; }
+      if (n_shared == 0 || n_shared > PASTA_MAX_STREAMS || too_long) {
         tensor = false;
         for (StreamUse &u : uses) u.local = -1;
       }
@@ -130,8 +131,8 @@ pasta_status_t build_plan(const HostPool &pool, const std::vector<StepQuery> &en
         pmeta.resize(m0 + np);
         int32_t *pm = pmeta.data() + m0;
         const int32_t n_all = std::min(np, min_vis / P);     // pages every thread of the request sees in full
-        for (int32_t k = 0; k < n_all; ++k) pm[k] = (k << 8) | u.local | PASTA_PMETA_ALL_VISIBLE;
-        for (int32_t k = n_all; k < np; ++k) pm[k] = (k << 8) | u.local;
+        for (int32_t k = 0; k < n_all; ++k) pm[k] = (k << PASTA_PMETA_STREAM_BITS) | u.local | PASTA_PMETA_ALL_VISIBLE;
+        for (int32_t k = n_all; k < np; ++k) pm[k] = (k << PASTA_PMETA_STREAM_BITS) | u.local;
       }
       t.n_pages = static_cast<int32_t>(pages.size()) - t.page_off;
       for (int32_t ti = 0; ti < T; ++ti) {

@@ -123,8 +123,24 @@ Slot HostPool::append_one(Request &r, int32_t thread) {
   return slot;
 }
 
+void HostPool::undo_step(const std::vector<StepUndo> &undo) {
+  for (auto it = undo.rbegin(); it != undo.rend(); ++it) {
+    Request &r = requests_[it->req];
+    Stream &s = r.streams[it->thread];
+    while (static_cast<int32_t>(s.pages.size()) > it->n_pages) {     // last taken, first back: the old order returns
+      free_.push_front(s.pages.back());
+      s.pages.pop_back();
+    }
+    s.len = it->len;
+    Thread &th = r.threads[it->thread];
+    th.view.resize(it->view_size);
+    if (it->view_size > 0) th.view.back().len = it->last_len;
+    th.pos_next = it->pos_next; th.pos_last = it->pos_last; th.pos_skip = it->pos_skip;
+  }
+}
+
 pasta_status_t HostPool::reserve_step(const std::vector<StepEntry> &entries, std::vector<StepQuery> *queries,
-                                      std::vector<Slot> *slots) {
+                                      std::vector<Slot> *slots, std::vector<StepUndo> *undo) {
   // pass 1: validate everything, count pages
   size_t need = 0;
   std::vector<std::pair<int32_t, int32_t>> seen;
@@ -167,8 +183,15 @@ pasta_status_t HostPool::reserve_step(const std::vector<StepEntry> &entries, std
   // pass 2: commit
   slots->clear();
   queries->clear();
+  if (undo) undo->clear();
   for (const StepEntry &e : entries) {
     Request &r = requests_[e.req];
+    if (undo && e.n_new > 0) {
+      const Thread &th = r.threads[e.thread];
+      undo->push_back(StepUndo{e.req, e.thread, r.streams[e.thread].len, static_cast<int32_t>(r.streams[e.thread].pages.size()),
+                               static_cast<int32_t>(th.view.size()), th.view.empty() ? 0 : th.view.back().len,
+                               th.pos_next, th.pos_last, th.pos_skip});
+    }
     if (e.n_new == 0) {
       slots->push_back(Slot{-1, -1, query_position(r.threads[e.thread])});
       queries->push_back(StepQuery{e.req, e.thread, 0});

@@ -54,6 +54,11 @@ struct StepQuery {
   int32_t req, thread, hide;
 };
 
+// What reserve_step changed for one appending entry, so that the step can be taken back when it cannot be planned.
+struct StepUndo {
+  int32_t req, thread, len, n_pages, view_size, last_len, pos_next, pos_last, pos_skip;
+};
+
 struct Slot {
   int32_t page, offset;   // {-1, -1} for a query without a new token
   int32_t pos;            // position id of the query's token
@@ -79,7 +84,10 @@ class HostPool {
   // Validates the whole step first, then reserves.  Outputs one element per QUERY, in entry order (an entry with
   // n_new tokens contributes max(1, n_new) of them).
   pasta_status_t reserve_step(const std::vector<StepEntry> &entries, std::vector<StepQuery> *queries,
-                              std::vector<Slot> *slots);
+                              std::vector<Slot> *slots, std::vector<StepUndo> *undo = nullptr);
+  // Takes a reserve_step back: lengths, page lists, views and position counters as they were, the pages back at
+  // the front of the free sequence in the order they had.
+  void undo_step(const std::vector<StepUndo> &undo);
   pasta_status_t reserve_run(int32_t req, int32_t thread, int32_t m, std::vector<Slot> *slots);
 
   const Request *request(int32_t req) const;

@@ -44,7 +44,7 @@ def run_plan(w, K, V, q, n_kv_heads):
                 s_all, v_all = [], []
                 for pi in range(tb * TILE_PAGES, min(te * TILE_PAGES, n_pages)):
                     page, meta = pages[page_off + pi], pmeta[page_off + pi]
-                    thr = vis[ti, meta & 255] - ((meta >> 8) & 0x3FFFFF) * PAGE
+                    thr = vis[ti, meta & 4095] - ((meta >> 12) & 0x3FFFF) * PAGE
                     cnt = int(np.clip(thr, 0, PAGE))
                     if meta & (1 << 30):        # the plan claims that no row needs a mask on this page
                         assert cnt == PAGE, (u, ti, pi)

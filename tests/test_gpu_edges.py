@@ -82,14 +82,27 @@ def test_group_sizes(lib, hq, hkv, d):
     run_script(lib, manual(ops, geo))
 
 
-def test_more_streams_than_the_tensor_path_takes(lib):
+def test_a_main_thread_that_merged_hundreds_of_chunks_stays_on_the_tensor_path(lib):
+    """A long response: 300 chunks merged into the main thread, two forks still decoding.  The request reads 303 streams;
+    it must keep its tensor-core units (the prefix staged once for its three threads), not fall back to one warp per
+    query and stream."""
     geo = Geometry(1, 8, 2, 128, 16)
-    n = 260
+    n = 300
     ops = [("begin", 0), ("run", 0, 0, 50)]
     for t in range(1, n + 1):
         ops += [("spawn", 0, t), ("run", 0, t, 1 + t % 3), ("finish", 0, t)]
-    ops += [("merge", 0, None), ("step", ((0, 0, 1),))]        # the main thread now reads 261 streams
-    run_script(lib, manual(ops, geo, n_pages=400, max_threads=n + 2, max_segments=2 * n + 4))
+    ops += [("merge", 0, None), ("run", 0, 0, 200), ("spawn", 0, n + 1), ("spawn", 0, n + 2), ("run", 0, n + 1, 21),
+            ("step", ((0, 0, 1), (0, n + 1, 1), (0, n + 2, 1)))]
+    script = manual(ops, geo, n_pages=500, max_threads=n + 4, max_segments=2 * n + 8)
+    from lib_replay import LibReplay, make_pool
+    pool = make_pool(script, host_only=True)
+    rep = LibReplay(script, pool)
+    for i in range(len(script.ops)):
+        rep.apply(i)
+    w = pool.plan_words()
+    assert w[4] > 0 and w[5] == 0                              # t-units only, no w-units
+    pool.close()
+    run_script(lib, script)
 
 
 def test_fork_spawned_before_any_token(lib):

@@ -205,3 +205,34 @@ def test_pending_spawn_matches_oracle(seed):
         elif what == 4:
             both("kv_append_run", "append_run", req, 0, int(rng.integers(0, 3)))
     pool.close()
+
+
+def test_a_step_that_cannot_be_planned_leaves_the_pool_unchanged():
+    """max_partial_rows too small for the step's partial results: pasta_step_begin returns CAPACITY and takes the
+    reservation back (lengths, page lists, free order, views, position ids), so the caller can go on with a smaller
+    step; the oracle's model, which never saw the failed step, stays equal to the pool."""
+    from oracle import PoolModel
+    build()
+    order = np.random.default_rng(3).permutation(64).astype(np.int32)
+    pool = binding.Pool(1, 8, 2, 128, 64, 2, 6, 12, free_order=order, flags=binding.FLAG_HOST_ONLY, max_partial_rows=40,
+                        max_step_queries=8)
+    model = PoolModel(64, 16, order, 2, 6, 12)
+    assert pool.request_begin() == model.request_begin() == 0
+    pool.kv_append_run(0, 0, 16); model.append_run(0, 0, 16)        # the next main-thread token opens a page
+    for _ in range(4):
+        assert pool.thread_spawn_predicted(0, 7) == model.thread_spawn(0, 7)
+    pool.kv_append_run(0, 1, 15); model.append_run(0, 1, 15)
+    before = pool.dump()
+    assert before == model.dump()
+    entries = [(0, 0, 1), (0, 1, 2), (0, 2, 1), (0, 3, 1), (0, 4, 1)]      # 6 queries x 4 heads x 2 kv heads = 48 partial rows > 40
+    with pytest.raises(binding.PastaError) as e:
+        pool.step_begin([x[0] for x in entries], [x[1] for x in entries], [x[2] for x in entries])
+    assert e.value.code == binding.CAPACITY
+    assert pool.dump() == before
+    small = [(0, 1, 2), (0, 0, 1)]                                   # 3 queries, 24 partial rows: fits
+    pool.step_begin([x[0] for x in small], [x[1] for x in small], [x[2] for x in small])
+    want_slots = model.reserve(small)
+    assert [(int(a), int(b)) for a, b in pool.step_slots()] == want_slots
+    assert pool.dump() == model.dump()
+    assert list(pool.step_positions()) == [model.last_position(0, 1) - 1, model.last_position(0, 1), model.last_position(0, 0)]
+    pool.close()
