@@ -330,6 +330,8 @@ def measure_steady(args, workload, size, steps, warmup, device, rank, world, loc
     else:
         pool, entries, randn = build_state(script, device, seed_offset=rank, grow_tokens=grow,
                                            flags=flags | (_b.FLAG_OUT_BF16 if out_dtype_name == "bf16" else 0))
+    if getattr(args, "tail", None):
+        pool.debug_set_tail(*[int(v) for v in args.tail.split(",")])
     n = len(entries)
     reqs = np.asarray([e[0] for e in entries], dtype=np.int32); thr = np.asarray([e[1] for e in entries], dtype=np.int32)
     ones = np.ones(n, dtype=np.int32)
@@ -1109,6 +1111,9 @@ def main():
                     help="skip the shorter runs of the other configurations that ride along with the default workload")
     ap.add_argument("--kernel", default="auto", choices=["auto", "warp"],
                     help="warp: send every stream through the warp-shuffle kernel (PASTA_FLAG_NO_TENSOR_PATH)")
+    ap.add_argument("--tail", default=None, metavar="PERCENT,TILES",
+                    help="share of the short runs' tiles that the tensor-core kernel's CTAs share out at run time, and the "
+                         "tiles per shared unit (pasta_debug_set_tail; the library's default when not given)")
     ap.add_argument("--out-dtype", default="fp32", choices=["fp32", "bf16"],
                     help="type of the attention output (bf16 halves the device-to-host bytes of the end-to-end path)")
     ap.add_argument("--layout", default="pool", choices=["pool", "naive_rows", "dense_mask"],

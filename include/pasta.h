@@ -365,6 +365,15 @@ pasta_status_t pasta_debug_set_wait_limit(pasta_pool_t *pool, int64_t cycles);
  */
 pasta_status_t pasta_debug_hold_roles(pasta_pool_t *pool, int32_t role_mask);
 /*
+ * Tuning hook (no counterpart in the paper).  The tensor-core kernel assigns the tiles of a step to its CTAs in
+ * advance, except that of the short (request, kv head) runs, those of at most 4 x `tiles` tiles, every so often a whole
+ * one is kept back, `percent` of their tiles in all (0 to 50; 10 by default), in units of at most `tiles` tiles (2 to
+ * 1024; 16 by default).  The CTAs take these from a shared counter once their own work is done: SMs that stream faster
+ * than others then do more of it.  0 percent assigns everything in advance.  Takes effect from the next
+ * pasta_step_begin, and only for steps large enough for it to matter (16 tiles per CTA).
+ */
+pasta_status_t pasta_debug_set_tail(pasta_pool_t *pool, int32_t percent, int32_t tiles);
+/*
  * Measurement aid (no counterpart in the paper): enqueues a kernel that reads `bytes` of device memory at `src`
  * (16-byte aligned; NULL = the pool's own KV memory, all of it) and does nothing with them, so that a benchmark can
  * time what a read-only kernel is given on this GPU next to the attention kernel.  mode 0: plain 16-byte loads;

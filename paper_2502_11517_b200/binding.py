@@ -29,7 +29,7 @@ EXPORTS = [
     "pasta_kv_append_run_rope", "pasta_step_device",
     "pasta_last_cuda_error", "pasta_debug_set_wait_limit", "pasta_debug_wait_expiry", "pasta_debug_hold_roles",
     "pasta_debug_stream_read", "pasta_step_host_begin", "pasta_step_host_wait",
-    "pasta_dense_mask_scratch_bytes", "pasta_dense_append", "pasta_dense_mask_attn",
+    "pasta_dense_mask_scratch_bytes", "pasta_dense_append", "pasta_dense_mask_attn", "pasta_debug_set_tail",
 ]
 
 
@@ -346,6 +346,9 @@ class Pool:
 
     def debug_set_wait_limit(self, cycles: int) -> None:
         _check(lib().pasta_debug_set_wait_limit(self._h, C.c_int64(cycles)), "pasta_debug_set_wait_limit")
+
+    def debug_set_tail(self, percent: int, tiles: int) -> None:
+        _check(lib().pasta_debug_set_tail(self._h, percent, tiles), "pasta_debug_set_tail")
 
     def debug_hold_roles(self, role_mask: int) -> None:
         _check(lib().pasta_debug_hold_roles(self._h, role_mask), "pasta_debug_hold_roles")

@@ -18,6 +18,8 @@ constexpr int kStaging = 4;           // pinned upload buffers in rotation
 constexpr size_t kSmallPlanWords = 2048;   // plans up to this size are uploaded in the caller's stream
 constexpr int kProfCalls = 512;        // timed pasta_decode_attn launches kept between two profile reads
 constexpr int kRunChunk = 8192;       // tokens whose slots are uploaded at once by pasta_kv_append_run
+constexpr int kTailPercent = 10;      // share of the short runs' tiles that the tensor-core kernel's CTAs share out at run time
+constexpr int kTailTiles = 16;        // tiles per unit of that share; runs of up to four times as many count as short
 int32_t g_last_cuda_error = 0;
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -40,15 +42,21 @@ pasta_status_t derive(const pasta_pool_config_t &c, Derived *d) {
   const int grid = 160;   // upper bound on CTAs of the tensor-core kernel, for sizing only
   d->max_queries = c.max_step_queries ? c.max_step_queries
                                       : static_cast<int32_t>(std::min<int64_t>(int64_t(c.max_requests) * 17, 1 << 20));
+  // units of the shared tail, at most: its share of all tiles in pieces of kTailTiles, plus one ragged piece per run
+  const int64_t tail_units = int64_t(c.n_pages) * c.n_kv_heads / PASTA_TILE_PAGES * kTailPercent / 100 / kTailTiles +
+                             int64_t(c.max_requests) * c.n_kv_heads;
+  const int64_t unit_rows = std::min<int64_t>(PASTA_MAX_ROWS, int64_t(c.max_threads_per_request) * d->group);
   d->max_rows = c.max_partial_rows ? c.max_partial_rows
                                    : static_cast<int32_t>(std::min<int64_t>(
-                                         int64_t(d->max_queries) * c.n_q_heads * 8 + int64_t(grid) * PASTA_MAX_ROWS, 1 << 28));
+                                         int64_t(d->max_queries) * c.n_q_heads * 8 + int64_t(grid) * PASTA_MAX_ROWS +
+                                             tail_units * unit_rows, 1 << 28));
   d->layers_per_launch = c.max_layers_per_launch ? std::min(c.max_layers_per_launch, c.n_layers)
                                                  : std::min(c.n_layers, 8);
   const int64_t nq = d->max_queries, nr = c.max_requests;
   d->max_words = PH_WORDS + 2 * nq + PQ_WORDS * nq + PT_WORDS * nr + 2 * nr * c.n_kv_heads +
                  PU_WORDS * (nr * c.n_kv_heads + grid) + 2 * grid + PW_WORDS * (int64_t(d->max_rows) / d->group + 1) +
-                 2 * int64_t(c.n_pages) + nq * std::min(PASTA_MAX_STREAMS, c.max_threads_per_request) + nq + 64;
+                 2 * int64_t(c.n_pages) + nq * std::min(PASTA_MAX_STREAMS, c.max_threads_per_request) + nq + 64 +
+                 PU_WORDS * tail_units + 2 * nr * c.n_kv_heads + 8;
   d->staging_words = std::max<int64_t>(d->max_words, 2 * kRunChunk);
   d->layer_stride = size_t(c.n_pages) * c.n_kv_heads * kv_block_bytes(c.head_dim);
   d->kv_bytes = d->layer_stride * c.n_layers;
@@ -90,6 +98,7 @@ struct pasta_pool {
   cudaEvent_t plan_ready[2] = {nullptr, nullptr};   // recorded on copy_stream after the upload of buffer b
   cudaEvent_t work_mark[2] = {nullptr, nullptr};    // recorded on the caller's stream at the start of step i (slot i % 2)
   int64_t step_index = 0;
+  int32_t tail_percent = kTailPercent, tail_tiles = kTailTiles;
   // pasta_step_host_begin / _wait: at most two steps in flight; their copies run on streams of the pool
   cudaStream_t d2h_stream = nullptr;
   cudaEvent_t host_inputs_ready[2] = {nullptr, nullptr};   // copy_stream: k / v / q of the step are on the device
@@ -145,6 +154,8 @@ PlanLimits limits_of(const pasta_pool *p) {
   l.max_words = p->d.max_words;
   l.grid = p->sm_count;
   l.tensor_path = p->cfg.head_dim == 128 && !(p->cfg.flags & PASTA_FLAG_NO_TENSOR_PATH) && tensor_path_available();
+  l.tail_percent = p->tail_percent;
+  l.tail_tiles = p->tail_tiles;
   return l;
 }
 
@@ -440,7 +451,7 @@ pasta_status_t pasta_decode_attn(pasta_pool_t *p, int32_t layer_begin, int32_t l
     cudaEvent_t *ev = timed ? &p->prof_events[4 * p->prof_calls] : nullptr;
     uint8_t mask = 0;
     if (timed) PASTA_CUDA(cudaEventRecord(ev[0], st));
-    if (p->hdr.w[PH_N_TUNITS] > 0) {
+    if (p->hdr.w[PH_N_TUNITS] + p->hdr.w[PH_N_DUNITS] > 0) {
       PASTA_CUDA(launch_attn_tensor(p->pv, p->hdr, layer_begin + done, cnt, qg, sc, st));
       p->launches += 1;
       mask |= 1;
@@ -721,6 +732,13 @@ pasta_status_t pasta_debug_stream_read(pasta_pool_t *p, const void *src, size_t 
   void *sink = reinterpret_cast<uint8_t *>(p->pv.status) + 64;      // inside the 256 status bytes of the workspace
   PASTA_CUDA(launch_stream_read(src, bytes, mode, sink, p->pv.status, p->sm_count, static_cast<cudaStream_t>(stream)));
   p->launches += 1;
+  return PASTA_OK;
+}
+
+pasta_status_t pasta_debug_set_tail(pasta_pool_t *p, int32_t percent, int32_t tiles) {
+  if (!p || percent < 0 || percent > 50 || tiles < 2 || tiles > 1024) return PASTA_ERR_INVALID_ARG;
+  p->tail_percent = percent;
+  p->tail_tiles = tiles;
   return PASTA_OK;
 }
 

@@ -48,8 +48,9 @@ constexpr int B_FULL = 0, B_EMPTY = B_FULL + T_STAGES, B_SFULL = B_EMPTY + T_STA
               B_DRAIN = B_MLFULL + 1,  // only used when a role gave up: completion of the MMAs still in flight
               B_COUNT = B_DRAIN + 1;
 constexpr int OFF_META = OFF_BAR + 8 * ((B_COUNT + 1) & ~1);   // per stage: 8 page metas
-constexpr int OFF_MISC = OFF_META + T_STAGES * 32;             // tmem base, abort flag
-constexpr int OFF_ML1 = OFF_MISC + 16;                         // (m_ref, l) of group 1's rows, for the epilogue
+constexpr int T_RING = 16;                                     // shared units the producer may be ahead of the slowest role
+constexpr int OFF_MISC = OFF_META + T_STAGES * 32;             // tmem base, abort flag, shared units taken, their ids
+constexpr int OFF_ML1 = OFF_MISC + 16 + 4 * T_RING;            // (m_ref, l) of group 1's rows, for the epilogue
 constexpr int T_SMEM_USED = OFF_ML1 + 128 * 8;
 constexpr int T_SMEM_BYTES = T_SMEM_USED + 1024;               // slack to align the base to 1024
 static_assert(T_SMEM_BYTES <= 232448, "shared memory budget");
@@ -227,9 +228,64 @@ __device__ __forceinline__ UnitInfo load_unit(const int32_t *plan, int off_tunit
 
 struct TensorArgs {
   int32_t off_tunit, off_treq, off_tcta, off_pages, off_pmeta, off_vis, off_tq;
+  int32_t off_dunit, n_dunits;      // units no CTA owns in advance (per layer): taken from a counter at run time
   int32_t n_queries, layer_begin, layer_count;
   float scale_log2;
 };
+
+// A role's place in its CTA's sequence of units: first the units assigned to the CTA, layer by layer, then units of the
+// shared pool (the last tiles of the runs, kept back by the planner).  The producer takes the next shared unit from a
+// counter in global memory when it gets there, which is ahead of every other role, and publishes its number in a small
+// ring in shared memory; the other roles read the same numbers in the same order.  -1 ends the sequence.
+struct Walk { int ll, u, k; };
+
+template <bool kProducer>
+__device__ __forceinline__ bool next_unit(Walk &w, const TensorArgs &a, const int32_t *plan, int u0, int u1, volatile int *ring,
+                                          int32_t *counter, int lane, bool whole_warp, volatile int *abort_flag,
+                                          long long limit, bool &ok, UnitInfo &x, int &ll) {
+  if (u0 < u1 && w.ll < a.layer_count) {
+    x = load_unit(plan, a.off_tunit, 0, w.u);
+    ll = w.ll;
+    if (++w.u == u1) { w.u = u0; ++w.ll; }
+    return true;
+  }
+  const int total = a.n_dunits * a.layer_count;
+  if (total == 0) return false;
+  int id = -1;
+  if (kProducer) {
+    if (lane == 0) {
+      id = atomicAdd(counter, 1);
+      if (id >= total) id = -1;
+      ring[2 + w.k % T_RING] = id;
+      __threadfence_block();
+      ring[0] = w.k + 1;
+    }
+    id = __shfl_sync(0xffffffffu, id, 0);
+  } else {
+    int got = 1;
+    if (!whole_warp || lane == 0) {
+      if (ring[0] <= w.k) {
+        const long long t0 = clock64();
+        while (ring[0] <= w.k) {
+          if (*abort_flag) { got = 0; break; }
+          if (clock64() - t0 > limit) { *abort_flag = 1; got = 0; break; }
+          __nanosleep(128);
+        }
+      }
+    }
+    if (whole_warp) {
+      got = __shfl_sync(0xffffffffu, got, 0);
+      __syncwarp();
+    }
+    if (!got) { ok = false; return false; }
+    id = ring[2 + w.k % T_RING];
+  }
+  ++w.k;
+  if (id < 0) return false;
+  ll = id / a.n_dunits;
+  x = load_unit(plan, a.off_dunit, 0, id - ll * a.n_dunits);
+  return true;
+}
 
 __global__ void __launch_bounds__(T_THREADS, 1)
 attn_tensor_kernel(PoolView pv, TensorArgs a, const __nv_bfloat16 *__restrict__ q) {
@@ -263,6 +319,7 @@ attn_tensor_kernel(PoolView pv, TensorArgs a, const __nv_bfloat16 *__restrict__ 
     mbar_init(bar + 8 * B_MLFULL, 4);
     mbar_init(bar + 8 * B_DRAIN, 1);
     misc[1] = 0;
+    misc[2] = 0;
     mbar_init_fence();
   }
   fence_proxy_async();
@@ -277,6 +334,8 @@ attn_tensor_kernel(PoolView pv, TensorArgs a, const __nv_bfloat16 *__restrict__ 
   const uint32_t tmem = misc[0];
   const long long limit = pv.wait_limit;
   uint32_t prod_it = 0;       // warp 0: tiles whose copies have been issued
+  volatile int *ring = reinterpret_cast<volatile int *>(misc + 2);
+  int32_t *counter = pv.status + PASTA_STATUS_TAIL_COUNTER;
 
   // test hook: a held role goes straight to the tear-down, so that the roles waiting for it run into their limits
   const int role = warp == 0 ? 0 : warp == 1 ? 1 : warp < 4 ? 2 : 3 + ((warp - 4) >> 2);
@@ -287,10 +346,12 @@ attn_tensor_kernel(PoolView pv, TensorArgs a, const __nv_bfloat16 *__restrict__ 
     bool ok = true;
     uint64_t policy;
     asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
-    for (int ll = 0; ll < a.layer_count && ok; ++ll) {
-      const uint8_t *kv_layer = pv.kv_base + (a.layer_begin + ll) * pv.layer_stride;
-      for (int u = u0; u < u1 && ok; ++u) {
-        const UnitInfo x = load_unit(plan, a.off_tunit, a.off_treq, u);
+    {
+      Walk wk{0, u0, 0};
+      UnitInfo x;
+      int ll = 0;
+      while (ok && next_unit<true>(wk, a, plan, u0, u1, ring, counter, lane, true, abort_flag, limit, ok, x, ll)) {
+        const uint8_t *kv_layer = pv.kv_base + (a.layer_begin + ll) * pv.layer_stride;
         for (int tile = x.tile_begin; tile < x.tile_end; ++tile, ++it) {
           const int s = it % T_STAGES;
           if (!warp_wait_or_abort(bar + 8 * (B_EMPTY + s), ((it / T_STAGES) & 1) ^ 1, abort_flag, limit)) { ok = false; break; }
@@ -327,9 +388,11 @@ attn_tensor_kernel(PoolView pv, TensorArgs a, const __nv_bfloat16 *__restrict__ 
       uint32_t it = 0, uc = 0;
       bool ok = true;
       const uint32_t q_addr = base + OFF_Q;
-      for (int ll = 0; ll < a.layer_count && ok; ++ll) {
-        for (int u = u0; u < u1 && ok; ++u, ++uc) {
-          const UnitInfo x = load_unit(plan, a.off_tunit, a.off_treq, u);
+      {
+        Walk wk{0, u0, 0};
+        UnitInfo x;
+        int ll = 0;
+        for (; ok && next_unit<false>(wk, a, plan, u0, u1, ring, counter, lane, false, abort_flag, limit, ok, x, ll); ++uc) {
           const int nt = x.tile_end - x.tile_begin;
           const uint32_t m_bits = x.n_threads * G <= T_M64_ROWS ? IDESC_M64 : IDESC_M128;
           if (!wait_or_abort(bar + 8 * B_QFULL, uc & 1, abort_flag, limit)) { ok = false; break; }
@@ -381,9 +444,11 @@ attn_tensor_kernel(PoolView pv, TensorArgs a, const __nv_bfloat16 *__restrict__ 
     const int t64 = tid - 64;
     uint32_t uc = 0;
     bool ok = true;
-    for (int ll = 0; ll < a.layer_count && ok; ++ll) {
-      for (int u = u0; u < u1; ++u, ++uc) {
-        const UnitInfo x = load_unit(plan, a.off_tunit, a.off_treq, u);
+    {
+      Walk wk{0, u0, 0};
+      UnitInfo x;
+      int ll = 0;
+      for (; ok && next_unit<false>(wk, a, plan, u0, u1, ring, counter, lane, true, abort_flag, limit, ok, x, ll); ++uc) {
         if (uc > 0 && !warp_wait_or_abort(bar + 8 * B_QFREE, (uc - 1) & 1, abort_flag, limit)) { ok = false; break; }
         const int rows = x.n_threads * G;
         // thread t64 builds rows 2 t64 and 2 t64 + 1; the 16 loads of a row are issued together before any store
@@ -422,9 +487,11 @@ attn_tensor_kernel(PoolView pv, TensorArgs a, const __nv_bfloat16 *__restrict__ 
     float2 *ml1 = reinterpret_cast<float2 *>(sm + OFF_ML1);
     uint32_t it = 0, uc = 0;
     bool ok = true;
-    for (int ll = 0; ll < a.layer_count && ok; ++ll) {
-      for (int u = u0; u < u1 && ok; ++u, ++uc) {
-        const UnitInfo x = load_unit(plan, a.off_tunit, a.off_treq, u);
+    {
+      Walk wk{0, u0, 0};
+      UnitInfo x;
+      int ll = 0;
+      for (; ok && next_unit<false>(wk, a, plan, u0, u1, ring, counter, lane, true, abort_flag, limit, ok, x, ll); ++uc) {
         const int nt = x.tile_end - x.tile_begin;
         const int rows = x.n_threads * G;
         // M = 128: row i of the score matrix sits in TMEM lane i.  M = 64: row i sits in lane 32 (i / 16) + i % 16, so
@@ -638,6 +705,7 @@ cudaError_t launch_attn_tensor(const PoolView &pv, const PlanHeader &h, int32_t 
   a.off_tunit = h.w[PH_OFF_TUNIT]; a.off_treq = h.w[PH_OFF_TREQ]; a.off_tcta = h.w[PH_OFF_TCTA];
   a.off_pages = h.w[PH_OFF_PAGES]; a.off_pmeta = h.w[PH_OFF_PMETA]; a.off_vis = h.w[PH_OFF_VIS];
   a.off_tq = h.w[PH_OFF_TQ];
+  a.off_dunit = h.w[PH_OFF_DUNIT]; a.n_dunits = h.w[PH_N_DUNITS];
   a.n_queries = h.w[PH_N_QUERIES]; a.layer_begin = layer_begin; a.layer_count = layer_count;
   a.scale_log2 = scale_log2;
   attn_tensor_kernel<<<grid, T_THREADS, T_SMEM_BYTES, st>>>(pv, a, static_cast<const __nv_bfloat16 *>(q));

@@ -44,6 +44,10 @@ struct PoolView {
 };
 
 __device__ __forceinline__ void report(int32_t *status, int32_t code) { atomicMax(status, code); }
+// The status word is the first of 64 words the library keeps for itself.  Word 8 counts the shared units the CTAs of
+// the tensor-core kernel have taken in the current launch (the merge that follows puts it back to zero); words 16-17
+// are the sink of the read-only measurement kernels.
+#define PASTA_STATUS_TAIL_COUNTER 8
 
 // ---------------------------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void *p) {

@@ -539,8 +539,10 @@ cudaError_t launch_attn_warp(const PoolView &pv, const PlanHeader &h, int32_t la
 template <bool kOutBf16>
 __global__ void __launch_bounds__(256)
 merge_kernel(PoolView pv, int32_t n_queries, int32_t layer_count, int32_t off_query, int32_t off_trange,
-             int32_t off_tunit, int32_t t_rows, int32_t layers_per_warp, void *__restrict__ out_raw,
-             float *__restrict__ lse) {
+             int32_t off_tunit, int32_t off_drange, int32_t off_dunit, int32_t t_rows, int32_t layers_per_warp,
+             void *__restrict__ out_raw, float *__restrict__ lse) {
+  // the tensor-core kernel of this launch group is over: its counter of shared units starts from zero next time
+  if (blockIdx.x == 0 && threadIdx.x == 0) pv.status[PASTA_STATUS_TAIL_COUNTER] = 0;
   const int D = pv.head_dim, Hq = pv.n_q_heads, G = Hq / pv.n_kv_heads;
   const int64_t gw = (static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x) >> 5;
   const int lane = threadIdx.x & 31;
@@ -553,15 +555,18 @@ merge_kernel(PoolView pv, int32_t n_queries, int32_t layer_count, int32_t off_qu
   const int g = h / G, hl = h % G;
   const int32_t *Q = pv.plan + off_query + n * PQ_WORDS;
   const int treq = Q[PQ_TREQ], tidx = Q[PQ_TIDX], w0 = Q[PQ_WUNIT0], nw = Q[PQ_NW];
-  int tb = 0, nt = 0;
+  int tb = 0, nt = 0, db = 0, nd = 0;
   if (treq >= 0) {
     tb = pv.plan[off_trange + (treq * pv.n_kv_heads + g) * 2];
     nt = pv.plan[off_trange + (treq * pv.n_kv_heads + g) * 2 + 1] - tb;
+    db = pv.plan[off_drange + (treq * pv.n_kv_heads + g) * 2];
+    nd = pv.plan[off_drange + (treq * pv.n_kv_heads + g) * 2 + 1] - db;
   }
-  const int total = nt + nw;
-  auto row_of = [&](int i) -> int64_t {     // within one layer
+  const int total = nt + nd + nw;
+  auto row_of = [&](int i) -> int64_t {     // within one layer: assigned units, shared units, warp-shuffle pieces
     if (i < nt) return pv.plan[off_tunit + (tb + i) * PU_WORDS + PU_ROW_BASE] + tidx * G + hl;
-    return t_rows + static_cast<int64_t>(w0 + g * nw + (i - nt)) * G + hl;
+    if (i < nt + nd) return pv.plan[off_dunit + (db + i - nt) * PU_WORDS + PU_ROW_BASE] + tidx * G + hl;
+    return t_rows + static_cast<int64_t>(w0 + g * nw + (i - nt - nd)) * G + hl;
   };
   const int E = D >> 5;                    // 4 or 2 elements per lane
   // lane i looks up partial row i (and i + 32, ...) once; the weighted sum then takes rows and weights from the
@@ -645,12 +650,12 @@ cudaError_t launch_merge(const PoolView &pv, const PlanHeader &h, int32_t layer_
   const int64_t blocks = (warps * 32 + 255) / 256;
   if (out_bf16)
     merge_kernel<true><<<static_cast<unsigned>(blocks), 256, 0, st>>>(pv, h.w[PH_N_QUERIES], layer_count, h.w[PH_OFF_QUERY],
-                                                                      h.w[PH_OFF_TRANGE], h.w[PH_OFF_TUNIT], h.w[PH_T_ROWS],
-                                                                      layers_per_warp, out, lse);
+                                                                      h.w[PH_OFF_TRANGE], h.w[PH_OFF_TUNIT], h.w[PH_OFF_DRANGE],
+                                                                      h.w[PH_OFF_DUNIT], h.w[PH_T_ROWS], layers_per_warp, out, lse);
   else
     merge_kernel<false><<<static_cast<unsigned>(blocks), 256, 0, st>>>(pv, h.w[PH_N_QUERIES], layer_count, h.w[PH_OFF_QUERY],
-                                                                       h.w[PH_OFF_TRANGE], h.w[PH_OFF_TUNIT], h.w[PH_T_ROWS],
-                                                                       layers_per_warp, out, lse);
+                                                                       h.w[PH_OFF_TRANGE], h.w[PH_OFF_TUNIT], h.w[PH_OFF_DRANGE],
+                                                                       h.w[PH_OFF_DUNIT], h.w[PH_T_ROWS], layers_per_warp, out, lse);
   return cudaGetLastError();
 }
 

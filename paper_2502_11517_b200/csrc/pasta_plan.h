@@ -13,9 +13,12 @@
 //              times the `group` query heads of one kv head: row = t_idx * group + h_local.
 //   t-unit     (t-request, kv head, tile range): one CTA-sized piece of the tensor-core kernel; it
 //              writes one partial result (m, l, O[d]) per row.
+//   d-unit     a t-unit that belongs to no CTA in advance: of the short (t-request, kv head) runs, every so often a
+//              whole one is kept back; the CTAs take these from a shared counter once their own units are done, so
+//              that SMs that stream faster than others end up doing more of the work.  Same record as a t-unit.
 //   w-unit     (query, kv head, token range of one stream) of a request that is no t-request: one warp of
 //              the warp-shuffle kernel; it writes `group` partial rows.
-//   partial rows are numbered per layer: t-unit rows first (row_base + row), then
+//   partial rows are numbered per layer: rows of the t-units and d-units first (row_base + row), then
 //              t_rows + w_unit * group + h_local.
 #pragma once
 #include <cstdint>
@@ -41,7 +44,7 @@ enum {
   PH_N_TREQ,
   PH_N_TUNITS,
   PH_N_WUNITS,
-  PH_T_ROWS,          // partial rows written by t-units
+  PH_T_ROWS,          // partial rows written by t-units and d-units
   PH_ROWS,            // all partial rows of one layer
   PH_T_GRID,          // CTAs of the tensor-core kernel that have work
   PH_OFF_APPEND,      // 2 words per appended token: page, offset
@@ -58,6 +61,9 @@ enum {
   PH_OFF_APOS,        // position id of every appended token (parallel to the append table)
   PH_OFF_QPOS,        // position id of every query's token
   PH_TOTAL_WORDS,
+  PH_N_DUNITS,        // d-units of one layer
+  PH_OFF_DUNIT,       // PU_WORDS per d-unit
+  PH_OFF_DRANGE,      // per (t-request, kv head): first d-unit, one past the last
   PH_WORDS = 32
 };
 

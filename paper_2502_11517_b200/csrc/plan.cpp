@@ -30,6 +30,14 @@ struct TUnit {
 
 }  // namespace
 
+// the same step planned with every tile assigned in advance: what is left when the shared tail does not fit the
+// pool's capacities (it adds units, hence partial rows and plan words)
+static pasta_status_t without_tail(const HostPool &pool, const std::vector<StepQuery> &entries,
+                                   const std::vector<Slot> &slots, PlanLimits lim, std::vector<int32_t> *out) {
+  lim.tail_percent = 0;
+  return build_plan(pool, entries, slots, lim, out);
+}
+
 pasta_status_t build_plan(const HostPool &pool, const std::vector<StepQuery> &entries,
                           const std::vector<Slot> &slots, const PlanLimits &lim,
                           std::vector<int32_t> *out) {
@@ -164,27 +172,54 @@ pasta_status_t build_plan(const HostPool &pool, const std::vector<StepQuery> &en
   // ---- t-units: cut the sequence of (t-request, kv head) tile runs into one contiguous range per CTA
   std::vector<TUnit> tunits;
   std::vector<int32_t> trange(treqs.size() * lim.n_kv_heads * 2, 0);
+  std::vector<int32_t> drange(treqs.size() * lim.n_kv_heads * 2, 0);
+  std::vector<TUnit> dunits;
   std::vector<int32_t> tcta;
   int32_t t_rows = 0;
   if (!treqs.empty()) {
-    // Every tile has a position on a cost axis (tiles, plus `overhead` at the start of each (t-request, kv head)
-    // run); CTA c owns positions [c, c + 1) * total / grid.  Positions are absolute, so rounding at one cut does
-    // not move the others.  Cuts that would leave fewer than `min_piece` tiles on one side snap to the run's end.
+    // Some of the work is kept back from the assignment below, as units which the CTAs share out among themselves at
+    // run time (equal tile counts do not finish at the same time: SMs differ in the bandwidth they get).  Only when
+    // there is enough work for that to matter.
+    int64_t all_tiles = 0;
+    for (const TReq &t : treqs) all_tiles += int64_t(lim.n_kv_heads) * ((t.n_pages + PASTA_TILE_PAGES - 1) / PASTA_TILE_PAGES);
+    const bool share_tail = lim.tail_percent > 0 && lim.tail_tiles > 0 && all_tiles >= 16LL * std::max(1, lim.grid);
+    // Runs of a few tiles go to the pool whole, every so often, until the pool holds its share of their tiles (`owed`
+    // counts what they still owe it): a whole run is a unit anyway, so sharing it costs no extra cut and no extra
+    // partial rows.  Long runs stay assigned: cutting their ends into short units cost more, in unit changes and
+    // partial rows, than the evener finish gave back (measured on 8 x 32768-token prefixes).
+    std::vector<int32_t> tail(treqs.size() * lim.n_kv_heads, 0);
+    if (share_tail) {
+      int64_t owed = 0;
+      for (size_t ti = 0; ti < treqs.size(); ++ti) {
+        const int32_t n_tiles = (treqs[ti].n_pages + PASTA_TILE_PAGES - 1) / PASTA_TILE_PAGES;
+        if (n_tiles > 4 * lim.tail_tiles) continue;
+        for (int32_t g = 0; g < lim.n_kv_heads; ++g) {
+          owed += int64_t(n_tiles) * lim.tail_percent;
+          if (owed >= int64_t(n_tiles) * 100) { tail[ti * lim.n_kv_heads + g] = n_tiles; owed -= int64_t(n_tiles) * 100; }
+        }
+      }
+    }
     const double overhead = 1.0;
     const int32_t min_piece = 1;
     double total = 0;
-    for (const TReq &t : treqs)
-      total += lim.n_kv_heads * ((t.n_pages + PASTA_TILE_PAGES - 1) / PASTA_TILE_PAGES + overhead);
+    for (size_t ti = 0; ti < treqs.size(); ++ti) {
+      const int32_t n_tiles = (treqs[ti].n_pages + PASTA_TILE_PAGES - 1) / PASTA_TILE_PAGES;
+      for (int32_t g = 0; g < lim.n_kv_heads; ++g) {
+        const int32_t kept = n_tiles - tail[ti * lim.n_kv_heads + g];
+        if (kept > 0) total += kept + overhead;
+      }
+    }
     const int32_t grid = std::max(1, lim.grid);
-    const double target = total / grid;
+    const double target = std::max(total, 1.0) / grid;
     std::vector<int32_t> unit_cta;
     double cum = 0;
     for (size_t ti = 0; ti < treqs.size(); ++ti) {
-      const int32_t n_tiles = (treqs[ti].n_pages + PASTA_TILE_PAGES - 1) / PASTA_TILE_PAGES;
+      const int32_t all = (treqs[ti].n_pages + PASTA_TILE_PAGES - 1) / PASTA_TILE_PAGES;
       const int32_t rows = treqs[ti].n_threads * G;
       for (int32_t g = 0; g < lim.n_kv_heads; ++g) {
+        const int32_t n_tiles = all - tail[ti * lim.n_kv_heads + g];       // what is assigned to CTAs here
         trange[(ti * lim.n_kv_heads + g) * 2] = static_cast<int32_t>(tunits.size());
-        cum += overhead;
+        if (n_tiles > 0) cum += overhead;
         int32_t begin = 0;
         while (begin < n_tiles) {
           const int32_t remaining = n_tiles - begin;
@@ -203,6 +238,12 @@ pasta_status_t build_plan(const HostPool &pool, const std::vector<StepQuery> &en
           cum += take;
         }
         trange[(ti * lim.n_kv_heads + g) * 2 + 1] = static_cast<int32_t>(tunits.size());
+        drange[(ti * lim.n_kv_heads + g) * 2] = static_cast<int32_t>(dunits.size());
+        for (int32_t b2 = n_tiles; b2 < all; b2 += lim.tail_tiles) {
+          dunits.push_back(TUnit{static_cast<int32_t>(ti), g, b2, std::min(all, b2 + lim.tail_tiles), t_rows});
+          t_rows += rows;
+        }
+        drange[(ti * lim.n_kv_heads + g) * 2 + 1] = static_cast<int32_t>(dunits.size());
       }
     }
     for (size_t u = 0; u < tunits.size(); ++u) {
@@ -212,7 +253,12 @@ pasta_status_t build_plan(const HostPool &pool, const std::vector<StepQuery> &en
         tcta.push_back(static_cast<int32_t>(u));
       }
     }
-    tcta.back() = static_cast<int32_t>(tunits.size());
+    if (!tcta.empty()) tcta.back() = static_cast<int32_t>(tunits.size());
+    // every CTA of the grid takes part in sharing out the tail, also those that were assigned nothing
+    while (!dunits.empty() && static_cast<int32_t>(tcta.size() / 2) < grid) {
+      tcta.push_back(static_cast<int32_t>(tunits.size()));
+      tcta.push_back(static_cast<int32_t>(tunits.size()));
+    }
   }
 
   // ---- w-units: pieces of at most `chunk` tokens, ordered (query, kv head, piece)
@@ -230,6 +276,7 @@ pasta_status_t build_plan(const HostPool &pool, const std::vector<StepQuery> &en
     n_wunits = 0;
     for (int32_t i = 0; i < n; ++i) n_wunits += static_cast<int64_t>(q_nw[i]) * lim.n_kv_heads;
     if (t_rows + n_wunits * G <= lim.max_rows) break;
+    if (!dunits.empty()) return without_tail(pool, entries, slots, lim, out);    // the shared tail costs rows: do without
     if (chunk >= (1 << 24)) return PASTA_ERR_CAPACITY;
     chunk *= 2;
   }
@@ -282,7 +329,7 @@ pasta_status_t build_plan(const HostPool &pool, const std::vector<StepQuery> &en
     qtab[i * PQ_WORDS + PQ_WUNIT0] = q_w0[i];
     qtab[i * PQ_WORDS + PQ_NW] = q_nw[i];
   }
-  std::vector<int32_t> ttab, utab;
+  std::vector<int32_t> ttab, utab, dtab;
   for (const TReq &t : treqs) {
     const int32_t rec[PT_WORDS] = {t.page_off, t.n_pages, t.n_threads, t.n_streams, t.vis_off, t.tq_off};
     ttab.insert(ttab.end(), rec, rec + PT_WORDS);
@@ -293,7 +340,14 @@ pasta_status_t build_plan(const HostPool &pool, const std::vector<StepQuery> &en
                                    t.n_threads, t.n_streams, t.vis_off, t.tq_off, 0};
     utab.insert(utab.end(), rec, rec + PU_WORDS);
   }
+  for (const TUnit &u : dunits) {
+    const TReq &t = treqs[u.treq];
+    const int32_t rec[PU_WORDS] = {u.treq, u.g, u.tile_begin, u.tile_end, u.row_base, t.page_off, t.n_pages,
+                                   t.n_threads, t.n_streams, t.vis_off, t.tq_off, 0};
+    dtab.insert(dtab.end(), rec, rec + PU_WORDS);
+  }
   w[PH_MAGIC] = PASTA_PLAN_MAGIC;
+  w[PH_N_DUNITS] = static_cast<int32_t>(dunits.size());
   w[PH_N_QUERIES] = n;
   w[PH_N_APPEND] = n_app;
   w[PH_N_TREQ] = static_cast<int32_t>(treqs.size());
@@ -315,8 +369,13 @@ pasta_status_t build_plan(const HostPool &pool, const std::vector<StepQuery> &en
   put(PH_OFF_TQ, tq_tab);
   put(PH_OFF_APOS, apos);
   put(PH_OFF_QPOS, qpos);
+  put(PH_OFF_DUNIT, dtab);
+  put(PH_OFF_DRANGE, drange);
   w[PH_TOTAL_WORDS] = static_cast<int32_t>(w.size());
-  if (static_cast<int64_t>(w.size()) > lim.max_words) return PASTA_ERR_CAPACITY;
+  if (static_cast<int64_t>(w.size()) > lim.max_words) {
+    if (!dunits.empty()) return without_tail(pool, entries, slots, lim, out);
+    return PASTA_ERR_CAPACITY;
+  }
   return PASTA_OK;
 }
 

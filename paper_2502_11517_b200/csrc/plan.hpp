@@ -14,6 +14,8 @@ struct PlanLimits {
   int64_t max_words;     // size of the device copy of the plan
   int32_t grid;          // CTAs the tensor-core kernel may use (one per SM)
   bool tensor_path;      // false: every stream goes to the warp-shuffle kernel
+  int32_t tail_percent;  // share of every long run's tiles that is handed out at run time (0: everything is assigned)
+  int32_t tail_tiles;    // tiles per unit of that share
 };
 
 // Plans the attention of one step: one query per element of `queries`, `slots` parallel to it.

@@ -6,7 +6,8 @@ import numpy as np
 # header word indices (pasta_plan.h)
 (PH_MAGIC, PH_N_QUERIES, PH_N_APPEND, PH_N_TREQ, PH_N_TUNITS, PH_N_WUNITS, PH_T_ROWS, PH_ROWS, PH_T_GRID,
  PH_OFF_APPEND, PH_OFF_QUERY, PH_OFF_TREQ, PH_OFF_TRANGE, PH_OFF_TUNIT, PH_OFF_TCTA, PH_OFF_WUNIT, PH_OFF_PAGES,
- PH_OFF_PMETA, PH_OFF_VIS, PH_OFF_TQ, PH_OFF_APOS, PH_OFF_QPOS, PH_TOTAL_WORDS) = range(23)
+ PH_OFF_PMETA, PH_OFF_VIS, PH_OFF_TQ, PH_OFF_APOS, PH_OFF_QPOS, PH_TOTAL_WORDS, PH_N_DUNITS, PH_OFF_DUNIT,
+ PH_OFF_DRANGE) = range(26)
 PQ, PT, PU, PW = 4, 6, 12, 4
 TILE_PAGES, PAGE = 8, 16
 STATS = {'flagged': 0, 'pages': 0}    # pages the plans marked as visible in full to every thread, of all pages walked
@@ -29,13 +30,18 @@ def run_plan(w, K, V, q, n_kv_heads):
         assert cta[0, 0] == 0 and cta[-1, 1] == w[PH_N_TUNITS]
         assert np.all(cta[1:, 0] == cta[:-1, 1]) and np.all(cta[:, 1] > cta[:, 0])
 
-    for u in range(w[PH_N_TUNITS]):
-        rec = w[w[PH_OFF_TUNIT] + u * PU: w[PH_OFF_TUNIT] + (u + 1) * PU]
+    # assigned units, then the units the CTAs share out at run time (same record, a table of their own)
+    recs = [w[w[PH_OFF_TUNIT] + u * PU: w[PH_OFF_TUNIT] + (u + 1) * PU] for u in range(w[PH_N_TUNITS])]
+    recs += [w[w[PH_OFF_DUNIT] + u * PU: w[PH_OFF_DUNIT] + (u + 1) * PU] for u in range(w[PH_N_DUNITS])]
+    STATS['dunits'] = STATS.get('dunits', 0) + int(w[PH_N_DUNITS])
+    covered = {}
+    for u, rec in enumerate(recs):
         treq, g, tb, te, row_base = rec[:5]
         T = w[PH_OFF_TREQ] + treq * PT
         page_off, n_pages, n_thr, n_str, vis_off, tq_off = w[T:T + PT]
         assert list(rec[5:11]) == [page_off, n_pages, n_thr, n_str, vis_off, tq_off]     # the unit repeats its t-request
         assert 0 <= tb < te <= -(-n_pages // TILE_PAGES)
+        covered.setdefault((int(treq), int(g)), []).append((int(tb), int(te), -(-int(n_pages) // TILE_PAGES)))
         vis = w[w[PH_OFF_VIS] + vis_off: w[PH_OFF_VIS] + vis_off + n_thr * n_str].reshape(n_thr, n_str)
         tq = w[w[PH_OFF_TQ] + tq_off: w[PH_OFF_TQ] + tq_off + n_thr]
         for ti in range(n_thr):
@@ -58,6 +64,11 @@ def run_plan(w, K, V, q, n_kv_heads):
                     m[row], l[row], O[row] = -np.inf, 0.0, 0.0
                 else:
                     m[row] = s.max(); e = np.exp(s - m[row]); l[row] = e.sum(); O[row] = e @ v
+
+    for spans in covered.values():          # the units of a run tile it exactly: every tile once
+        spans.sort()
+        assert spans[0][0] == 0 and spans[-1][1] == spans[0][2]
+        assert all(a[1] == b[0] for a, b in zip(spans, spans[1:]))
 
     for u in range(w[PH_N_WUNITS]):
         qi, g, page_off, n_tok = w[w[PH_OFF_WUNIT] + u * PW: w[PH_OFF_WUNIT] + (u + 1) * PW]
@@ -83,6 +94,10 @@ def run_plan(w, K, V, q, n_kv_heads):
                 for u in range(tr[(treq * n_kv_heads + g) * 2], tr[(treq * n_kv_heads + g) * 2 + 1]):
                     assert w[w[PH_OFF_TUNIT] + u * PU] == treq and w[w[PH_OFF_TUNIT] + u * PU + 1] == g
                     rows_i.append(w[w[PH_OFF_TUNIT] + u * PU + 4] + tidx * G + hl)
+                dr = w[w[PH_OFF_DRANGE]:]
+                for u in range(dr[(treq * n_kv_heads + g) * 2], dr[(treq * n_kv_heads + g) * 2 + 1]):
+                    assert w[w[PH_OFF_DUNIT] + u * PU] == treq and w[w[PH_OFF_DUNIT] + u * PU + 1] == g
+                    rows_i.append(w[w[PH_OFF_DUNIT] + u * PU + 4] + tidx * G + hl)
             rows_i += [t_rows + (w0 + g * nw + k) * G + hl for k in range(nw)]
             rows_i = [r for r in rows_i if l[r] > 0]
             ms = max(m[r] for r in rows_i)

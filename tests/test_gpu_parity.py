@@ -33,11 +33,13 @@ def compare(got, got_lse, want, want_lse, what=""):
     return err.max(), err.mean()
 
 
-def run_script(lib, script, flags=0, layers=None, check_steps=None, **kw):
+def run_script(lib, script, flags=0, layers=None, check_steps=None, tail=None, **kw):
     """Replays on both sides; compares bookkeeping after every op and attention at every (chosen) step."""
     from lib_replay import LibReplay, make_pool
     layers = list(range(script.geometry.n_layers)) if layers is None else layers
     pool = make_pool(script, flags=flags, **kw)
+    if tail is not None:
+        pool.debug_set_tail(*tail)
     rep = LibReplay(script, pool)
     ora = OracleReplay(script, layers=layers)
     worst = (0.0, 0.0)
@@ -297,3 +299,26 @@ def test_step_host_in_two_halves_keeps_two_steps_in_flight(lib, slots):
     assert e.value.code == lib.BAD_STATE
     assert pool.dump() == ora.model.dump() and pool.status() == 0
     pool.close()
+
+
+@pytest.mark.parametrize("tail", [(10, 16), (50, 10), (0, 4)])
+def test_units_shared_out_at_run_time_long_runs(lib, tail):
+    """Enough tiles (64 runs of 38) for the planner to keep whole runs back as units the CTAs take from a counter at
+    run time; with half of all tiles shared in units of 10 tiles every CTA goes through several of them."""
+    from lib_replay import LibReplay, make_pool
+    script = cfg4_long_prefix(8, 4000, 4, n_new=1)
+    pool = make_pool(script, host_only=True)
+    pool.debug_set_tail(*tail)
+    rep = LibReplay(script, pool)
+    for i in range(len(script.ops)):
+        rep.apply(i)
+    assert (pool.plan_words()[23] > 0) == (tail[0] > 0)          # shared units in the plan
+    pool.close()
+    run_script(lib, script, tail=tail)
+
+
+def test_units_shared_out_at_run_time_short_runs_three_layers(lib):
+    """The batched configuration with three layers in one launch: whole short runs go to the shared pool, and a shared
+    unit is a (layer, unit) pair.  Two launches in a row: the counter starts from zero each time."""
+    run_script(lib, cfg3_batched(64, 3, n_new=1), tail=(20, 3))
+    run_script(lib, cfg3_batched(64, 3), tail=(20, 3), max_layers_per_launch=2)

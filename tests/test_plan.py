@@ -20,9 +20,11 @@ def _f64(t):
     return t.to(torch.float32).numpy().astype(np.float64)
 
 
-def check_script(script, flags=0, steps=None, **kw):
+def check_script(script, flags=0, steps=None, tail=None, **kw):
     geo = script.geometry
     pool = make_pool(script, host_only=True, flags=flags, **kw)
+    if tail is not None:
+        pool.debug_set_tail(*tail)
     lib = LibReplay(script, pool)
     ora = OracleReplay(script)
     K = np.zeros((script.n_pages, 16, geo.n_kv_heads, geo.head_dim)); V = np.zeros_like(K)
@@ -97,6 +99,47 @@ def test_small_partial_budget_still_plans():
     script = cfg3_batched(4, 1, prefix_range=(300, 600))
     n = len(script.ops[-1][1])
     check_script(script, max_partial_rows=n * 32 * 2 + 160 * 128)
+
+
+@pytest.mark.parametrize("tail", [None, (25, 10), (50, 16), (25, 2), (0, 4)])
+def test_plan_with_shared_units(tail):
+    """Enough tiles (64 runs of 38) for the planner to keep whole runs back as units the CTAs share out at run time,
+    when runs of 38 tiles count as short (at most four units long): every run must still be tiled exactly once and the
+    merged result must equal the oracle's."""
+    from plan_interpreter import STATS
+    before = STATS.get("dunits", 0)
+    check_script(cfg4_long_prefix(8, 4000, 4), tail=tail)
+    assert (STATS.get("dunits", 0) > before) == (tail not in ((0, 4), (25, 2)))
+
+
+def test_plan_with_a_shared_tail_short_runs():
+    """Many short runs (the batched configuration, one layer): whole runs go to the shared pool, every so often."""
+    from plan_interpreter import STATS
+    before = STATS.get("dunits", 0)
+    check_script(cfg3_batched(64, 1))
+    assert STATS.get("dunits", 0) > before
+
+
+def test_shared_tail_is_dropped_when_it_does_not_fit():
+    """With room for the partial rows of the assigned units only, the step is planned without a shared tail instead of
+    being refused."""
+    script = cfg4_long_prefix(8, 4000, 4)
+
+    def plan(tail, **kw):
+        pool = make_pool(script, host_only=True, **kw)
+        if tail:
+            pool.debug_set_tail(*tail)
+        lib = LibReplay(script, pool)
+        for i in range(len(script.ops)):
+            lib.apply(i)
+        w = pool.plan_words()
+        pool.close()
+        return int(w[7]), int(w[23])               # partial rows of a layer, shared units
+
+    rows_without, none = plan((0, 4))
+    rows_with, some = plan(None)
+    assert none == 0 and some > 0 and rows_with > rows_without
+    assert plan(None, max_partial_rows=rows_without + 8) == (rows_without, 0)
 
 
 def test_zz_all_visible_page_flag_is_exercised():
