@@ -46,65 +46,80 @@ pasta_status_t build_plan(const HostPool &pool, const std::vector<StepQuery> &en
   const int32_t P = PASTA_PAGE;
   if (n > lim.max_queries) return PASTA_ERR_CAPACITY;
 
-  // ---- group the queries by request, in order of first appearance
-  std::vector<int32_t> req_order;
-  std::vector<std::vector<int32_t>> by_req;
+  // Scratch that keeps its capacity from one step to the next (a pool plans a step at a time; the planner of another
+  // pool on another host thread has its own): this function runs once per decode step and most of what it does is
+  // small.
+  static thread_local std::vector<int32_t> req_order, slot_of, group_begin, order, vis_of, use_index, q_vis;
+  static thread_local std::vector<StreamUse> uses;
+  static thread_local std::vector<int32_t> pages, pmeta, vis_tab, tq_tab;
+
+  // ---- group the queries by request, in order of first appearance: order[group_begin[g] .. group_begin[g + 1])
+  req_order.clear();
+  slot_of.clear();
+  group_begin.clear();
+  for (int32_t i = 0; i < n; ++i) {
+    const int32_t r = entries[i].req;
+    if (r >= static_cast<int32_t>(slot_of.size())) slot_of.resize(r + 1, -1);
+    if (slot_of[r] < 0) {
+      slot_of[r] = static_cast<int32_t>(req_order.size());
+      req_order.push_back(r);
+      group_begin.push_back(0);
+    }
+    group_begin[slot_of[r]] += 1;
+  }
   {
-    std::vector<std::pair<int32_t, int32_t>> first;   // (req, group index), small linear map would be O(n^2)
-    std::vector<int32_t> slot_of;
+    int32_t at = 0;
+    for (int32_t &b : group_begin) { const int32_t c = b; b = at; at += c; }
+    group_begin.push_back(at);
+    order.assign(n, 0);
+    std::vector<int32_t> &fill = vis_of;          // borrowed as the groups' fill counters
+    fill.assign(req_order.size(), 0);
     for (int32_t i = 0; i < n; ++i) {
-      const int32_t r = entries[i].req;
-      if (r >= static_cast<int32_t>(slot_of.size())) slot_of.resize(r + 1, -1);
-      if (slot_of[r] < 0) {
-        slot_of[r] = static_cast<int32_t>(by_req.size());
-        req_order.push_back(r);
-        by_req.emplace_back();
-      }
-      by_req[slot_of[r]].push_back(i);
+      const int32_t g = slot_of[entries[i].req];
+      order[group_begin[g] + fill[g]++] = i;
     }
   }
 
-  std::vector<int32_t> pages, pmeta, vis_tab, tq_tab;
+  pages.clear(); pmeta.clear(); vis_tab.clear(); tq_tab.clear();
   std::vector<TReq> treqs;
   std::vector<WPiece> wpieces;
   std::vector<int32_t> q_treq(n, -1), q_tidx(n, 0);
-  std::vector<int32_t> vis_of;      // scratch: stream -> visible length for the current query
-  std::vector<int32_t> use_index;   // scratch: stream -> index in `uses`
   int64_t w_tokens = 0;
 
-  for (size_t gi = 0; gi < by_req.size(); ++gi) {
+  for (size_t gi = 0; gi < req_order.size(); ++gi) {
     const Request *r = pool.request(req_order[gi]);
-    const std::vector<int32_t> &qs = by_req[gi];
-    const int32_t T = static_cast<int32_t>(qs.size());
+    const int32_t *qs = order.data() + group_begin[gi];
+    const int32_t T = group_begin[gi + 1] - group_begin[gi];
     const int32_t n_streams_all = static_cast<int32_t>(r->streams.size());
+    // the streams the step's threads of this request read, in order of first appearance in their views
     use_index.assign(n_streams_all, -1);
-    std::vector<StreamUse> uses;
-    std::vector<std::vector<int32_t>> q_vis(T);       // per query: visible length per entry of `uses` (grown lazily)
+    uses.clear();
+    for (int32_t ti = 0; ti < T; ++ti)
+      for (const Seg &sg : r->threads[entries[qs[ti]].thread].view)
+        if (use_index[sg.stream] < 0) {
+          use_index[sg.stream] = static_cast<int32_t>(uses.size());
+          uses.push_back(StreamUse{sg.stream, 0, 0});
+        }
+    const int32_t U = static_cast<int32_t>(uses.size());
+    // q_vis[ti * U + u]: how much of stream uses[u] query ti sees
+    q_vis.assign(static_cast<size_t>(T) * U, 0);
     for (int32_t ti = 0; ti < T; ++ti) {
-      const Thread &th = r->threads[entries[qs[ti]].thread];
-      vis_of.assign(n_streams_all, 0);
-      for (const Seg &s : th.view) vis_of[s.stream] = std::max(vis_of[s.stream], s.start + s.len);
+      const StepQuery &e = entries[qs[ti]];
+      int32_t *row = q_vis.data() + static_cast<size_t>(ti) * U;
+      for (const Seg &sg : r->threads[e.thread].view) {
+        int32_t &v = row[use_index[sg.stream]];
+        v = std::max(v, sg.start + sg.len);
+      }
       // a query for an earlier one of several tokens appended in this step does not see the later ones: they are
       // the end of the thread's own stream (stream id = thread id)
-      vis_of[entries[qs[ti]].thread] -= entries[qs[ti]].hide;
-      for (const Seg &s : th.view) {
-        if (use_index[s.stream] < 0) {
-          use_index[s.stream] = static_cast<int32_t>(uses.size());
-          uses.push_back(StreamUse{s.stream, 0, 0});
-        }
-      }
-      q_vis[ti].assign(uses.size(), 0);
-      for (size_t u = 0; u < uses.size(); ++u) {
-        const int32_t v = vis_of[uses[u].stream];
-        q_vis[ti][u] = v;
-        if (v > 0) {
+      if (e.hide && use_index[e.thread] >= 0) row[use_index[e.thread]] -= e.hide;
+      for (int32_t u = 0; u < U; ++u)
+        if (row[u] > 0) {
           // count each (query, stream) once: views list a stream several times only for the main stream pieces
           uses[u].n_seen += 1;
-          uses[u].max_vis = std::max(uses[u].max_vis, v);
+          uses[u].max_vis = std::max(uses[u].max_vis, row[u]);
         }
-      }
     }
-    for (int32_t ti = 0; ti < T; ++ti) q_vis[ti].resize(uses.size(), 0);
 
     // A request whose stacked rows fit one MMA tile sends EVERY stream it reads through the tensor-core kernel, the
     // private chunks too: rows that may not see a page are masked there, the MMA costs the same for any number of
@@ -133,7 +148,7 @@ pasta_status_t build_plan(const HostPool &pool, const std::vector<StepQuery> &en
         const std::vector<int32_t> &sp = r->streams[u.stream].pages;
         const int32_t np = (u.max_vis + P - 1) / P;
         int32_t min_vis = u.max_vis;             // what EVERY thread of the request sees of this stream
-        for (int32_t ti = 0; ti < T; ++ti) min_vis = std::min(min_vis, q_vis[ti][ui]);
+        for (int32_t ti = 0; ti < T; ++ti) min_vis = std::min(min_vis, q_vis[static_cast<size_t>(ti) * U + ui]);
         pages.insert(pages.end(), sp.begin(), sp.begin() + np);
         const size_t m0 = pmeta.size();
         pmeta.resize(m0 + np);
@@ -145,7 +160,7 @@ pasta_status_t build_plan(const HostPool &pool, const std::vector<StepQuery> &en
       t.n_pages = static_cast<int32_t>(pages.size()) - t.page_off;
       for (int32_t ti = 0; ti < T; ++ti) {
         for (size_t u = 0; u < uses.size(); ++u)
-          if (uses[u].local >= 0) vis_tab.push_back(q_vis[ti][u]);   // uses are in local order
+          if (uses[u].local >= 0) vis_tab.push_back(q_vis[static_cast<size_t>(ti) * U + u]);   // uses are in local order
         tq_tab.push_back(qs[ti]);
         q_treq[qs[ti]] = static_cast<int32_t>(treqs.size());
         q_tidx[qs[ti]] = ti;
@@ -155,7 +170,7 @@ pasta_status_t build_plan(const HostPool &pool, const std::vector<StepQuery> &en
     // streams that stay on the warp path: their pages are stored once per request
     for (int32_t ti = 0; ti < T; ++ti) {
       for (size_t u = 0; u < uses.size(); ++u) {
-        if (uses[u].local >= 0 || q_vis[ti][u] == 0) continue;
+        if (uses[u].local >= 0 || q_vis[static_cast<size_t>(ti) * U + u] == 0) continue;
         if (uses[u].page_off < 0) {
           uses[u].page_off = static_cast<int32_t>(pages.size());
           const std::vector<int32_t> &sp = r->streams[uses[u].stream].pages;
@@ -163,18 +178,18 @@ pasta_status_t build_plan(const HostPool &pool, const std::vector<StepQuery> &en
           pages.insert(pages.end(), sp.begin(), sp.begin() + np);
           pmeta.insert(pmeta.end(), np, 0);
         }
-        wpieces.push_back(WPiece{qs[ti], uses[u].page_off, q_vis[ti][u]});
-        w_tokens += q_vis[ti][u];
+        wpieces.push_back(WPiece{qs[ti], uses[u].page_off, q_vis[static_cast<size_t>(ti) * U + u]});
+        w_tokens += q_vis[static_cast<size_t>(ti) * U + u];
       }
     }
   }
 
   // ---- t-units: cut the sequence of (t-request, kv head) tile runs into one contiguous range per CTA
-  std::vector<TUnit> tunits;
-  std::vector<int32_t> trange(treqs.size() * lim.n_kv_heads * 2, 0);
-  std::vector<int32_t> drange(treqs.size() * lim.n_kv_heads * 2, 0);
-  std::vector<TUnit> dunits;
-  std::vector<int32_t> tcta;
+  static thread_local std::vector<TUnit> tunits, dunits;
+  static thread_local std::vector<int32_t> trange, drange, tcta, unit_cta, tail;
+  tunits.clear(); dunits.clear(); tcta.clear(); unit_cta.clear();
+  trange.assign(treqs.size() * lim.n_kv_heads * 2, 0);
+  drange.assign(treqs.size() * lim.n_kv_heads * 2, 0);
   int32_t t_rows = 0;
   if (!treqs.empty()) {
     // Some of the work is kept back from the assignment below, as units which the CTAs share out among themselves at
@@ -187,7 +202,7 @@ pasta_status_t build_plan(const HostPool &pool, const std::vector<StepQuery> &en
     // counts what they still owe it): a whole run is a unit anyway, so sharing it costs no extra cut and no extra
     // partial rows.  Long runs stay assigned: cutting their ends into short units cost more, in unit changes and
     // partial rows, than the evener finish gave back (measured on 8 x 32768-token prefixes).
-    std::vector<int32_t> tail(treqs.size() * lim.n_kv_heads, 0);
+    tail.assign(treqs.size() * lim.n_kv_heads, 0);
     if (share_tail) {
       int64_t owed = 0;
       for (size_t ti = 0; ti < treqs.size(); ++ti) {
@@ -211,7 +226,6 @@ pasta_status_t build_plan(const HostPool &pool, const std::vector<StepQuery> &en
     }
     const int32_t grid = std::max(1, lim.grid);
     const double target = std::max(total, 1.0) / grid;
-    std::vector<int32_t> unit_cta;
     double cum = 0;
     for (size_t ti = 0; ti < treqs.size(); ++ti) {
       const int32_t all = (treqs[ti].n_pages + PASTA_TILE_PAGES - 1) / PASTA_TILE_PAGES;
@@ -316,20 +330,21 @@ pasta_status_t build_plan(const HostPool &pool, const std::vector<StepQuery> &en
     w.insert(w.end(), v.begin(), v.end());
     while (w.size() % 4) w.push_back(0);   // keep every table 16-byte aligned
   };
-  std::vector<int32_t> app, apos, qpos;
+  static thread_local std::vector<int32_t> app, apos, qpos, qtab, ttab, utab, dtab;
+  app.clear(); apos.clear(); qpos.clear(); ttab.clear(); utab.clear(); dtab.clear();
   for (int32_t i = 0; i < n; ++i) {
     const int32_t pos = slots[i].pos;
     qpos.push_back(pos);
     if (slots[i].page >= 0) { app.push_back(slots[i].page); app.push_back(slots[i].offset); apos.push_back(pos); }
   }
-  std::vector<int32_t> qtab(static_cast<size_t>(n) * PQ_WORDS);
+  qtab.assign(static_cast<size_t>(n) * PQ_WORDS, 0);
   for (int32_t i = 0; i < n; ++i) {
     qtab[i * PQ_WORDS + PQ_TREQ] = q_treq[i];
     qtab[i * PQ_WORDS + PQ_TIDX] = q_tidx[i];
     qtab[i * PQ_WORDS + PQ_WUNIT0] = q_w0[i];
     qtab[i * PQ_WORDS + PQ_NW] = q_nw[i];
   }
-  std::vector<int32_t> ttab, utab, dtab;
+
   for (const TReq &t : treqs) {
     const int32_t rec[PT_WORDS] = {t.page_off, t.n_pages, t.n_threads, t.n_streams, t.vis_off, t.tq_off};
     ttab.insert(ttab.end(), rec, rec + PT_WORDS);
