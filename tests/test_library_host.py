@@ -236,3 +236,18 @@ def test_a_step_that_cannot_be_planned_leaves_the_pool_unchanged():
     assert pool.dump() == model.dump()
     assert list(pool.step_positions()) == [model.last_position(0, 1) - 1, model.last_position(0, 1), model.last_position(0, 0)]
     pool.close()
+
+
+def test_tuning_and_test_hooks_check_their_arguments():
+    build()
+    pool = binding.Pool(1, 8, 2, 128, 16, 1, 2, 4, flags=binding.FLAG_HOST_ONLY)
+    pool.debug_set_tail(0, 2); pool.debug_set_tail(50, 1024); pool.debug_set_tail(10, 16)
+    for bad in ((-1, 4), (51, 4), (10, 1), (10, 1025)):
+        with pytest.raises(binding.PastaError) as e:
+            pool.debug_set_tail(*bad)
+        assert e.value.code == binding.INVALID_ARG
+    for call in (lambda: pool.debug_set_wait_limit(1000), lambda: pool.debug_hold_roles(1)):
+        with pytest.raises(binding.PastaError) as e:       # a host-only pool launches nothing
+            call()
+        assert e.value.code == binding.BAD_STATE
+    pool.close()
