@@ -134,7 +134,13 @@ class Pool:
             torch.cuda.synchronize(dev)
         _check(L.pasta_pool_create(C.byref(cfg), C.byref(self._h)), "pasta_pool_create")
         self.n_layers, self.n_q_heads, self.n_kv_heads, self.head_dim = n_layers, n_q_heads, n_kv_heads, head_dim
-        self._last_n = 0
+        self._last_entries = (0, None)
+
+    @property
+    def _last_n(self) -> int:
+        """Queries of the last planned step: one per entry, or one per new token of an entry that appends several."""
+        n, nn = self._last_entries
+        return n if nn is None else int(np.maximum(nn, 1).sum())
 
     def close(self) -> None:
         if self._h:
@@ -183,8 +189,7 @@ class Pool:
         nn = None if n_new is None else _i32(n_new)
         st = C.c_void_p(0) if self.host_only else _stream(stream)
         _check(lib().pasta_step_begin(self._h, len(r), _ptr(r), _ptr(t), _ptr(nn), st), "pasta_step_begin")
-        # queries of the step: one per entry, or one per new token of an entry that appends several
-        self._last_n = len(r) if nn is None else int(np.maximum(nn, 1).sum())
+        self._last_entries = (len(r), nn)             # the step's number of queries is worked out when asked for
 
     def step_slots(self) -> np.ndarray:
         out = np.empty((self._last_n, 2), dtype=np.int32)
@@ -243,7 +248,7 @@ class Pool:
         nn = None if n_new is None else _i32(n_new)
         _check(lib().pasta_step_device(self._h, len(r), _ptr(r), _ptr(t), _ptr(nn), _dev(k_new), _dev(v_new), _dev(q),
                                        _dev(out), _dev(lse), C.c_float(scale), _stream(stream)), "pasta_step_device")
-        self._last_n = len(r) if nn is None else int(np.maximum(nn, 1).sum())
+        self._last_entries = (len(r), nn)
 
     def step_host_bytes(self, n: int) -> int:
         out = C.c_size_t()
@@ -258,7 +263,7 @@ class Pool:
         _check(lib().pasta_step_host(self._h, len(r), _ptr(r), _ptr(t), _ptr(nn), _dev(k_new), _dev(v_new), _dev(q),
                                      _dev(out), _dev(staging), C.c_size_t(staging.numel() * staging.element_size()),
                                      C.c_float(scale), _stream(stream)), "pasta_step_host")
-        self._last_n = len(r)
+        self._last_entries = (len(r), None)
 
     def step_host_begin(self, req_ids, thread_ids, n_new, k_new, v_new, q, out, staging, scale: float = 0.0,
                         stream=None) -> None:
@@ -268,7 +273,7 @@ class Pool:
         _check(lib().pasta_step_host_begin(self._h, len(r), _ptr(r), _ptr(t), _ptr(nn), _dev(k_new), _dev(v_new), _dev(q),
                                            _dev(out), _dev(staging), C.c_size_t(staging.numel() * staging.element_size()),
                                            C.c_float(scale), _stream(stream)), "pasta_step_host_begin")
-        self._last_n = len(r)
+        self._last_entries = (len(r), None)
 
     def step_host_wait(self) -> None:
         _check(lib().pasta_step_host_wait(self._h), "pasta_step_host_wait")
