@@ -15,7 +15,7 @@ using namespace pasta;
 namespace {
 
 constexpr int kStaging = 4;           // pinned upload buffers in rotation
-constexpr size_t kSmallPlanWords = 2048;   // plans up to this size are uploaded in the caller's stream
+constexpr size_t kSmallPlanWords = 8192;   // plans up to this size are uploaded in the caller's stream
 constexpr int kProfCalls = 512;        // timed pasta_decode_attn launches kept between two profile reads
 constexpr int kRunChunk = 8192;       // tokens whose slots are uploaded at once by pasta_kv_append_run
 constexpr int kTailPercent = 10;      // share of the short runs' tiles that the tensor-core kernel's CTAs share out at run time
