@@ -1114,6 +1114,9 @@ def main():
     ap.add_argument("--tail", default=None, metavar="PERCENT,TILES",
                     help="share of the short runs' tiles that the tensor-core kernel's CTAs share out at run time, and the "
                          "tiles per shared unit (pasta_debug_set_tail; the library's default when not given)")
+    ap.add_argument("--no-launch-overlap", action="store_true",
+                    help="launch the kernels of a step strictly one after the other (pasta_debug_set_launch_overlap(0)) "
+                         "instead of letting each set itself up while the one ahead drains")
     ap.add_argument("--out-dtype", default="fp32", choices=["fp32", "bf16"],
                     help="type of the attention output (bf16 halves the device-to-host bytes of the end-to-end path)")
     ap.add_argument("--layout", default="pool", choices=["pool", "naive_rows", "dense_mask"],
@@ -1124,6 +1127,11 @@ def main():
     ap.add_argument("--size", default="full", choices=["full", "small"],
                     help="small: a reduced copy of the workload for profiler captures (prefix 8192 / 4 layers)")
     args = ap.parse_args()
+    if args.no_launch_overlap and args.impl != "reference":
+        from paper_2502_11517_b200 import binding as _binding
+        from paper_2502_11517_b200.build import build as _build
+        _build()
+        _binding.Pool.debug_set_launch_overlap(False)
     if args.impl == "reference":
         if args.steps == 200:
             args.steps, args.warmup = 3, 1

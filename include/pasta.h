@@ -374,6 +374,14 @@ pasta_status_t pasta_debug_hold_roles(pasta_pool_t *pool, int32_t role_mask);
  */
 pasta_status_t pasta_debug_set_tail(pasta_pool_t *pool, int32_t percent, int32_t tiles);
 /*
+ * Tuning hook (no counterpart in the paper), process-wide.  The kernels of a step (append, the two attention passes, the
+ * merge) are launched so that each may set itself up while the one ahead of it in the stream drains (programmatic
+ * dependent launch); every kernel waits for the one ahead to have completed before it touches anything that one reads
+ * or writes, so results do not depend on the setting.  on = 0 launches them one strictly after the other; on = 1
+ * (default) overlaps them.  Takes effect from the next launch.
+ */
+void pasta_debug_set_launch_overlap(int32_t on);
+/*
  * Measurement aid (no counterpart in the paper): enqueues a kernel that reads `bytes` of device memory at `src`
  * (16-byte aligned; NULL = the pool's own KV memory, all of it) and does nothing with them, so that a benchmark can
  * time what a read-only kernel is given on this GPU next to the attention kernel.  mode 0: plain 16-byte loads;

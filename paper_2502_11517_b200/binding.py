@@ -30,6 +30,7 @@ EXPORTS = [
     "pasta_last_cuda_error", "pasta_debug_set_wait_limit", "pasta_debug_wait_expiry", "pasta_debug_hold_roles",
     "pasta_debug_stream_read", "pasta_step_host_begin", "pasta_step_host_wait",
     "pasta_dense_mask_scratch_bytes", "pasta_dense_append", "pasta_dense_mask_attn", "pasta_debug_set_tail",
+    "pasta_debug_set_launch_overlap",
 ]
 
 
@@ -67,6 +68,7 @@ def lib() -> C.CDLL:
         _lib = C.CDLL(LIB)
         for name in EXPORTS:
             getattr(_lib, name).restype = C.c_int32
+        _lib.pasta_debug_set_launch_overlap.restype = None
     return _lib
 
 
@@ -354,6 +356,10 @@ class Pool:
 
     def debug_set_tail(self, percent: int, tiles: int) -> None:
         _check(lib().pasta_debug_set_tail(self._h, percent, tiles), "pasta_debug_set_tail")
+
+    @staticmethod
+    def debug_set_launch_overlap(on: bool) -> None:
+        lib().pasta_debug_set_launch_overlap(1 if on else 0)
 
     def debug_hold_roles(self, role_mask: int) -> None:
         _check(lib().pasta_debug_hold_roles(self._h, role_mask), "pasta_debug_hold_roles")

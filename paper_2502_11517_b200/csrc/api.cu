@@ -452,7 +452,7 @@ pasta_status_t pasta_decode_attn(pasta_pool_t *p, int32_t layer_begin, int32_t l
     uint8_t mask = 0;
     if (timed) PASTA_CUDA(cudaEventRecord(ev[0], st));
     if (p->hdr.w[PH_N_TUNITS] + p->hdr.w[PH_N_DUNITS] > 0) {
-      PASTA_CUDA(launch_attn_tensor(p->pv, p->hdr, layer_begin + done, cnt, qg, sc, st));
+      PASTA_CUDA(launch_attn_tensor(p->pv, p->hdr, layer_begin + done, cnt, qg, sc, og, lg, out_bf16, st));
       p->launches += 1;
       mask |= 1;
     }
@@ -741,6 +741,8 @@ pasta_status_t pasta_debug_set_tail(pasta_pool_t *p, int32_t percent, int32_t ti
   p->tail_tiles = tiles;
   return PASTA_OK;
 }
+
+void pasta_debug_set_launch_overlap(int32_t on) { set_launch_overlap(on != 0); }
 
 pasta_status_t pasta_debug_hold_roles(pasta_pool_t *p, int32_t role_mask) {
   if (!p || role_mask < 0 || role_mask > 31) return PASTA_ERR_INVALID_ARG;

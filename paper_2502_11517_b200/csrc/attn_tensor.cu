@@ -48,9 +48,9 @@ constexpr int B_FULL = 0, B_EMPTY = B_FULL + T_STAGES, B_SFULL = B_EMPTY + T_STA
               B_DRAIN = B_MLFULL + 1,  // only used when a role gave up: completion of the MMAs still in flight
               B_COUNT = B_DRAIN + 1;
 constexpr int OFF_META = OFF_BAR + 8 * ((B_COUNT + 1) & ~1);   // per stage: 8 page metas
-constexpr int T_RING = 16;                                     // shared units the producer may be ahead of the slowest role
+constexpr int T_RING = 8;                                      // unit records the producer keeps published (64 B each)
 constexpr int OFF_MISC = OFF_META + T_STAGES * 32;             // tmem base, abort flag, shared units taken, their ids
-constexpr int OFF_ML1 = OFF_MISC + 16 + 4 * T_RING;            // (m_ref, l) of group 1's rows, for the epilogue
+constexpr int OFF_ML1 = OFF_MISC + 16 + 64 * T_RING;           // (m_ref, l) of group 1's rows, for the epilogue
 constexpr int T_SMEM_USED = OFF_ML1 + 128 * 8;
 constexpr int T_SMEM_BYTES = T_SMEM_USED + 1024;               // slack to align the base to 1024
 static_assert(T_SMEM_BYTES <= 232448, "shared memory budget");
@@ -121,21 +121,45 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float *v) {
 #pragma unroll
   for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
-// 16 consecutive fp32 columns
-__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float *v) {
-  uint32_t r[16];
+// The same load without its wait, and the wait by itself, so that several loads can be in flight before one wait.  The
+// wait (and tmem_ld_order for a second register set) names the registers so that nothing that uses them can be
+// scheduled above it.
+__device__ __forceinline__ void tmem_ld32_issue(uint32_t taddr, uint32_t *r) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,"
+      "%29,%30,%31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+}
+#define PASTA_RW32(r)                                                                                                  \
+  "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]), "+r"(r[8]),          \
+  "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]), "+r"(r[16]), "+r"(r[17]),   \
+  "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]), "+r"(r[23]), "+r"(r[24]), "+r"(r[25]), "+r"(r[26]),  \
+  "+r"(r[27]), "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
+__device__ __forceinline__ void tmem_ld_wait32(uint32_t *r) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;" : PASTA_RW32(r) :: "memory");
+}
+__device__ __forceinline__ void tmem_ld_order32(uint32_t *r) { asm volatile("" : PASTA_RW32(r) :: "memory"); }
+// 16 consecutive fp32 columns, issued without the wait
+__device__ __forceinline__ void tmem_ld16_issue(uint32_t taddr, uint32_t *r) {
   asm volatile(
       "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
       : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
         "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
       : "r"(taddr)
       : "memory");
-  asm volatile("tcgen05.wait::ld.sync.aligned;"
-      : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]), "+r"(r[8]),
-        "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15])
-      :: "memory");
-#pragma unroll
-  for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+#define PASTA_RW16(r)                                                                                                  \
+  "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]), "+r"(r[8]),          \
+  "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15])
+// waits for every load of this thread in flight; names the registers of two of them
+__device__ __forceinline__ void tmem_ld_wait16x2(uint32_t *r0, uint32_t *r1) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;" : PASTA_RW16(r0), PASTA_RW16(r1) :: "memory");
 }
 __device__ __forceinline__ void tmem_st32(uint32_t taddr, const float *v) {
   uint32_t r[32];
@@ -212,7 +236,7 @@ __device__ __forceinline__ void bulk_g2s_stream(uint32_t dst, const void *src, u
 
 struct UnitInfo {
   int treq, g, tile_begin, tile_end, row_base;
-  int page_off, n_pages, n_threads, n_streams, vis_off, tq_off;
+  int page_off, n_pages, n_threads, n_streams, vis_off, tq_off, final_rows;
 };
 
 __device__ __forceinline__ UnitInfo load_unit(const int32_t *plan, int off_tunit, int off_treq, int u) {
@@ -222,7 +246,7 @@ __device__ __forceinline__ UnitInfo load_unit(const int32_t *plan, int off_tunit
   UnitInfo x;
   x.treq = a.x; x.g = a.y; x.tile_begin = a.z; x.tile_end = a.w;
   x.row_base = b.x; x.page_off = b.y; x.n_pages = b.z; x.n_threads = b.w;
-  x.n_streams = c.x; x.vis_off = c.y; x.tq_off = c.z;
+  x.n_streams = c.x; x.vis_off = c.y; x.tq_off = c.z; x.final_rows = c.w;
   return x;
 }
 
@@ -231,12 +255,19 @@ struct TensorArgs {
   int32_t off_dunit, n_dunits;      // units no CTA owns in advance (per layer): taken from a counter at run time
   int32_t n_queries, layer_begin, layer_count;
   float scale_log2;
+  void *out;                        // [layer_count, n_queries, Hq, 128], fp32 or bf16: rows of final units go here
+  float *lse;                       // [layer_count, n_queries, Hq] or null
+  int32_t out_bf16;
 };
 
-// A role's place in its CTA's sequence of units: first the units assigned to the CTA, layer by layer, then units of the
-// shared pool (the last tiles of the runs, kept back by the planner).  The producer takes the next shared unit from a
-// counter in global memory when it gets there, which is ahead of every other role, and publishes its number in a small
-// ring in shared memory; the other roles read the same numbers in the same order.  -1 ends the sequence.
+// A role's place in its CTA's sequence of units: first the units assigned to the CTA, layer by layer, whose records every
+// role reads from the plan itself; then units of the shared pool (whole short runs kept back by the planner), taken from
+// a counter in global memory.  Only the producer, which gets to every unit first, touches the counter: it publishes the
+// record (and layer) of each shared unit it takes in a ring of T_RING slots in shared memory, and the other roles read
+// the records from there in the same order, without a round trip to global memory at the start of a unit.  A record
+// with tile_end = 0 ends the sequence.  The producer is at most T_STAGES tiles, hence units, ahead of the tile whose
+// P.V has finished, and no role is a whole unit behind that one when it reads its next record, so a slot is not
+// overwritten before everybody has read it.
 struct Walk { int ll, u, k; };
 
 template <bool kProducer, bool kShared>
@@ -250,41 +281,55 @@ __device__ __forceinline__ bool next_unit(Walk &w, const TensorArgs &a, const in
     return true;
   }
   if (!kShared) return false;        // this build of the kernel serves plans without shared units
-  const int total = a.n_dunits * a.layer_count;
-  if (total == 0) return false;
-  int id = -1;
+  if (a.n_dunits == 0) return false;
+  int32_t *slot = const_cast<int32_t *>(reinterpret_cast<volatile int32_t *>(ring)) + 2 + 16 * (w.k % T_RING);
   if (kProducer) {
+    int id = -1;
     if (lane == 0) {
       id = atomicAdd(counter, 1);
-      if (id >= total) id = -1;
-      ring[2 + w.k % T_RING] = id;
+      if (id >= a.n_dunits * a.layer_count) id = -1;
+    }
+    id = __shfl_sync(0xffffffffu, id, 0);
+    if (id >= 0) {
+      ll = id / a.n_dunits;
+      x = load_unit(plan, a.off_dunit, 0, id - ll * a.n_dunits);
+    }
+    if (lane == 0) {
+      int4 *s4 = reinterpret_cast<int4 *>(slot);
+      s4[0] = make_int4(x.treq, x.g, x.tile_begin, id >= 0 ? x.tile_end : 0);
+      s4[1] = make_int4(x.row_base, x.page_off, x.n_pages, x.n_threads);
+      s4[2] = make_int4(x.n_streams, x.vis_off, x.tq_off, ll);
+      s4[3] = make_int4(x.final_rows, 0, 0, 0);
       __threadfence_block();
       ring[0] = w.k + 1;
     }
-    id = __shfl_sync(0xffffffffu, id, 0);
-  } else {
-    int got = 1;
-    if (!whole_warp || lane == 0) {
-      if (ring[0] <= w.k) {
-        const long long t0 = clock64();
-        while (ring[0] <= w.k) {
-          if (*abort_flag) { got = 0; break; }
-          if (clock64() - t0 > limit) { *abort_flag = 1; got = 0; break; }
-          __nanosleep(128);
-        }
+    ++w.k;
+    return id >= 0;
+  }
+  int got = 1;
+  if (!whole_warp || lane == 0) {
+    if (ring[0] <= w.k) {
+      const long long t0 = clock64();
+      while (ring[0] <= w.k) {
+        if (*abort_flag) { got = 0; break; }
+        if (clock64() - t0 > limit) { *abort_flag = 1; got = 0; break; }
+        __nanosleep(64);
       }
     }
-    if (whole_warp) {
-      got = __shfl_sync(0xffffffffu, got, 0);
-      __syncwarp();
-    }
-    if (!got) { ok = false; return false; }
-    id = ring[2 + w.k % T_RING];
   }
+  if (whole_warp) {
+    got = __shfl_sync(0xffffffffu, got, 0);
+    __syncwarp();
+  }
+  if (!got) { ok = false; return false; }
+  const int4 *s4 = reinterpret_cast<const int4 *>(slot);
+  const int4 ra = s4[0], rb = s4[1], rc = s4[2];
+  x.final_rows = s4[3].x;
   ++w.k;
-  if (id < 0) return false;
-  ll = id / a.n_dunits;
-  x = load_unit(plan, a.off_dunit, 0, id - ll * a.n_dunits);
+  if (ra.w == 0) return false;
+  x.treq = ra.x; x.g = ra.y; x.tile_begin = ra.z; x.tile_end = ra.w;
+  x.row_base = rb.x; x.page_off = rb.y; x.n_pages = rb.z; x.n_threads = rb.w;
+  x.n_streams = rc.x; x.vis_off = rc.y; x.tq_off = rc.z; ll = rc.w;
   return true;
 }
 
@@ -334,6 +379,10 @@ attn_tensor_kernel(PoolView pv, TensorArgs a, const __nv_bfloat16 *__restrict__ 
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = misc[0];
+  // everything above overlaps the end of the kernel ahead in the stream (the append of this step's tokens); from here on
+  // that kernel's writes are needed, and the kernels behind this one may start their own set-up
+  grid_dependency_wait();
+  grid_launch_dependents();
   const long long limit = pv.wait_limit;
   uint32_t prod_it = 0;       // warp 0: tiles whose copies have been issued
   volatile int *ring = reinterpret_cast<volatile int *>(misc + 2);
@@ -451,12 +500,15 @@ attn_tensor_kernel(PoolView pv, TensorArgs a, const __nv_bfloat16 *__restrict__ 
       UnitInfo x;
       int ll = 0;
       for (; ok && next_unit<false, kShared>(wk, a, plan, u0, u1, ring, counter, lane, true, abort_flag, limit, ok, x, ll); ++uc) {
-        if (uc > 0 && !warp_wait_or_abort(bar + 8 * B_QFREE, (uc - 1) & 1, abort_flag, limit)) { ok = false; break; }
         const int rows = x.n_threads * G;
-        // thread t64 builds rows 2 t64 and 2 t64 + 1; the 16 loads of a row are issued together before any store
+        // thread t64 builds rows t64 and 64 + t64.  The 16 loads of a row are issued together, and those of the first
+        // row before the wait for the operand buffer: the producer publishes a unit while the one before it is still
+        // being worked on, so a unit of up to 64 rows has its whole operand in registers by the time the last Q.K^T of
+        // its predecessor lets go of the buffer
 #pragma unroll 1
         for (int rr = 0; rr < 2; ++rr) {
-          const int row = t64 * 2 + rr;
+          const int row = rr * 64 + t64;
+          if (rr == 1 && rows <= 64) break;
           uint4 val[16];
           if (row < rows) {
             const int t = row / G, hl = row - t * G;
@@ -469,12 +521,14 @@ attn_tensor_kernel(PoolView pv, TensorArgs a, const __nv_bfloat16 *__restrict__ 
 #pragma unroll
             for (int c = 0; c < 16; ++c) val[c] = make_uint4(0, 0, 0, 0);
           }
+          if (rr == 0 && uc > 0 && !warp_wait_or_abort(bar + 8 * B_QFREE, (uc - 1) & 1, abort_flag, limit)) { ok = false; break; }
           const int r8 = row & 7;
           uint8_t *dst = sm + OFF_Q + (row >> 3) * 1024 + r8 * 128;
 #pragma unroll
           for (int c = 0; c < 16; ++c)
             *reinterpret_cast<uint4 *>(dst + (c >> 3) * 16384 + (((c & 7) ^ r8) << 4)) = val[c];
         }
+        if (!ok) break;
         fence_proxy_async();
         __syncwarp();
         if (lane == 0) mbar_arrive(bar + 8 * B_QFULL);
@@ -505,6 +559,8 @@ attn_tensor_kernel(PoolView pv, TensorArgs a, const __nv_bfloat16 *__restrict__ 
         const int32_t *visrow = plan + a.off_vis + x.vis_off + (active ? row / G : 0) * x.n_streams;
         // the row's visible lengths of the first four local streams stay in registers for the whole unit: a global
         // load per page would otherwise sit between two tiles of this group
+        // where the unit's rows go, in one register: the first partial row, or for a final unit ~(offset of its queries)
+        const int dest = x.final_rows ? ~x.tq_off : x.row_base;
         int vis0 = visrow[0];
         int vis1 = x.n_streams > 1 ? visrow[1] : 0;
         int vis2 = x.n_streams > 2 ? visrow[2] : 0;
@@ -558,8 +614,13 @@ attn_tensor_kernel(PoolView pv, TensorArgs a, const __nv_bfloat16 *__restrict__ 
           tc_fence_after();
           if (warp_active) {
             float sc[T_HALF];
-            tmem_ld32(tmem + lane_addr + col_s, sc);
-            tmem_ld32(tmem + lane_addr + col_s + 32, sc + 32);
+            {
+              uint32_t *raw_sc = reinterpret_cast<uint32_t *>(sc);      // both halves in flight before one wait
+              tmem_ld32_issue(tmem + lane_addr + col_s, raw_sc);
+              tmem_ld32_issue(tmem + lane_addr + col_s + 32, raw_sc + 32);
+              tmem_ld_wait32(raw_sc);
+              tmem_ld_order32(raw_sc + 32);
+            }
             if (!full) {
 #pragma unroll
               for (int j = 0; j < T_HALF; ++j)
@@ -619,6 +680,8 @@ attn_tensor_kernel(PoolView pv, TensorArgs a, const __nv_bfloat16 *__restrict__ 
         }
         if (!ok) break;
         // ---- epilogue: the unit's rows leave TMEM; group 0 folds group 1's accumulator into its own
+        // (the query a final unit's row belongs to: asked for before the wait, which outlasts the load)
+        const int qn_row = (grp == 0 && dest < 0 && active) ? __ldg(plan + a.off_tq + ~dest + row / G) : 0;
         if (!warp_wait_or_abort(bar + 8 * B_OFULL, uc & 1, abort_flag, limit)) { ok = false; break; }
         tc_fence_after();
         if (grp == 1) {
@@ -635,24 +698,47 @@ attn_tensor_kernel(PoolView pv, TensorArgs a, const __nv_bfloat16 *__restrict__ 
           const float f1 = other.y > 0.f ? fast_exp2(other.x - m_all) : 0.f;
           const float l_all = f0 * l + f1 * other.y;
           const bool any0 = __any_sync(0xffffffffu, f0 != 0.f), any1 = __any_sync(0xffffffffu, f1 != 0.f);
-          const int64_t prow = static_cast<int64_t>(ll) * pv.rows_per_layer + x.row_base + row;
-          if (active) pv.part_ml[prow] = make_float2(m_all, l_all);
+          // a final unit's rows are the result: normalised and written to the output here, with the arithmetic the
+          // merge applies to a row that has a single partial (weight 1, then times 1 / l)
+          const bool fin = dest < 0;
+          const int64_t prow = static_cast<int64_t>(ll) * pv.rows_per_layer + dest + row;
+          int64_t orow = 0;
+          float inv = 1.f;
+          if (fin) {
+            if (active) {
+              orow = (static_cast<int64_t>(ll) * a.n_queries + qn_row) * pv.n_q_heads + x.g * G + (row - (row / G) * G);
+              inv = l_all > 0.f ? 1.f / l_all : 0.f;
+              if (a.lse) a.lse[orow] = (m_all + log2f(l_all)) * 0.6931471805599453f;
+            }
+          } else if (active) {
+            pv.part_ml[prow] = make_float2(m_all, l_all);
+          }
+          const bool write = active && (fin || l_all > 0.f);      // an output row with nothing visible is written as zeros
+          // partial rows are multiplied by inv = 1 (exact); fp32 rows of either kind go to one address
+          float *orow_f32 = fin ? static_cast<float *>(a.out) + orow * 128 : pv.part_o + prow * 128;
 #pragma unroll 1
           for (int cb = 0; cb < 8; ++cb) {
-            float o0[16], o1[16];
-            if (any0) tmem_ld16(tmem + lane_addr + COL_O + cb * 16, o0);
-            if (any1) tmem_ld16(tmem + lane_addr + COL_O + 128 + cb * 16, o1);
-            if (active && l_all > 0.f) {
-              float4 *dst = reinterpret_cast<float4 *>(pv.part_o + prow * 128 + cb * 16);
+            // 16 columns of both accumulators in flight before one wait
+            uint32_t q0[16], q1[16];
+            if (any0) tmem_ld16_issue(tmem + lane_addr + COL_O + cb * 16, q0);
+            if (any1) tmem_ld16_issue(tmem + lane_addr + COL_O + 128 + cb * 16, q1);
+            tmem_ld_wait16x2(q0, q1);
+            if (write) {
+              // a factor of exactly 0 means that accumulator was never written for this row: do not touch it
+              float r[16];
 #pragma unroll
-              for (int j = 0; j < 4; ++j) {
-                float4 r4;
-                // a factor of exactly 0 means that accumulator was never written for this row: do not touch it
-                r4.x = (f0 != 0.f ? f0 * o0[4 * j] : 0.f) + (f1 != 0.f ? f1 * o1[4 * j] : 0.f);
-                r4.y = (f0 != 0.f ? f0 * o0[4 * j + 1] : 0.f) + (f1 != 0.f ? f1 * o1[4 * j + 1] : 0.f);
-                r4.z = (f0 != 0.f ? f0 * o0[4 * j + 2] : 0.f) + (f1 != 0.f ? f1 * o1[4 * j + 2] : 0.f);
-                r4.w = (f0 != 0.f ? f0 * o0[4 * j + 3] : 0.f) + (f1 != 0.f ? f1 * o1[4 * j + 3] : 0.f);
-                dst[j] = r4;
+              for (int j = 0; j < 16; ++j)
+                r[j] = ((f0 != 0.f ? f0 * __uint_as_float(q0[j]) : 0.f) + (f1 != 0.f ? f1 * __uint_as_float(q1[j]) : 0.f)) * inv;
+              if (fin && a.out_bf16) {
+                uint4 *dst = reinterpret_cast<uint4 *>(static_cast<__nv_bfloat16 *>(a.out) + orow * 128 + cb * 16);
+#pragma unroll
+                for (int j = 0; j < 2; ++j)
+                  dst[j] = make_uint4(pack_bf16(r[8 * j], r[8 * j + 1]), pack_bf16(r[8 * j + 2], r[8 * j + 3]),
+                                      pack_bf16(r[8 * j + 4], r[8 * j + 5]), pack_bf16(r[8 * j + 6], r[8 * j + 7]));
+              } else {
+                float4 *dst = reinterpret_cast<float4 *>(orow_f32 + cb * 16);
+#pragma unroll
+                for (int j = 0; j < 4; ++j) dst[j] = make_float4(r[4 * j], r[4 * j + 1], r[4 * j + 2], r[4 * j + 3]);
               }
             }
           }
@@ -694,7 +780,7 @@ attn_tensor_kernel(PoolView pv, TensorArgs a, const __nv_bfloat16 *__restrict__ 
 bool tensor_path_available() { return true; }
 
 cudaError_t launch_attn_tensor(const PoolView &pv, const PlanHeader &h, int32_t layer_begin, int32_t layer_count,
-                               const void *q, float scale_log2, cudaStream_t st) {
+                               const void *q, float scale_log2, void *out, float *lse, bool out_bf16, cudaStream_t st) {
   if (pv.head_dim != 128) return cudaErrorInvalidValue;
   static uint64_t prepared[2] = {0, 0};
   const bool shared_units = h.w[PH_N_DUNITS] > 0;
@@ -713,10 +799,10 @@ cudaError_t launch_attn_tensor(const PoolView &pv, const PlanHeader &h, int32_t 
   a.off_dunit = h.w[PH_OFF_DUNIT]; a.n_dunits = h.w[PH_N_DUNITS];
   a.n_queries = h.w[PH_N_QUERIES]; a.layer_begin = layer_begin; a.layer_count = layer_count;
   a.scale_log2 = scale_log2;
+  a.out = out; a.lse = lse; a.out_bf16 = out_bf16 ? 1 : 0;
   // two builds of the kernel: the one without the shared part of the walk is a little faster (0.7 % on long runs)
-  if (shared_units) attn_tensor_kernel<true><<<grid, T_THREADS, T_SMEM_BYTES, st>>>(pv, a, static_cast<const __nv_bfloat16 *>(q));
-  else attn_tensor_kernel<false><<<grid, T_THREADS, T_SMEM_BYTES, st>>>(pv, a, static_cast<const __nv_bfloat16 *>(q));
-  return cudaGetLastError();
+  return launch_overlapped(shared_units ? attn_tensor_kernel<true> : attn_tensor_kernel<false>, dim3(grid), dim3(T_THREADS),
+                           T_SMEM_BYTES, st, pv, a, static_cast<const __nv_bfloat16 *>(q));
 }
 
 }  // namespace pasta

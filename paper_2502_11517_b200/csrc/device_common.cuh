@@ -49,6 +49,16 @@ __device__ __forceinline__ void report(int32_t *status, int32_t code) { atomicMa
 // are the sink of the read-only measurement kernels.
 #define PASTA_STATUS_TAIL_COUNTER 8
 
+// Overlap of consecutive launches of a step (programmatic dependent launch).  A kernel launched with launch_overlapped()
+// may start while the kernel before it in the stream is still running, once every CTA of that kernel has called
+// grid_launch_dependents() or has exited; it must call grid_dependency_wait(), in every thread and before its first
+// access to anything the earlier kernel reads or writes, which returns when the earlier kernel has completed and its
+// writes are visible.  What runs before that call (barrier set-up, TMEM allocation, the launch itself) is hidden behind
+// the earlier kernel's last CTAs.  Each kernel waits before it lets its own successor go, so that the completion of a
+// kernel implies that of all its predecessors.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // ---------------------------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void *p) {
   return static_cast<uint32_t>(__cvta_generic_to_shared(p));

@@ -5,7 +5,14 @@
 
 #include <cmath>
 
+#include <atomic>
+
 namespace pasta {
+
+static std::atomic<bool> g_launch_overlap{true};
+bool launch_overlap_enabled() { return g_launch_overlap.load(std::memory_order_relaxed); }
+void set_launch_overlap(bool on) { g_launch_overlap.store(on, std::memory_order_relaxed); }
+
 
 // =============================================================================================
 // K1: KV append.  One thread moves one 16-byte chunk (8 bf16) of K or V of one token.
@@ -13,6 +20,7 @@ namespace pasta {
 __global__ void kv_append_kernel(PoolView pv, const int32_t *__restrict__ slots, int32_t n_tok,
                                  int32_t layer_begin, int32_t layer_count,
                                  const uint4 *__restrict__ k_new, const uint4 *__restrict__ v_new) {
+  grid_launch_dependents();       // the attention kernel may set itself up meanwhile; it waits for this grid to finish
   const int chunks = pv.head_dim >> 3;
   const int64_t total = static_cast<int64_t>(layer_count) * n_tok * pv.n_kv_heads * 2 * chunks;
   const int64_t idx = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
@@ -98,6 +106,7 @@ __device__ __forceinline__ void rope_apply(uint4 &lo, uint4 &hi, const double *s
 __global__ void kv_append_rope_kernel(PoolView pv, const int32_t *__restrict__ slots, const int32_t *__restrict__ pos,
                                       int32_t pos0, int32_t n_tok, int32_t layer_begin, int32_t layer_count,
                                       const uint4 *__restrict__ k_new, const uint4 *__restrict__ v_new, double log2_theta) {
+  grid_launch_dependents();
   const int chunks = pv.head_dim >> 3, half_chunks = chunks >> 1;
   const int64_t n_k = static_cast<int64_t>(layer_count) * n_tok * half_chunks;
   const int64_t n_v = n_k * pv.n_kv_heads;
@@ -141,6 +150,7 @@ __global__ void kv_append_rope_kernel(PoolView pv, const int32_t *__restrict__ s
 // (layer, query, chunk pair), all heads of the query in turn
 __global__ void rope_queries_kernel(const int32_t *__restrict__ pos, int32_t n, int32_t n_q_heads, int32_t D,
                                     int32_t layer_count, uint4 *__restrict__ q, double log2_theta) {
+  grid_launch_dependents();
   const int chunks = D >> 3, half_chunks = chunks >> 1;
   const int64_t total = static_cast<int64_t>(layer_count) * n * half_chunks;
   const int64_t idx = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
@@ -344,6 +354,8 @@ attn_warp_kernel(PoolView pv, int32_t off_wunit, int32_t off_pages, int32_t n_wu
   constexpr int E = D / 32;            // output elements per lane
   constexpr int CH = D / 16;           // 16-byte chunks of a K row handled by one lane
   extern __shared__ __align__(1024) uint8_t smem_raw[];
+  grid_dependency_wait();         // the kernel ahead in the stream (append or tensor-core pass) has completed
+  grid_launch_dependents();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int64_t gw = static_cast<int64_t>(blockIdx.x) * W_WARPS + warp;
   if (gw >= static_cast<int64_t>(n_wunits) * layer_count) return;
@@ -513,10 +525,9 @@ static cudaError_t launch_warp_t(const PoolView &pv, const PlanHeader &h, int32_
   const int64_t warps = static_cast<int64_t>(h.w[PH_N_WUNITS]) * layer_count;
   if (warps == 0) return cudaSuccess;
   const int64_t blocks = (warps + W_WARPS - 1) / W_WARPS;
-  attn_warp_kernel<D, G><<<static_cast<unsigned>(blocks), W_WARPS * 32, S::TOTAL, st>>>(
-      pv, h.w[PH_OFF_WUNIT], h.w[PH_OFF_PAGES], h.w[PH_N_WUNITS], h.w[PH_T_ROWS], h.w[PH_N_QUERIES], layer_begin,
-      layer_count, static_cast<const __nv_bfloat16 *>(q), scale_log2);
-  return cudaGetLastError();
+  return launch_overlapped(attn_warp_kernel<D, G>, dim3(static_cast<unsigned>(blocks)), dim3(W_WARPS * 32), S::TOTAL, st, pv,
+                           h.w[PH_OFF_WUNIT], h.w[PH_OFF_PAGES], h.w[PH_N_WUNITS], h.w[PH_T_ROWS], h.w[PH_N_QUERIES],
+                           layer_begin, layer_count, static_cast<const __nv_bfloat16 *>(q), scale_log2);
 }
 
 cudaError_t launch_attn_warp(const PoolView &pv, const PlanHeader &h, int32_t layer_begin, int32_t layer_count,
@@ -541,6 +552,7 @@ __global__ void __launch_bounds__(256)
 merge_kernel(PoolView pv, int32_t n_queries, int32_t layer_count, int32_t off_query, int32_t off_trange,
              int32_t off_tunit, int32_t off_drange, int32_t off_dunit, int32_t t_rows, int32_t layers_per_warp,
              void *__restrict__ out_raw, float *__restrict__ lse) {
+  grid_dependency_wait();         // every partial row has been written
   // the tensor-core kernel of this launch group is over: its counter of shared units starts from zero next time
   if (blockIdx.x == 0 && threadIdx.x == 0) pv.status[PASTA_STATUS_TAIL_COUNTER] = 0;
   const int D = pv.head_dim, Hq = pv.n_q_heads, G = Hq / pv.n_kv_heads;
@@ -561,6 +573,10 @@ merge_kernel(PoolView pv, int32_t n_queries, int32_t layer_count, int32_t off_qu
     nt = pv.plan[off_trange + (treq * pv.n_kv_heads + g) * 2 + 1] - tb;
     db = pv.plan[off_drange + (treq * pv.n_kv_heads + g) * 2];
     nd = pv.plan[off_drange + (treq * pv.n_kv_heads + g) * 2 + 1] - db;
+  }
+  if (nw == 0 && nt + nd == 1) {            // a final unit has written this pair's result itself
+    const int32_t *rec = nt ? pv.plan + off_tunit + tb * PU_WORDS : pv.plan + off_dunit + db * PU_WORDS;
+    if (rec[PU_FINAL]) return;
   }
   const int total = nt + nd + nw;
   auto row_of = [&](int i) -> int64_t {     // within one layer: assigned units, shared units, warp-shuffle pieces
@@ -648,15 +664,9 @@ cudaError_t launch_merge(const PoolView &pv, const PlanHeader &h, int32_t layer_
   const int32_t layers_per_warp = static_cast<int32_t>((layer_count + groups - 1) / groups);
   const int64_t warps = per_group * ((layer_count + layers_per_warp - 1) / layers_per_warp);
   const int64_t blocks = (warps * 32 + 255) / 256;
-  if (out_bf16)
-    merge_kernel<true><<<static_cast<unsigned>(blocks), 256, 0, st>>>(pv, h.w[PH_N_QUERIES], layer_count, h.w[PH_OFF_QUERY],
-                                                                      h.w[PH_OFF_TRANGE], h.w[PH_OFF_TUNIT], h.w[PH_OFF_DRANGE],
-                                                                      h.w[PH_OFF_DUNIT], h.w[PH_T_ROWS], layers_per_warp, out, lse);
-  else
-    merge_kernel<false><<<static_cast<unsigned>(blocks), 256, 0, st>>>(pv, h.w[PH_N_QUERIES], layer_count, h.w[PH_OFF_QUERY],
-                                                                       h.w[PH_OFF_TRANGE], h.w[PH_OFF_TUNIT], h.w[PH_OFF_DRANGE],
-                                                                       h.w[PH_OFF_DUNIT], h.w[PH_T_ROWS], layers_per_warp, out, lse);
-  return cudaGetLastError();
+  return launch_overlapped(out_bf16 ? merge_kernel<true> : merge_kernel<false>, dim3(static_cast<unsigned>(blocks)), dim3(256), 0,
+                           st, pv, h.w[PH_N_QUERIES], layer_count, h.w[PH_OFF_QUERY], h.w[PH_OFF_TRANGE], h.w[PH_OFF_TUNIT],
+                           h.w[PH_OFF_DRANGE], h.w[PH_OFF_DUNIT], h.w[PH_T_ROWS], layers_per_warp, out, lse);
 }
 
 }  // namespace pasta

@@ -25,6 +25,25 @@ inline cudaError_t raise_smem_limit(const void *kernel, int bytes, uint64_t *don
   return cudaSuccess;
 }
 
+// Launches `kernel` so that it may start before the kernel ahead of it in the stream has drained (see
+// grid_dependency_wait in device_common.cuh); with overlap switched off (pasta_debug_set_launch_overlap) an ordinary launch.
+bool launch_overlap_enabled();
+void set_launch_overlap(bool on);
+template <typename... KArgs, typename... Args>
+cudaError_t launch_overlapped(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args &&...args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = launch_overlap_enabled() ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 // K1: copies the new tokens of `layer_count` layers into their slots.  slots: device, 2 words per token.
 cudaError_t launch_kv_append(const PoolView &pv, const int32_t *slots, int32_t n_tok, int32_t layer_begin,
                              int32_t layer_count, const void *k_new, const void *v_new, cudaStream_t st);
@@ -41,9 +60,10 @@ cudaError_t launch_rope_queries(const PoolView &pv, const int32_t *pos, int32_t 
 // K3: warp-shuffle pass for requests the tensor-core kernel does not take (other head sizes, too many rows or streams)
 cudaError_t launch_attn_warp(const PoolView &pv, const PlanHeader &h, int32_t layer_begin, int32_t layer_count,
                              const void *q, float scale_log2, cudaStream_t st);
-// K2: tensor-core pass over all streams of a request whose stacked queries fit 128 rows (head_dim 128 only)
+// K2: tensor-core pass over all streams of a request whose stacked queries fit 128 rows (head_dim 128 only).  Rows of
+// units the plan marks final go straight to out / lse (the layout launch_merge writes), all others to the partial rows.
 cudaError_t launch_attn_tensor(const PoolView &pv, const PlanHeader &h, int32_t layer_begin, int32_t layer_count,
-                               const void *q, float scale_log2, cudaStream_t st);
+                               const void *q, float scale_log2, void *out, float *lse, bool out_bf16, cudaStream_t st);
 bool tensor_path_available();       // false while the tensor-core kernel is compiled out
 // test kernel: a bounded wait that runs out (one warp, PoolView::wait_limit cycles), reported as PASTA_ERR_TIMEOUT
 cudaError_t launch_wait_expiry(const PoolView &pv, cudaStream_t st);

@@ -12,7 +12,9 @@
 //              tiles of PASTA_TILE_PAGES pages; rows of the score matrix are the request's queries
 //              times the `group` query heads of one kv head: row = t_idx * group + h_local.
 //   t-unit     (t-request, kv head, tile range): one CTA-sized piece of the tensor-core kernel; it
-//              writes one partial result (m, l, O[d]) per row.
+//              writes one partial result (m, l, O[d]) per row.  A unit that covers all tiles of its (t-request, kv
+//              head) run, of a request none of whose queries has w-units, is FINAL: its rows are the result, the
+//              kernel normalises them and writes them to the output itself, and the merge skips them.
 //   d-unit     a t-unit that belongs to no CTA in advance: of the short (t-request, kv head) runs, every so often a
 //              whole one is kept back; the CTAs take these from a shared counter once their own units are done, so
 //              that SMs that stream faster than others end up doing more of the work.  Same record as a t-unit.
@@ -101,7 +103,7 @@ enum {
   PU_N_STREAMS,
   PU_VIS_OFF,
   PU_TQ_OFF,
-  PU_PAD,
+  PU_FINAL,           // 1: the unit's rows are the whole result of their (query, head) pairs
   PU_WORDS
 };
 static_assert(PU_WORDS == 12, "t-unit records are read as three int4");

@@ -349,18 +349,18 @@ pasta_status_t build_plan(const HostPool &pool, const std::vector<StepQuery> &en
     const int32_t rec[PT_WORDS] = {t.page_off, t.n_pages, t.n_threads, t.n_streams, t.vis_off, t.tq_off};
     ttab.insert(ttab.end(), rec, rec + PT_WORDS);
   }
-  for (const TUnit &u : tunits) {
+  // a unit is final when nothing else contributes to its rows: it covers its whole run, and no query of its request
+  // has streams on the warp path
+  auto unit_record = [&](const TUnit &u, std::vector<int32_t> &tab) {
     const TReq &t = treqs[u.treq];
+    bool final_rows = u.tile_begin == 0 && u.tile_end == (t.n_pages + PASTA_TILE_PAGES - 1) / PASTA_TILE_PAGES;
+    for (int32_t ti = 0; final_rows && ti < t.n_threads; ++ti) final_rows = q_nw[tq_tab[t.tq_off + ti]] == 0;
     const int32_t rec[PU_WORDS] = {u.treq, u.g, u.tile_begin, u.tile_end, u.row_base, t.page_off, t.n_pages,
-                                   t.n_threads, t.n_streams, t.vis_off, t.tq_off, 0};
-    utab.insert(utab.end(), rec, rec + PU_WORDS);
-  }
-  for (const TUnit &u : dunits) {
-    const TReq &t = treqs[u.treq];
-    const int32_t rec[PU_WORDS] = {u.treq, u.g, u.tile_begin, u.tile_end, u.row_base, t.page_off, t.n_pages,
-                                   t.n_threads, t.n_streams, t.vis_off, t.tq_off, 0};
-    dtab.insert(dtab.end(), rec, rec + PU_WORDS);
-  }
+                                   t.n_threads, t.n_streams, t.vis_off, t.tq_off, final_rows ? 1 : 0};
+    tab.insert(tab.end(), rec, rec + PU_WORDS);
+  };
+  for (const TUnit &u : tunits) unit_record(u, utab);
+  for (const TUnit &u : dunits) unit_record(u, dtab);
   w[PH_MAGIC] = PASTA_PLAN_MAGIC;
   w[PH_N_DUNITS] = static_cast<int32_t>(dunits.size());
   w[PH_N_QUERIES] = n;

@@ -1,6 +1,7 @@
 """Executes a step plan (the int32 words pasta_step_begin uploads) with NumPy, unit by unit, the way
 the kernels are meant to: every t-unit and w-unit yields partial (m, l, O) rows, the merge combines
-them.  It lets the planner be checked against the oracle without a GPU.  Tests only."""
+them; the rows of a unit marked final go to the output as they are, and must then be the only rows of their
+(query, head) pairs.  It lets the planner be checked against the oracle without a GPU.  Tests only."""
 import numpy as np
 
 # header word indices (pasta_plan.h)
@@ -35,6 +36,8 @@ def run_plan(w, K, V, q, n_kv_heads):
     recs += [w[w[PH_OFF_DUNIT] + u * PU: w[PH_OFF_DUNIT] + (u + 1) * PU] for u in range(w[PH_N_DUNITS])]
     STATS['dunits'] = STATS.get('dunits', 0) + int(w[PH_N_DUNITS])
     covered = {}
+    final = set()                           # partial rows that are the whole result of their (query, head) pair
+    STATS['final_units'] = STATS.get('final_units', 0) + sum(int(rec[11]) for rec in recs)
     for u, rec in enumerate(recs):
         treq, g, tb, te, row_base = rec[:5]
         T = w[PH_OFF_TREQ] + treq * PT
@@ -60,6 +63,9 @@ def run_plan(w, K, V, q, n_kv_heads):
                 s = np.concatenate(s_all); v = np.concatenate(v_all)
                 row = row_base + ti * G + hl
                 written[row] += 1
+                assert rec[11] in (0, 1)
+                if rec[11]:
+                    final.add(int(row))
                 if len(s) == 0:
                     m[row], l[row], O[row] = -np.inf, 0.0, 0.0
                 else:
@@ -99,6 +105,11 @@ def run_plan(w, K, V, q, n_kv_heads):
                     assert w[w[PH_OFF_DUNIT] + u * PU] == treq and w[w[PH_OFF_DUNIT] + u * PU + 1] == g
                     rows_i.append(w[w[PH_OFF_DUNIT] + u * PU + 4] + tidx * G + hl)
             rows_i += [t_rows + (w0 + g * nw + k) * G + hl for k in range(nw)]
+            if any(int(r) in final for r in rows_i):      # written by the unit itself: nothing else may contribute
+                assert len(rows_i) == 1
+            elif len(rows_i) == 1 and nw == 0:            # a lone unit is final unless its request has w-units
+                qt = w[w[PH_OFF_QUERY]: w[PH_OFF_QUERY] + n * PQ].reshape(n, PQ)
+                assert np.any(qt[qt[:, 0] == treq, 3] > 0)
             rows_i = [r for r in rows_i if l[r] > 0]
             ms = max(m[r] for r in rows_i)
             L = sum(np.exp(m[r] - ms) * l[r] for r in rows_i)

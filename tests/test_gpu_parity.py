@@ -322,3 +322,74 @@ def test_units_shared_out_at_run_time_short_runs_three_layers(lib):
     unit is a (layer, unit) pair.  Two launches in a row: the counter starts from zero each time."""
     run_script(lib, cfg3_batched(64, 3, n_new=1), tail=(20, 3))
     run_script(lib, cfg3_batched(64, 3), tail=(20, 3), max_layers_per_launch=2)
+
+
+def _one_step(lib, script, flags=0, overlap=True, want_lse=True):
+    """Replays `script` up to its last step and runs that step through pasta_step_device; returns out, lse, plan words."""
+    import torch
+    from lib_replay import LibReplay, make_pool
+    lib.Pool.debug_set_launch_overlap(overlap)
+    try:
+        pool = make_pool(script, flags=flags)
+        rep = LibReplay(script, pool)
+        last = max(i for i, op in enumerate(script.ops) if op[0] == "step")
+        for i in range(last):
+            rep.apply(i, attend=False)
+        op = script.ops[last]
+        L = range(script.geometry.n_layers)
+        ks, vs, qs = zip(*[step_tensors(script, last, l) for l in L])
+        k = torch.stack(ks).cuda(); v = torch.stack(vs).cuda(); q = torch.stack(qs).cuda()
+        out = torch.full(q.shape, float("nan"), dtype=torch.bfloat16 if flags & lib.FLAG_OUT_BF16 else torch.float32, device="cuda")
+        lse = torch.full(q.shape[:3], float("nan"), dtype=torch.float32, device="cuda") if want_lse else None
+        pool.step_device([e[0] for e in op[1]], [e[1] for e in op[1]], [e[2] for e in op[1]], k, v, q, out, lse)
+        torch.cuda.synchronize()
+        assert pool.status() == 0
+        words = np.array(pool.plan_words())
+        pool.close()
+        return out.cpu(), None if lse is None else lse.cpu(), words
+    finally:
+        lib.Pool.debug_set_launch_overlap(True)
+
+
+def _final_flags(words):
+    """The final marks of a plan's assigned and shared units (word 11 of every 12-word record)."""
+    t = words[words[13]: words[13] + 12 * words[4]].reshape(-1, 12)[:, 11]
+    d = words[words[24]: words[24] + 12 * words[23]].reshape(-1, 12)[:, 11]
+    return np.concatenate([t, d])
+
+
+def test_a_step_with_final_and_merged_rows(lib):
+    """The batched configuration cuts some of its runs at CTA boundaries and leaves most whole: whole runs are final
+    units, whose rows the tensor-core kernel writes to the output itself, the rest goes through partial rows and the
+    merge.  Every output element is written by exactly one of the two (none stays NaN), both equal the oracle's, with
+    fp32 and bf16 outputs (bf16 = the fp32 result rounded once), with and without a log-sum-exp output."""
+    import torch
+    script = cfg3_batched(64, 2, n_new=1)
+    out32, lse32, words = _one_step(lib, script)
+    fin = _final_flags(words)
+    assert 0 < fin.sum() < len(fin), "the step should mix final and merged units"
+    ora = OracleReplay(script, layers=[0, 1])
+    last = max(i for i, op in enumerate(script.ops) if op[0] == "step")
+    for i in range(last):
+        ora.apply(i, attend=False)
+    want = ora.apply(last)
+    for l in (0, 1):
+        compare(out32[l], lse32[l], want[l][0], want[l][1], f"layer {l}")
+    out16, lse16, _ = _one_step(lib, script, flags=lib.FLAG_OUT_BF16)
+    assert torch.equal(out32.to(torch.bfloat16), out16) and torch.equal(lse32, lse16)
+    out_nolse, _, _ = _one_step(lib, script, want_lse=False)
+    assert torch.equal(out_nolse, out32)
+
+
+@pytest.mark.parametrize("maker", [lambda: cfg3_batched(64, 3, n_new=1), lambda: cfg4_long_prefix(4, 3000, 6, n_new=1),
+                                   lambda: random_script(3, n_ops=80, geo=Geometry(2, 4, 2, 64, 16))])
+def test_launch_overlap_does_not_change_results(lib, maker):
+    """The kernels of a step launched so that each sets itself up while the one ahead drains, against the same step
+    launched strictly in sequence: identical bits (tensor-core path with several layers per launch, long runs with a
+    merge, and the warp-shuffle path)."""
+    import torch
+    script = maker()
+    a = _one_step(lib, script, overlap=True)
+    b = _one_step(lib, script, overlap=False)
+    assert torch.equal(a[0], b[0]) and torch.equal(a[1], b[1])
+    assert not torch.isnan(a[0]).any() and not torch.isnan(a[1]).any()

@@ -142,6 +142,21 @@ def test_shared_tail_is_dropped_when_it_does_not_fit():
     assert plan(None, max_partial_rows=rows_without + 8) == (rows_without, 0)
 
 
+def test_final_units_are_marked_and_only_those():
+    """Short runs fit one unit each: the plan marks such units final (their rows are the result, the merge skips them),
+    the interpreter checks that a final row is the only row of its (query, head) pair
+    and that every lone row is marked.  With runs cut in several pieces by a small grid's worth of work, cut runs stay
+    unmarked."""
+    from plan_interpreter import STATS
+    before = STATS.get("final_units", 0)
+    stats = check_script(cfg3_batched(20, 1, prefix_range=(64, 700)))
+    marked = STATS["final_units"] - before
+    assert 0 < marked <= stats["tunits"]
+    before = STATS["final_units"]
+    stats = check_script(cfg4_long_prefix(2, 3000, 3))            # 16 runs of 24 tiles over 148 CTAs: every run is cut
+    assert STATS["final_units"] == before and stats["tunits"] > 16
+
+
 def test_zz_all_visible_page_flag_is_exercised():
     """The plans interpreted above marked some pages as visible in full to every thread (checked page by page in
     plan_interpreter.run_plan) and left others unmarked."""
