@@ -195,6 +195,13 @@ __device__ __forceinline__ void fma2(float &x0, float &x1, float a0, float a1, f
       "fma.rn.f32x2 rd, ra, rb, rc;\n\tmov.b64 {%0, %1}, rd;\n\t}"
       : "=f"(x0), "=f"(x1) : "f"(a0), "f"(a1), "f"(b), "f"(c));
 }
+// {x0, x1} = {a0, a1} * {b, b} + {c0, c1}
+__device__ __forceinline__ void fma2v(float &x0, float &x1, float a0, float a1, float b, float c0, float c1) {
+  asm("{\n\t.reg .b64 ra, rb, rc, rd;\n\t"
+      "mov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %4};\n\tmov.b64 rc, {%5, %6};\n\t"
+      "fma.rn.f32x2 rd, ra, rb, rc;\n\tmov.b64 {%0, %1}, rd;\n\t}"
+      : "=f"(x0), "=f"(x1) : "f"(a0), "f"(a1), "f"(b), "f"(c0), "f"(c1));
+}
 // {s0, s1} += {p0, p1}
 __device__ __forceinline__ void add2(float &s0, float &s1, float p0, float p1) {
   asm("{\n\t.reg .b64 ra, rb, rd;\n\t"
@@ -714,8 +721,16 @@ attn_tensor_kernel(PoolView pv, TensorArgs a, const __nv_bfloat16 *__restrict__ 
             pv.part_ml[prow] = make_float2(m_all, l_all);
           }
           const bool write = active && (fin || l_all > 0.f);      // an output row with nothing visible is written as zeros
-          // partial rows are multiplied by inv = 1 (exact); fp32 rows of either kind go to one address
+          // partial rows keep inv = 1; fp32 rows of either kind go to one address
           float *orow_f32 = fin ? static_cast<float *>(a.out) + orow * 128 : pv.part_o + prow * 128;
+          // One warp per scheduler is at work here and every instruction waits for the one before it, so the epilogue
+          // costs what its instruction count says.  The usual case, where every row of the warp has weights in both
+          // accumulators (or all of them only in the first), takes two (one) packed instructions per pair of columns;
+          // the general case guards each product: a factor of exactly 0 means that accumulator was never written for
+          // this row, and whatever TMEM holds there must not be touched.
+          const float g0 = f0 * inv, g1 = f1 * inv;
+          const bool both = __all_sync(0xffffffffu, !active || (f0 != 0.f && f1 != 0.f));
+          const bool only0 = !both && __all_sync(0xffffffffu, !active || (f0 != 0.f && f1 == 0.f));
 #pragma unroll 1
           for (int cb = 0; cb < 8; ++cb) {
             // 16 columns of both accumulators in flight before one wait
@@ -723,12 +738,23 @@ attn_tensor_kernel(PoolView pv, TensorArgs a, const __nv_bfloat16 *__restrict__ 
             if (any0) tmem_ld16_issue(tmem + lane_addr + COL_O + cb * 16, q0);
             if (any1) tmem_ld16_issue(tmem + lane_addr + COL_O + 128 + cb * 16, q1);
             tmem_ld_wait16x2(q0, q1);
-            if (write) {
-              // a factor of exactly 0 means that accumulator was never written for this row: do not touch it
-              float r[16];
+            float r[16];
+            if (both) {
+#pragma unroll
+              for (int j = 0; j < 16; j += 2) {
+                float t0, t1;
+                fma2(t0, t1, __uint_as_float(q1[j]), __uint_as_float(q1[j + 1]), g1, 0.f);
+                fma2v(r[j], r[j + 1], __uint_as_float(q0[j]), __uint_as_float(q0[j + 1]), g0, t0, t1);
+              }
+            } else if (only0) {
+#pragma unroll
+              for (int j = 0; j < 16; j += 2) fma2(r[j], r[j + 1], __uint_as_float(q0[j]), __uint_as_float(q0[j + 1]), g0, 0.f);
+            } else {
 #pragma unroll
               for (int j = 0; j < 16; ++j)
-                r[j] = ((f0 != 0.f ? f0 * __uint_as_float(q0[j]) : 0.f) + (f1 != 0.f ? f1 * __uint_as_float(q1[j]) : 0.f)) * inv;
+                r[j] = (f0 != 0.f ? g0 * __uint_as_float(q0[j]) : 0.f) + (f1 != 0.f ? g1 * __uint_as_float(q1[j]) : 0.f);
+            }
+            if (write) {
               if (fin && a.out_bf16) {
                 uint4 *dst = reinterpret_cast<uint4 *>(static_cast<__nv_bfloat16 *>(a.out) + orow * 128 + cb * 16);
 #pragma unroll
