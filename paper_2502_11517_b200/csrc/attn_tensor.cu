@@ -349,6 +349,8 @@ attn_tensor_kernel(PoolView pv, TensorArgs a, const __nv_bfloat16 *__restrict__ 
   uint8_t *sm = smem_raw + (base - raw);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int G = pv.n_q_heads / pv.n_kv_heads;
+  // row / G sits between two units for every role: a shift when G is a power of two (it usually is), the division otherwise
+  auto div_g = [&](int r) { return (G & (G - 1)) == 0 ? r >> (31 - __clz(G)) : r / G; };
   const uint32_t bar = base + OFF_BAR;
   int32_t *meta_s = reinterpret_cast<int32_t *>(sm + OFF_META);
   uint32_t *misc = reinterpret_cast<uint32_t *>(sm + OFF_MISC);
@@ -518,7 +520,7 @@ attn_tensor_kernel(PoolView pv, TensorArgs a, const __nv_bfloat16 *__restrict__ 
           if (rr == 1 && rows <= 64) break;
           uint4 val[16];
           if (row < rows) {
-            const int t = row / G, hl = row - t * G;
+            const int t = div_g(row), hl = row - t * G;
             const int qn = plan[a.off_tq + x.tq_off + t];
             const uint4 *src = reinterpret_cast<const uint4 *>(
                 q + ((static_cast<int64_t>(ll) * a.n_queries + qn) * pv.n_q_heads + x.g * G + hl) * 128);
@@ -563,7 +565,7 @@ attn_tensor_kernel(PoolView pv, TensorArgs a, const __nv_bfloat16 *__restrict__ 
         const int row = m64 ? (lane < 16 ? wq * 16 + lane : 128) : wq * 32 + lane;
         const bool active = row < rows;
         const bool warp_active = (m64 ? wq * 16 : wq * 32) < rows;
-        const int32_t *visrow = plan + a.off_vis + x.vis_off + (active ? row / G : 0) * x.n_streams;
+        const int32_t *visrow = plan + a.off_vis + x.vis_off + (active ? div_g(row) : 0) * x.n_streams;
         // the row's visible lengths of the first four local streams stay in registers for the whole unit: a global
         // load per page would otherwise sit between two tiles of this group
         // where the unit's rows go, in one register: the first partial row, or for a final unit ~(offset of its queries)
@@ -688,7 +690,7 @@ attn_tensor_kernel(PoolView pv, TensorArgs a, const __nv_bfloat16 *__restrict__ 
         if (!ok) break;
         // ---- epilogue: the unit's rows leave TMEM; group 0 folds group 1's accumulator into its own
         // (the query a final unit's row belongs to: asked for before the wait, which outlasts the load)
-        const int qn_row = (grp == 0 && dest < 0 && active) ? __ldg(plan + a.off_tq + ~dest + row / G) : 0;
+        const int qn_row = (grp == 0 && dest < 0 && active) ? __ldg(plan + a.off_tq + ~dest + div_g(row)) : 0;
         if (!warp_wait_or_abort(bar + 8 * B_OFULL, uc & 1, abort_flag, limit)) { ok = false; break; }
         tc_fence_after();
         if (grp == 1) {
@@ -713,7 +715,7 @@ attn_tensor_kernel(PoolView pv, TensorArgs a, const __nv_bfloat16 *__restrict__ 
           float inv = 1.f;
           if (fin) {
             if (active) {
-              orow = (static_cast<int64_t>(ll) * a.n_queries + qn_row) * pv.n_q_heads + x.g * G + (row - (row / G) * G);
+              orow = (static_cast<int64_t>(ll) * a.n_queries + qn_row) * pv.n_q_heads + x.g * G + (row - div_g(row) * G);
               inv = l_all > 0.f ? 1.f / l_all : 0.f;
               if (a.lse) a.lse[orow] = (m_all + log2f(l_all)) * 0.6931471805599453f;
             }
