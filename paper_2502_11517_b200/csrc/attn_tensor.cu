@@ -371,8 +371,8 @@ attn_tensor_kernel(PoolView pv, TensorArgs a, const __nv_bfloat16 *__restrict__ 
     mbar_init(bar + 8 * B_QFULL, 2);
     mbar_init(bar + 8 * B_QFREE, 1);
     mbar_init(bar + 8 * B_OFULL, 1);
-    mbar_init(bar + 8 * B_OFREE, 4);
-    mbar_init(bar + 8 * B_MLFULL, 4);
+    mbar_init(bar + 8 * B_OFREE, 8);       // one arrival per softmax warp, of both groups
+    mbar_init(bar + 8 * B_MLFULL, 8);
     mbar_init(bar + 8 * B_DRAIN, 1);
     misc[1] = 0;
     misc[2] = 0;
@@ -688,24 +688,33 @@ attn_tensor_kernel(PoolView pv, TensorArgs a, const __nv_bfloat16 *__restrict__ 
           if (lane == 0) mbar_arrive(bar + 8 * (B_PFULL + 2 * b + grp));
         }
         if (!ok) break;
-        // ---- epilogue: the unit's rows leave TMEM; group 0 folds group 1's accumulator into its own
+        // ---- epilogue: the unit's rows leave TMEM as f0 O_0 + f1 O_1, the two groups' accumulators brought to one
+        // reference.  The groups hand each other their (m_ref, l) through shared memory.  A unit of up to 64 rows
+        // (`low`; its rows sit in the first 64 entries, so the table holds both groups') is written out by both groups,
+        // 64 columns each: the time from a unit's last P.V to the next unit's first is mostly this epilogue.  A higher
+        // unit is written out by group 0 alone.
+        const bool low = m64;
         // (the query a final unit's row belongs to: asked for before the wait, which outlasts the load)
-        const int qn_row = (grp == 0 && dest < 0 && active) ? __ldg(plan + a.off_tq + ~dest + div_g(row)) : 0;
+        const int qn_row = ((grp == 0 || low) && dest < 0 && active) ? __ldg(plan + a.off_tq + ~dest + div_g(row)) : 0;
         if (!warp_wait_or_abort(bar + 8 * B_OFULL, uc & 1, abort_flag, limit)) { ok = false; break; }
         tc_fence_after();
-        if (grp == 1) {
-          if (active) ml1[row] = make_float2(m_ref, l);
-          __syncwarp();
-          if (lane == 0) mbar_arrive(bar + 8 * B_MLFULL);
+        if (active && (grp == 1 || low)) ml1[(grp == 0 ? 64 : 0) + row] = make_float2(m_ref, l);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar + 8 * B_MLFULL);
+        if (grp == 1 && !low) {                 // nothing to read out of TMEM
+          if (lane == 0) mbar_arrive(bar + 8 * B_OFREE);
           continue;
         }
         if (!warp_wait_or_abort(bar + 8 * B_MLFULL, uc & 1, abort_flag, limit)) { ok = false; break; }
         if (warp_active) {
-          const float2 other = active ? ml1[row] : make_float2(-INFINITY, 0.f);
-          const float m_all = fmaxf(m_ref, other.x);
-          const float f0 = l > 0.f ? fast_exp2(m_ref - m_all) : 0.f;
-          const float f1 = other.y > 0.f ? fast_exp2(other.x - m_all) : 0.f;
-          const float l_all = f0 * l + f1 * other.y;
+          const float2 other = active ? ml1[(grp == 0 ? 0 : 64) + row] : make_float2(-INFINITY, 0.f);
+          // accumulator 0 is group 0's, accumulator 1 group 1's; both groups get the same factors from the same values
+          const float m0 = grp == 0 ? m_ref : other.x, l0 = grp == 0 ? l : other.y;
+          const float m1 = grp == 0 ? other.x : m_ref, l1 = grp == 0 ? other.y : l;
+          const float m_all = fmaxf(m0, m1);
+          const float f0 = l0 > 0.f ? fast_exp2(m0 - m_all) : 0.f;
+          const float f1 = l1 > 0.f ? fast_exp2(m1 - m_all) : 0.f;
+          const float l_all = f0 * l0 + f1 * l1;
           const bool any0 = __any_sync(0xffffffffu, f0 != 0.f), any1 = __any_sync(0xffffffffu, f1 != 0.f);
           // a final unit's rows are the result: normalised and written to the output here, with the arithmetic the
           // merge applies to a row that has a single partial (weight 1, then times 1 / l)
@@ -717,9 +726,9 @@ attn_tensor_kernel(PoolView pv, TensorArgs a, const __nv_bfloat16 *__restrict__ 
             if (active) {
               orow = (static_cast<int64_t>(ll) * a.n_queries + qn_row) * pv.n_q_heads + x.g * G + (row - div_g(row) * G);
               inv = l_all > 0.f ? 1.f / l_all : 0.f;
-              if (a.lse) a.lse[orow] = (m_all + log2f(l_all)) * 0.6931471805599453f;
+              if (a.lse && grp == 0) a.lse[orow] = (m_all + log2f(l_all)) * 0.6931471805599453f;
             }
-          } else if (active) {
+          } else if (active && grp == 0) {
             pv.part_ml[prow] = make_float2(m_all, l_all);
           }
           const bool write = active && (fin || l_all > 0.f);      // an output row with nothing visible is written as zeros
@@ -733,8 +742,9 @@ attn_tensor_kernel(PoolView pv, TensorArgs a, const __nv_bfloat16 *__restrict__ 
           const float g0 = f0 * inv, g1 = f1 * inv;
           const bool both = __all_sync(0xffffffffu, !active || (f0 != 0.f && f1 != 0.f));
           const bool only0 = !both && __all_sync(0xffffffffu, !active || (f0 != 0.f && f1 == 0.f));
+          const int cb0 = low ? grp * 4 : 0, cb1 = low ? cb0 + 4 : 8;
 #pragma unroll 1
-          for (int cb = 0; cb < 8; ++cb) {
+          for (int cb = cb0; cb < cb1; ++cb) {
             // 16 columns of both accumulators in flight before one wait
             uint32_t q0[16], q1[16];
             if (any0) tmem_ld16_issue(tmem + lane_addr + COL_O + cb * 16, q0);
