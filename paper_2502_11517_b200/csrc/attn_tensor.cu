@@ -11,7 +11,8 @@
 //
 // The two halves h of a tile (pages 0-3 and 4-7) belong to two softmax groups.  Each group has its own running
 // reference m_ref, sum l and accumulator O_h, so the groups exchange nothing until the unit's epilogue, where
-// group 0 folds both accumulators into one partial row.  m_ref is raised only when a half tile's maximum exceeds
+// the two accumulators are folded into one row on their way out of TMEM: a partial row (m, l, O) for the merge kernel,
+// or, for a unit that covers its whole (request, kv head) run, the normalised output row itself.  m_ref is raised only when a half tile's maximum exceeds
 // it by more than 2^8 (then O_h and l are rescaled in TMEM).  P overwrites the first 32 columns of the scores it
 // was computed from; S is double-buffered so that Q.K^T of the next tile runs during the softmax of this one.
 //
@@ -359,8 +360,9 @@ attn_tensor_kernel(PoolView pv, TensorArgs a, const __nv_bfloat16 *__restrict__ 
   const int u0 = plan[a.off_tcta + 2 * blockIdx.x], u1 = plan[a.off_tcta + 2 * blockIdx.x + 1];
 
   // ---- set-up.  Operand bytes that no copy fills meet zero weights, so they only have to be finite: the Q builder
-  // writes all 128 rows of every unit, and the producer clears the page slots a partial tile leaves empty the first
-  // time each stage is used (afterwards they hold an earlier tile's keys and values).
+  // writes every row a unit's MMAs read (64 or 128, zeros beyond the unit's last), and the producer clears the page
+  // slots a partial tile leaves empty the first time each stage is used (afterwards they hold an earlier tile's keys
+  // and values).
   if (tid == 0) {
     for (int s = 0; s < T_STAGES; ++s) { mbar_init(bar + 8 * (B_FULL + s), 1); mbar_init(bar + 8 * (B_EMPTY + s), 1); }
     for (int b = 0; b < 2; ++b) {
