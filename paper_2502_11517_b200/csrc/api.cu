@@ -463,9 +463,11 @@ pasta_status_t pasta_decode_attn(pasta_pool_t *p, int32_t layer_begin, int32_t l
       mask |= 2;
     }
     if (timed) PASTA_CUDA(cudaEventRecord(ev[2], st));
-    PASTA_CUDA(launch_merge(p->pv, p->hdr, cnt, og, lg, st, out_bf16));
-    p->launches += 1;
-    mask |= 4;
+    if (plan_needs_merge(p->hdr)) {
+      PASTA_CUDA(launch_merge(p->pv, p->hdr, cnt, og, lg, st, out_bf16));
+      p->launches += 1;
+      mask |= 4;
+    }
     if (timed) {
       PASTA_CUDA(cudaEventRecord(ev[3], st));
       p->prof_mask[p->prof_calls++] = mask;

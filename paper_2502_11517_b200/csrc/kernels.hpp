@@ -72,6 +72,10 @@ cudaError_t launch_wait_expiry(const PoolView &pv, cudaStream_t st);
 cudaError_t launch_stream_read(const void *src, size_t bytes, int mode, void *sink, int32_t *status, int sm_count,
                                cudaStream_t st);
 // K4: log-sum-exp merge of all partial rows of every (query, head)
+// False when every row of the step leaves the tensor-core kernel as the output (all its units final, nothing on the
+// warp path): the merge then has nothing to do and is not launched.  A plan with shared units keeps its merge launch,
+// which also puts their counter back to zero.
+inline bool plan_needs_merge(const PlanHeader &h) { return h.w[PH_N_PARTIAL] > 0 || h.w[PH_N_DUNITS] > 0; }
 // out: device fp32 [layer_count, n, Hq, D], or bf16 of the same shape when out_bf16
 cudaError_t launch_merge(const PoolView &pv, const PlanHeader &h, int32_t layer_count, void *out, float *lse,
                          cudaStream_t st, bool out_bf16 = false);

@@ -67,7 +67,7 @@ extern "C" pasta_status_t pasta_decode_attn_noalloc(pasta_pool_t *pool, int32_t 
   int launched = 0;
   if (hdr.w[PH_N_TUNITS] + hdr.w[PH_N_DUNITS] > 0) { e = launch_attn_tensor(pv, hdr, layer, 1, q, sc, out, lse, false, st); ++launched; }
   if (e == cudaSuccess && hdr.w[PH_N_WUNITS] > 0) { e = launch_attn_warp(pv, hdr, layer, 1, q, sc, st); ++launched; }
-  if (e == cudaSuccess) { e = launch_merge(pv, hdr, 1, static_cast<float *>(out), lse, st); ++launched; }
+  if (e == cudaSuccess && plan_needs_merge(hdr)) { e = launch_merge(pv, hdr, 1, static_cast<float *>(out), lse, st); ++launched; }
   pool_count_launches(pool, launched);
   return e == cudaSuccess ? PASTA_OK : PASTA_ERR_CUDA;
 }

@@ -66,6 +66,7 @@ enum {
   PH_N_DUNITS,        // d-units of one layer
   PH_OFF_DUNIT,       // PU_WORDS per d-unit
   PH_OFF_DRANGE,      // per (t-request, kv head): first d-unit, one past the last
+  PH_N_PARTIAL,       // units that leave partial rows for the merge: t-units and d-units that are not final, and all w-units
   PH_WORDS = 32
 };
 

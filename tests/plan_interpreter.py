@@ -8,7 +8,7 @@ import numpy as np
 (PH_MAGIC, PH_N_QUERIES, PH_N_APPEND, PH_N_TREQ, PH_N_TUNITS, PH_N_WUNITS, PH_T_ROWS, PH_ROWS, PH_T_GRID,
  PH_OFF_APPEND, PH_OFF_QUERY, PH_OFF_TREQ, PH_OFF_TRANGE, PH_OFF_TUNIT, PH_OFF_TCTA, PH_OFF_WUNIT, PH_OFF_PAGES,
  PH_OFF_PMETA, PH_OFF_VIS, PH_OFF_TQ, PH_OFF_APOS, PH_OFF_QPOS, PH_TOTAL_WORDS, PH_N_DUNITS, PH_OFF_DUNIT,
- PH_OFF_DRANGE) = range(26)
+ PH_OFF_DRANGE, PH_N_PARTIAL) = range(27)
 PQ, PT, PU, PW = 4, 6, 12, 4
 TILE_PAGES, PAGE = 8, 16
 STATS = {'flagged': 0, 'pages': 0}    # pages the plans marked as visible in full to every thread, of all pages walked
@@ -38,6 +38,9 @@ def run_plan(w, K, V, q, n_kv_heads):
     covered = {}
     final = set()                           # partial rows that are the whole result of their (query, head) pair
     STATS['final_units'] = STATS.get('final_units', 0) + sum(int(rec[11]) for rec in recs)
+    # the header's count of units that leave partial rows (0 = the library does not launch the merge)
+    assert w[PH_N_PARTIAL] == sum(1 - int(rec[11]) for rec in recs) + w[PH_N_WUNITS]
+    STATS['no_merge_plans'] = STATS.get('no_merge_plans', 0) + int(w[PH_N_PARTIAL] == 0)
     for u, rec in enumerate(recs):
         treq, g, tb, te, row_base = rec[:5]
         T = w[PH_OFF_TREQ] + treq * PT

@@ -120,7 +120,7 @@ def test_kernel_timing_can_sample_every_kth_step(lib):
     r = pool.request_begin()
     g = torch.Generator(device="cuda"); g.manual_seed(5)
     rnd = lambda *shape: torch.randn(shape, generator=g, device="cuda").to(torch.bfloat16)
-    pool.kv_append_run(r, 0, 40, rnd(1, 40, 2, 128), rnd(1, 40, 2, 128))
+    pool.kv_append_run(r, 0, 600, rnd(1, 600, 2, 128), rnd(1, 600, 2, 128))    # five tiles per run: cut, so a merge follows
     q, out = rnd(1, 1, 8, 128), torch.empty((1, 1, 8, 128), dtype=torch.float32, device="cuda")
     for stride, steps, want in ((1, 5, 5), (3, 7, 3), (8, 8, 1)):
         pool.profile_enable(stride)

@@ -341,10 +341,13 @@ def _one_step(lib, script, flags=0, overlap=True, want_lse=True):
         k = torch.stack(ks).cuda(); v = torch.stack(vs).cuda(); q = torch.stack(qs).cuda()
         out = torch.full(q.shape, float("nan"), dtype=torch.bfloat16 if flags & lib.FLAG_OUT_BF16 else torch.float32, device="cuda")
         lse = torch.full(q.shape[:3], float("nan"), dtype=torch.float32, device="cuda") if want_lse else None
+        before = pool.launch_count()
         pool.step_device([e[0] for e in op[1]], [e[1] for e in op[1]], [e[2] for e in op[1]], k, v, q, out, lse)
         torch.cuda.synchronize()
         assert pool.status() == 0
         words = np.array(pool.plan_words())
+        if words[26] == 0 and words[23] == 0:        # nothing to merge: append and attention, no third launch
+            assert pool.launch_count() - before <= 2
         pool.close()
         return out.cpu(), None if lse is None else lse.cpu(), words
     finally:
@@ -393,3 +396,19 @@ def test_launch_overlap_does_not_change_results(lib, maker):
     b = _one_step(lib, script, overlap=False)
     assert torch.equal(a[0], b[0]) and torch.equal(a[1], b[1])
     assert not torch.isnan(a[0]).any() and not torch.isnan(a[1]).any()
+
+
+def test_a_step_with_nothing_to_merge(lib):
+    """Two responses with short contexts: every run is one final unit, the plan counts no unit that leaves partial rows,
+    the library launches no merge kernel, and every output element and log-sum-exp still arrives (none stays NaN) and
+    equals the oracle's."""
+    script = cfg3_batched(2, 2, prefix_range=(20, 40), n_new=1)
+    out, lse, words = _one_step(lib, script)
+    assert words[26] == 0 and words[23] == 0 and words[4] > 0          # nothing partial, no shared units, tensor path
+    ora = OracleReplay(script, layers=[0, 1])
+    last = max(i for i, op in enumerate(script.ops) if op[0] == "step")
+    for i in range(last):
+        ora.apply(i, attend=False)
+    want = ora.apply(last)
+    for l in (0, 1):
+        compare(out[l], lse[l], want[l][0], want[l][1], f"layer {l}")

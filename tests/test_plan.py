@@ -51,7 +51,7 @@ def check_script(script, flags=0, steps=None, tail=None, **kw):
                 continue
             want, want_lse = ora.apply(i)[0]
             w = pool.plan_words()
-            stats["tunits"] += int(w[4]); stats["wunits"] += int(w[5])
+            stats["tunits"] += int(w[4]); stats["wunits"] += int(w[5]); stats["steps"] = stats.get("steps", 0) + 1
             got, got_lse = run_plan(w, K, V, _f64(q), geo.n_kv_heads)
             np.testing.assert_allclose(got, want, rtol=0, atol=1e-11)
             np.testing.assert_allclose(got_lse, want_lse, rtol=0, atol=1e-11)
@@ -155,6 +155,18 @@ def test_final_units_are_marked_and_only_those():
     before = STATS["final_units"]
     stats = check_script(cfg4_long_prefix(2, 3000, 3))            # 16 runs of 24 tiles over 148 CTAs: every run is cut
     assert STATS["final_units"] == before and stats["tunits"] > 16
+
+
+def test_small_steps_are_not_cut():
+    """Two responses with contexts of a few dozen tokens (every run has a CTA of its own and is a tile or two long): the
+    runs stay whole, every unit is final and the plan says that nothing is left to merge.  Ten-tile runs are cut."""
+    from plan_interpreter import STATS
+    before = STATS.get("no_merge_plans", 0)
+    stats = check_script(cfg3_batched(2, 1, prefix_range=(20, 40)))
+    assert STATS["no_merge_plans"] - before == stats["steps"] > 0
+    before = STATS["no_merge_plans"]
+    check_script(cfg2_single_request("a"))
+    assert STATS["no_merge_plans"] == before
 
 
 def test_zz_all_visible_page_flag_is_exercised():
