@@ -198,7 +198,8 @@ pasta_status_t pasta_kv_append(pasta_pool_t *pool, int32_t layer_begin, int32_t 
  * head and scored against all those threads' queries on tensor cores (rows that may not see a page are
  * masked), as long as threads x (n_q_heads / n_kv_heads) <= 128 and the request has at most 4095 streams;
  * other requests and head sizes take a warp-shuffle kernel; a merge kernel combines the partial results
- * (fp32 throughout).
+ * (fp32 throughout).  Where one piece of work covers everything a (query, kv head) pair reads, the tensor-core pass
+ * writes that pair's rows of out and lse itself; a step made of such pieces only launches no merge kernel.
  */
 pasta_status_t pasta_decode_attn(pasta_pool_t *pool, int32_t layer_begin, int32_t layer_count,
                                  const void *q, void *out, float *lse, float scale, void *stream);
