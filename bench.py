@@ -410,8 +410,8 @@ def measure_steady(args, workload, size, steps, warmup, device, rank, world, loc
     e2e = None
     if with_e2e:
         k_h = k_new.cpu().pin_memory(); v_h = v_new.cpu().pin_memory(); q_h = q.cpu().pin_memory()
-        out_h = [torch.empty(q.shape, dtype=out_dtype).pin_memory() for _ in range(2)]
-        staging = torch.empty(2 * pool.step_host_bytes(n), dtype=torch.uint8, device=device)
+        out_h = [torch.empty(q.shape, dtype=out_dtype).pin_memory() for _ in range(3)]
+        staging = torch.empty(3 * pool.step_host_bytes(n), dtype=torch.uint8, device=device)
         for _ in range(3):
             pool.step_host(reqs, thr, ones, k_h, v_h, q_h, out_h[0], staging)
         torch.cuda.synchronize(device)
@@ -422,14 +422,15 @@ def measure_steady(args, workload, size, steps, warmup, device, rank, world, loc
         for _ in range(e2e_steps):
             pool.step_host(reqs, thr, ones, k_h, v_h, q_h, out_h[0], staging)
         serial_s = time.perf_counter() - t0
-        # (b) two steps in flight: the copies of a step overlap the kernels of its neighbour
+        # (b) three steps in flight: the copies and the planning of a step overlap the kernels of its neighbours
         torch.cuda.synchronize(device)
         t0 = time.perf_counter()
-        pool.step_host_begin(reqs, thr, ones, k_h, v_h, q_h, out_h[0], staging)
-        for i in range(1, e2e_steps):
-            pool.step_host_begin(reqs, thr, ones, k_h, v_h, q_h, out_h[i & 1], staging)
+        for i in range(e2e_steps):
+            pool.step_host_begin(reqs, thr, ones, k_h, v_h, q_h, out_h[i % 3], staging)
+            if i >= 2:
+                pool.step_host_wait()
+        for _ in range(min(2, e2e_steps)):
             pool.step_host_wait()
-        pool.step_host_wait()
         piped_s = time.perf_counter() - t0
         torch.cuda.synchronize(device)
         assert pool.status() == 0
@@ -437,7 +438,7 @@ def measure_steady(args, workload, size, steps, warmup, device, rank, world, loc
         _, serial_s = aggregate(float(n * e2e_steps), serial_s)
         e2e = {"value": e2e_tokens / piped_s, "unit": UNIT, "h2d_bytes_per_step": k_h.numel() * 2 * 2 + q_h.numel() * 2,
                "d2h_bytes_per_step": out_h[0].numel() * out_h[0].element_size(), "steps": e2e_steps,
-               "how": "pasta_step_host_begin / _wait, two steps in flight, pinned host buffers",
+               "how": "pasta_step_host_begin / _wait, three steps in flight, pinned host buffers",
                "one_step_at_a_time": e2e_tokens / serial_s}
     if sampler:
         sampler.stop(0, 0)

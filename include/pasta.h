@@ -242,15 +242,18 @@ pasta_status_t pasta_step_device(pasta_pool_t *pool, int32_t n, const int32_t *r
  */
 pasta_status_t pasta_step_host_bytes(pasta_pool_t *pool, int32_t n, size_t *out);
 /*
- * The same step in two halves, so that a caller can keep two steps in flight (Section 3: the decode loop is one
- * step after the other; what overlaps here are the copies of one step with the kernels of its neighbour).
+ * The same step in two halves, so that a caller can keep two or three steps in flight (Section 3: the decode loop is
+ * one step after the other; what overlaps here are the copies and the host's planning of one step with the kernels of
+ * its neighbours).
  * pasta_step_host_begin enqueues everything pasta_step_host does (the input copies and the copy of `out` back to
  * the host run on streams of the pool's own, ordered with `stream` by events) and returns without waiting;
  * pasta_step_host_wait blocks until the OLDEST step begun and not yet waited for has delivered its `out`.
  * k_new, v_new, q and out must stay untouched between the two calls.  At most two steps may be begun and not
- * waited for (a third begin: BAD_STATE, as is a wait with nothing begun).  With `staging_bytes` of at least twice
- * pasta_step_host_bytes the inputs of a step are copied while the step before still computes; with less, the
- * copies wait for that step to leave the area.  Pinned host memory is required for any overlap.
+ * waited for, three when `staging_bytes` is at least three times pasta_step_host_bytes (one begin more: BAD_STATE, as
+ * is a wait with nothing begun).  With `staging_bytes` of at least twice pasta_step_host_bytes the inputs of a step
+ * are copied while the step before still computes; with less, the copies wait for that step to leave the area.  With
+ * three steps in flight the host never waits for a step's outputs to cross the bus before it plans the next but one.
+ * Pinned host memory is required for any overlap; use the same staging area and size for all steps in flight.
  */
 pasta_status_t pasta_step_host_begin(pasta_pool_t *pool, int32_t n, const int32_t *req_ids,
                                      const int32_t *thread_ids, const int32_t *n_new,

@@ -15,6 +15,7 @@ using namespace pasta;
 namespace {
 
 constexpr int kStaging = 4;           // pinned upload buffers in rotation
+constexpr int kHostInflight = 3;           // host-buffer steps that may be between begin and wait
 constexpr size_t kSmallPlanWords = 8192;   // plans up to this size are uploaded in the caller's stream
 constexpr int kProfCalls = 512;        // timed pasta_decode_attn launches kept between two profile reads
 constexpr int kRunChunk = 8192;       // tokens whose slots are uploaded at once by pasta_kv_append_run
@@ -101,10 +102,11 @@ struct pasta_pool {
   int32_t tail_percent = kTailPercent, tail_tiles = kTailTiles;
   // pasta_step_host_begin / _wait: at most two steps in flight; their copies run on streams of the pool
   cudaStream_t d2h_stream = nullptr;
-  cudaEvent_t host_inputs_ready[2] = {nullptr, nullptr};   // copy_stream: k / v / q of the step are on the device
-  cudaEvent_t host_attn_done[2] = {nullptr, nullptr};      // caller's stream: the step's outputs are in the staging area
-  cudaEvent_t host_out_ready[2] = {nullptr, nullptr};      // d2h_stream: the outputs are in the caller's host buffer
-  int host_slot_of[2] = {0, 0};                            // staging slot used by the step with event slot e
+  // pasta_step_host_begin / _wait: up to kHostInflight steps between begin and wait; step i uses event set i % kHostInflight
+  cudaEvent_t host_inputs_ready[kHostInflight] = {};       // copy_stream: k / v / q of the step are on the device
+  cudaEvent_t host_attn_done[kHostInflight] = {};          // caller's stream: the step's outputs are in the staging area
+  cudaEvent_t host_out_ready[kHostInflight] = {};          // d2h_stream: the outputs are in the caller's host buffer
+  int host_slot_of[kHostInflight] = {};                    // staging slot used by the step with that event set
   int64_t host_submitted = 0, host_waited = 0;
   // kernel timing (pasta_profile_*): events[4 * i .. 4 * i + 3] bracket the three kernels of call i
   bool profiling = false;
@@ -228,7 +230,9 @@ pasta_status_t pasta_pool_create(const pasta_pool_config_t *cfg, pasta_pool_t **
     for (int b = 0; b < 2 && e == cudaSuccess; ++b) {
       e = cudaEventCreateWithFlags(&p->plan_ready[b], cudaEventDisableTiming);
       if (e == cudaSuccess) e = cudaEventCreateWithFlags(&p->work_mark[b], cudaEventDisableTiming);
-      if (e == cudaSuccess) e = cudaEventCreateWithFlags(&p->host_inputs_ready[b], cudaEventDisableTiming);
+    }
+    for (int b = 0; b < kHostInflight && e == cudaSuccess; ++b) {
+      e = cudaEventCreateWithFlags(&p->host_inputs_ready[b], cudaEventDisableTiming);
       if (e == cudaSuccess) e = cudaEventCreateWithFlags(&p->host_attn_done[b], cudaEventDisableTiming);
       if (e == cudaSuccess) e = cudaEventCreateWithFlags(&p->host_out_ready[b], cudaEventDisableTiming);
     }
@@ -274,6 +278,8 @@ pasta_status_t pasta_pool_destroy(pasta_pool_t *p) {
   for (int b = 0; b < 2; ++b) {
     if (p->plan_ready[b]) cudaEventDestroy(p->plan_ready[b]);
     if (p->work_mark[b]) cudaEventDestroy(p->work_mark[b]);
+  }
+  for (int b = 0; b < kHostInflight; ++b) {
     if (p->host_inputs_ready[b]) cudaEventDestroy(p->host_inputs_ready[b]);
     if (p->host_attn_done[b]) cudaEventDestroy(p->host_attn_done[b]);
     if (p->host_out_ready[b]) cudaEventDestroy(p->host_out_ready[b]);
@@ -551,11 +557,15 @@ pasta_status_t pasta_step_host_begin(pasta_pool_t *p, int32_t n, const int32_t *
                                      void *staging, size_t staging_bytes, float scale, void *stream) {
   if (!p || !q || !out || !staging) return PASTA_ERR_INVALID_ARG;
   if (p->host_only) return PASTA_ERR_BAD_STATE;
-  if (p->host_submitted - p->host_waited >= 2) return PASTA_ERR_BAD_STATE;      // two steps are in flight already
   size_t need = 0;
   pasta_status_t s = pasta_step_host_bytes(p, n, &need);
   if (s != PASTA_OK) return s;
   if (staging_bytes < need || (reinterpret_cast<uintptr_t>(staging) & 255)) return PASTA_ERR_INVALID_ARG;
+  // A staging area of twice (three times) the size holds two (three) steps: the inputs of this step then travel while
+  // the kernels of the steps before still read theirs.  Two steps may be in flight in any case (with one slot the
+  // copies wait until the step before has left the area), three when the area holds three.
+  const int n_slots = static_cast<int>(std::min<size_t>(kHostInflight, staging_bytes / need));
+  if (p->host_submitted - p->host_waited >= std::max(2, n_slots)) return PASTA_ERR_BAD_STATE;   // no room for another step
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   size_t n_app = static_cast<size_t>(n);
   if (n_new) {
@@ -566,13 +576,9 @@ pasta_status_t pasta_step_host_begin(pasta_pool_t *p, int32_t n, const int32_t *
     }
   }
   if (n_app > 0 && (!k_new || !v_new)) return PASTA_ERR_INVALID_ARG;
-  // A staging area of twice the size holds two steps: the inputs of this step then travel while the kernels of the
-  // step before still read theirs.  With one slot the copies wait until that step has left the area.
-  const int n_slots = staging_bytes >= 2 * need ? 2 : 1;
   const int64_t i = p->host_submitted;
-  const int e = static_cast<int>(i & 1);
-  int slot = 0;
-  if (i > p->host_waited) slot = n_slots == 2 ? p->host_slot_of[e ^ 1] ^ 1 : 0;
+  const int e = static_cast<int>(i % kHostInflight);
+  const int slot = static_cast<int>(i % n_slots);
   const size_t L = p->cfg.n_layers, d = p->cfg.head_dim;
   const size_t kv_full = align_up(L * n * p->cfg.n_kv_heads * d * 2, 256);
   const size_t kv_bytes = L * n_app * p->cfg.n_kv_heads * d * 2;
@@ -580,9 +586,11 @@ pasta_status_t pasta_step_host_begin(pasta_pool_t *p, int32_t n, const int32_t *
   uint8_t *base = static_cast<uint8_t *>(staging) + size_t(slot) * need;
   uint8_t *k_dev = base, *v_dev = base + kv_full, *q_dev = base + 2 * kv_full;
   uint8_t *o_dev = q_dev + align_up(q_bytes, 256);
-  // the input copies go first, on the pool's copy stream: the host plans the step while they are in flight.  The
-  // step in flight (if any) is done with the slot once its outputs have reached the host, when it shares the slot.
-  if (i > p->host_waited && n_slots == 1) PASTA_CUDA(cudaStreamWaitEvent(p->copy_stream, p->host_out_ready[e ^ 1], 0));
+  // the input copies go first, on the pool's copy stream: the host plans the step while they are in flight.  A step
+  // still in flight that uses the same slot is done with it once its outputs have reached the host.
+  for (int64_t j = p->host_waited; j < i; ++j)
+    if (p->host_slot_of[j % kHostInflight] == slot)
+      PASTA_CUDA(cudaStreamWaitEvent(p->copy_stream, p->host_out_ready[j % kHostInflight], 0));
   if (n_app > 0) {
     PASTA_CUDA(cudaMemcpyAsync(k_dev, k_new, kv_bytes, cudaMemcpyHostToDevice, p->copy_stream));
     PASTA_CUDA(cudaMemcpyAsync(v_dev, v_new, kv_bytes, cudaMemcpyHostToDevice, p->copy_stream));
@@ -609,7 +617,7 @@ pasta_status_t pasta_step_host_begin(pasta_pool_t *p, int32_t n, const int32_t *
 pasta_status_t pasta_step_host_wait(pasta_pool_t *p) {
   if (!p) return PASTA_ERR_INVALID_ARG;
   if (p->host_only || p->host_waited == p->host_submitted) return PASTA_ERR_BAD_STATE;
-  PASTA_CUDA(cudaEventSynchronize(p->host_out_ready[p->host_waited & 1]));
+  PASTA_CUDA(cudaEventSynchronize(p->host_out_ready[p->host_waited % kHostInflight]));
   p->host_waited += 1;
   return PASTA_OK;
 }

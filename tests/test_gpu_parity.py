@@ -256,16 +256,17 @@ def test_step_host_entry_point(lib):
     pool.close()
 
 
-@pytest.mark.parametrize("slots", [1, 2])
+@pytest.mark.parametrize("slots", [1, 2, 3])
 def test_step_host_in_two_halves_keeps_two_steps_in_flight(lib, slots):
-    """pasta_step_host_begin / _wait: four appending steps, the next one begun before the previous one is waited for;
-    every step's output against the oracle, with a staging area for one step and for two."""
+    """pasta_step_host_begin / _wait: five appending steps, the next ones begun before the previous ones are waited for
+    (two in flight; three with a staging area for three steps); every step's output against the oracle, with a staging
+    area for one, two and three steps."""
     import torch
     from lib_replay import LibReplay, make_pool
     script = cfg2_single_request("a")
     first = next(i for i, op in enumerate(script.ops) if op[0] == "step")
     entries = tuple((r, t, 1) for r, t, _ in script.ops[first][1])
-    script.ops = script.ops[:first] + [("step", entries)] * 4
+    script.ops = script.ops[:first] + [("step", entries)] * 5
     pool = make_pool(script); rep = LibReplay(script, pool)
     ora = OracleReplay(script)
     for i in range(first):
@@ -274,7 +275,7 @@ def test_step_host_in_two_halves_keeps_two_steps_in_flight(lib, slots):
     staging = torch.empty(slots * pool.step_host_bytes(n), dtype=torch.uint8, device="cuda")
     reqs = [e[0] for e in entries]; thr = [e[1] for e in entries]; nn = [e[2] for e in entries]
     bufs = []
-    for i in range(first, first + 4):
+    for i in range(first, first + 5):
         k, v, q = step_tensors(script, i, 0)
         bufs.append([t.unsqueeze(0).contiguous().pin_memory() for t in (k, v, q)] +
                     [torch.full((1,) + tuple(q.shape), float("nan"), dtype=torch.float32).pin_memory()])
@@ -285,15 +286,18 @@ def test_step_host_in_two_halves_keeps_two_steps_in_flight(lib, slots):
         err = np.abs(bufs[j][3][0].double().numpy() - want[0])
         assert err.max() <= MAX_ABS and err.mean() <= MEAN_ABS, (j, err.max())
 
-    for j in range(4):
+    depth = max(2, slots)                             # steps that may be in flight
+    waited = 0
+    for j in range(5):
         pool.step_host_begin(reqs, thr, nn, bufs[j][0], bufs[j][1], bufs[j][2], bufs[j][3], staging)
-        if j == 1:                                    # two in flight: a third begin is refused, nothing changes
+        if j == depth - 1:                            # all in flight: one begin more is refused, nothing changes
             with pytest.raises(lib.PastaError) as e:
-                pool.step_host_begin(reqs, thr, nn, bufs[2][0], bufs[2][1], bufs[2][2], bufs[2][3], staging)
+                pool.step_host_begin(reqs, thr, nn, bufs[j + 1][0], bufs[j + 1][1], bufs[j + 1][2], bufs[j + 1][3], staging)
             assert e.value.code == lib.BAD_STATE
-        if j >= 1:
-            check(j - 1)
-    check(3)
+        if j >= depth - 1:
+            check(waited); waited += 1
+    while waited < 5:
+        check(waited); waited += 1
     with pytest.raises(lib.PastaError) as e:
         pool.step_host_wait()
     assert e.value.code == lib.BAD_STATE
